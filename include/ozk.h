@@ -1,0 +1,167 @@
+/*
+ * ozk — FP64 GEMM emulated on NVIDIA B200 FP4 tensor cores by Ozaki scheme II on
+ * base-13 E2M1 limbs, and bit-exact INT8 GEMM on the same limbs.
+ *
+ * C ABI.  Every matrix pointer is a DEVICE pointer owned by the caller; matrices are
+ * column-major (element (r,c) at ptr[r + c*ld]).  `stream` is a cudaStream_t passed as
+ * void* (NULL = the legacy default stream).  Compute calls enqueue work on `stream` and
+ * return without synchronising; they allocate no memory.  All scratch lives in ONE
+ * caller-owned device workspace registered with ozk_set_workspace(); calls that share
+ * the workspace must be ordered by the caller (same stream, or events).
+ *
+ * Errors.  Argument errors are returned synchronously and enqueue nothing.
+ * Data-dependent conditions (a NaN/Inf input, a bounded device wait that expired) are
+ * recorded in a status word inside the workspace and reported by
+ * ozk_get_async_status(), which synchronises the stream.  After OZK_ERR_NONFINITE or
+ * OZK_ERR_DEVICE_TIMEOUT the output matrix is unspecified.
+ */
+#ifndef OZK_H_
+#define OZK_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int ozk_status;
+enum {
+  OZK_OK = 0,
+  OZK_ERR_INVALID_ARG = -1,    /* null pointer, negative size, ld too small, bad alignment */
+  OZK_ERR_UNSUPPORTED = -2,    /* num_moduli out of range, K beyond an exactness bound, device is not sm_100 */
+  OZK_ERR_WORKSPACE = -3,      /* no workspace registered, or it is too small for this call */
+  OZK_ERR_CUDA = -4,           /* a CUDA runtime/driver call failed (launch, tensor-map encode) */
+  OZK_ERR_NONFINITE = -5,      /* asynchronous: an input element is NaN or Inf */
+  OZK_ERR_DEVICE_TIMEOUT = -6  /* asynchronous: a bounded wait inside a kernel gave up */
+};
+
+enum { OZK_MIN_MODULI = 2, OZK_MAX_MODULI = 27, OZK_DEFAULT_MODULI = 19 };
+
+/* ---------------------------------------------------------------------------------------
+ * Constants of the method (host-side, no GPU needed).
+ * ------------------------------------------------------------------------------------- */
+
+/* Section 5.1: the first `num_moduli` moduli chosen greedily in descending order from 169,
+ * pairwise coprime, 169 the only multiple of 13, every residue class representable by two
+ * limbs c0 + 13 c1 with c0, c1 in S = {0,+-1,+-2,+-3,+-4,+-6,+-8,+-12}.  The first 19 are the
+ * list printed in the paper; 20..27 continue the same rule.  Writes num_moduli ints to
+ * `out` (host memory); returns num_moduli, or OZK_ERR_INVALID_ARG. */
+int ozk_get_moduli(int num_moduli, int* out);
+
+/* Eq. 3 read for a general integer width: the largest c <= 53 with 2*K*2^(2c) < P, P the
+ * product of the first num_moduli moduli.  Inputs are converted to integers of at most c
+ * bits (Section 4.2).  Returns c >= 1, or OZK_ERR_UNSUPPORTED when no c >= 1 exists, or
+ * OZK_ERR_INVALID_ARG. */
+int ozk_capacity_bits(int64_t K, int num_moduli);
+
+/* Section 5.2: the CRT constants for the first num_moduli moduli as little-endian 32-bit
+ * words, 6 words each: P into P_words[6], w_l = (P/m_l) * ((P/m_l)^-1 mod m_l) into
+ * weights[6*l .. 6*l+5] (host memory).  Returns OZK_OK or OZK_ERR_INVALID_ARG. */
+ozk_status ozk_get_crt_constants(int num_moduli, uint32_t* P_words, uint32_t* weights);
+
+const char* ozk_status_string(ozk_status status);
+const char* ozk_version(void);
+
+/* ---------------------------------------------------------------------------------------
+ * Workspace.
+ * ------------------------------------------------------------------------------------- */
+
+/* Bytes of device workspace ozk_dgemm(M,N,K,...,num_moduli) needs: status block, limb-pair
+ * tables, shifts s (rows of A) and t (columns of B), 2*num_moduli E2M1 limb planes per
+ * operand padded to 128 rows x 256 k, and num_moduli residue matrices of one byte per
+ * element of the padded C.  Returns 0 on invalid arguments. */
+size_t ozk_dgemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int num_moduli);
+
+/* Bytes of device workspace ozk_igemm_i8(M,N,K,...) needs (3 limb planes per operand). */
+size_t ozk_igemm_i8_workspace_bytes(int64_t M, int64_t N, int64_t K);
+
+/* Registers the caller-owned device buffer used by all later compute calls of this
+ * process.  `dev_ptr` must be 1024-byte aligned (any cudaMalloc / PyTorch allocation is).
+ * The library never frees it.  Passing NULL unregisters. */
+ozk_status ozk_set_workspace(void* dev_ptr, size_t bytes);
+
+/* Synchronises `stream`, then reads and clears the status word in the workspace.
+ * Returns OZK_OK, OZK_ERR_NONFINITE, OZK_ERR_DEVICE_TIMEOUT, OZK_ERR_WORKSPACE or OZK_ERR_CUDA. */
+ozk_status ozk_get_async_status(void* stream);
+
+/* ---------------------------------------------------------------------------------------
+ * The hot path.
+ * ------------------------------------------------------------------------------------- */
+
+/* Emulated DGEMM, C = A*B with every C_ij the exact product of the integer-converted
+ * inputs rounded once (Sections 4.2, 5; Fig. 3): shared-exponent conversion of the rows
+ * of A and columns of B to integers of ozk_capacity_bits(K, num_moduli) bits, residues
+ * mod each modulus as two base-13 E2M1 limbs, four FP4 limb products per modulus on the
+ * tensor cores with the residue composed in the epilogue, single-pass integer CRT,
+ * inverse scaling, one round-to-nearest-even.
+ *   A: M x K, lda >= max(1,M).  B: K x N, ldb >= max(1,K).  C: M x N, ldc >= max(1,M), overwritten.
+ *   num_moduli in [OZK_MIN_MODULI, OZK_MAX_MODULI]; 19 keeps all 53 bits for K <= 76549.
+ *   K must not exceed 131072 (FP32 accumulators stay exact integers: 128*K <= 2^24 with
+ *   limbs |c| <= 8, Lemma 3 tightened).  M, N, K = 0 are allowed (K = 0 gives C = 0).
+ * Returns OZK_OK once the work is enqueued. */
+ozk_status ozk_dgemm(int64_t M, int64_t N, int64_t K,
+                     const double* A, int64_t lda,
+                     const double* B, int64_t ldb,
+                     double* C, int64_t ldc,
+                     int num_moduli, void* stream);
+
+/* Bit-exact INT8 x INT8 -> INT32 GEMM on FP4 tensor cores (Section 3, last paragraph;
+ * Eq. 1 with p = q = 3): every int8 becomes three greedy base-13 limbs, nine limb
+ * products are accumulated in five groups i+j = g and combined as sum_g 13^g G_g.
+ *   A: M x K int8, B: K x N int8, C: M x N int32, column-major as above.
+ *   K <= 87381 (three products of magnitude <= 64 share an FP32 accumulator:
+ *   192*K <= 2^24); the int32 result is exact for K <= 131071 anyway. */
+ozk_status ozk_igemm_i8(int64_t M, int64_t N, int64_t K,
+                        const int8_t* A, int64_t lda,
+                        const int8_t* B, int64_t ldb,
+                        int32_t* C, int64_t ldc, void* stream);
+
+/* ---------------------------------------------------------------------------------------
+ * Staged entry points: the same kernels one stage at a time, used by the parity tests.
+ * They use the registered workspace exactly as ozk_dgemm does.
+ * ------------------------------------------------------------------------------------- */
+
+/* Stage 1 (Section 4.2 + Section 5.1): exponent scan, integer conversion, residues,
+ * limb planes.  Optional device outputs (NULL to skip):
+ *   s_out[M], t_out[N]          the shifts s_i, t_j (int32)
+ *   At_out[M*K], Bt_out[K*N]    the converted integers, column-major with ld = M and K (int64)
+ * The limb planes stay in the workspace; ozk_stage_read_planes() copies them out. */
+ozk_status ozk_stage_preprocess(int64_t M, int64_t N, int64_t K,
+                                const double* A, int64_t lda, const double* B, int64_t ldb,
+                                int num_moduli, int32_t* s_out, int32_t* t_out,
+                                int64_t* At_out, int64_t* Bt_out, void* stream);
+
+/* Decodes limb plane (modulus index l, limb 0|1) of operand 'A' or 'B' from the workspace
+ * into doubled-E2M1 integers (int8, values in S): out[r + k*rows], r < rows (M for 'A',
+ * N for 'B'), k < K.  Valid after ozk_stage_preprocess / ozk_dgemm on the same sizes. */
+ozk_status ozk_stage_read_planes(char operand, int64_t M, int64_t N, int64_t K, int num_moduli,
+                                 int l, int limb, int8_t* out, void* stream);
+
+/* Stage 2 (Section 5.1, Section 6.4): the limb GEMM with residue composition, on the
+ * planes in the workspace.  residues_out (optional, device): num_moduli matrices of
+ * M x N bytes, column-major with ld = M, r_l = (A~ B~) mod m_l in [0, m_l). */
+ozk_status ozk_stage_residue_gemm(int64_t M, int64_t N, int64_t K, int num_moduli,
+                                  uint8_t* residues_out, void* stream);
+
+/* Stage 3 (Section 5.2 + Section 4.2): direct CRT, symmetric representative, inverse
+ * scaling, one rounding.  residues_in (optional, device; same layout as residues_out): if
+ * given together with s_in[M], t_in[N], the stage runs on them instead of the workspace
+ * contents.  x_out (optional, device): the reconstructed integer of every element as
+ * 6 little-endian 32-bit words, two's complement, element (i,j) at x_out[6*(i + j*M)]. */
+ozk_status ozk_stage_crt(int64_t M, int64_t N, int64_t K, int num_moduli,
+                         const uint8_t* residues_in, const int32_t* s_in, const int32_t* t_in,
+                         double* C, int64_t ldc, uint32_t* x_out, void* stream);
+
+/* One tcgen05.mma.kind::mxf4.block_scale instruction sequence on caller-supplied packed
+ * E2M1 operands, used to pin the hardware byte formats (nibble order, E2M1 codes, UE8M0
+ * scale byte, FP32 accumulator exactness): D[128 x 128] (FP32, row-major, device) =
+ * scale^2 * sum_k P[r,k] Q[c,k], P and Q being 128 x K nibbles, K-contiguous, two per byte,
+ * K a multiple of 256.  scale_byte is the UE8M0 byte given to every block of both operands. */
+ozk_status ozk_stage_mma_probe(const uint8_t* P, const uint8_t* Q, int64_t K, int scale_byte,
+                               float* D, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* OZK_H_ */

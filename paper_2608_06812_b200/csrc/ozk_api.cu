@@ -1,0 +1,256 @@
+// C-ABI entry points of the ozk library: argument checks, workspace layout, stage sequencing.
+#include <stdio.h>
+#include <string.h>
+
+#include "ozk_common.cuh"
+
+namespace ozk {
+namespace {
+
+struct Workspace {
+  uint8_t* ptr = nullptr;
+  size_t bytes = 0;
+};
+Workspace g_ws;
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Workspace layout for an (M, N, K, L) problem.  Returns false on invalid sizes.
+bool make_geometry(int64_t M, int64_t N, int64_t K, int L, Geometry* g) {
+  if (M < 0 || N < 0 || K < 0 || L < OZK_MIN_MODULI || L > OZK_MAX_MODULI) return false;
+  memset(g, 0, sizeof *g);
+  g->M = M;
+  g->N = N;
+  g->K = K;
+  g->L = L;
+  g->Mp = round_up(M > 0 ? M : 1, kTileRows);
+  g->Np = round_up(N > 0 ? N : 1, kTileRows);
+  g->Kp = round_up(K > 0 ? K : 1, kTileKNibbles);
+  g->c_bits = host_capacity_bits(K, L);
+  size_t off = 0;
+  g->off_status = off;
+  off += align_up(sizeof(StatusBlock), 1024);
+  g->off_lut = off;
+  off += align_up((size_t)kMaxModuli * kLutStride, 1024);
+  g->off_amax_a = off;
+  off += (size_t)g->Mp * 8;
+  g->off_amax_b = off;  // must follow amax_a directly: both are cleared by one memset
+  off += (size_t)g->Np * 8;
+  off = align_up(off, 1024);
+  g->off_s = off;
+  off += align_up((size_t)g->Mp * 4, 1024);
+  g->off_t = off;
+  off += align_up((size_t)g->Np * 4, 1024);
+  g->plane_bytes_a = (size_t)g->Mp * (size_t)(g->Kp / 2);
+  g->plane_bytes_b = (size_t)g->Np * (size_t)(g->Kp / 2);
+  g->off_planes_a = off;
+  off += 2 * (size_t)L * g->plane_bytes_a;
+  g->off_planes_b = off;
+  off += 2 * (size_t)L * g->plane_bytes_b;
+  g->off_res = off;
+  off += (size_t)L * (size_t)g->Mp * (size_t)g->Np;
+  g->total = align_up(off, 1024);
+  return true;
+}
+
+ozk_status check_common(int64_t M, int64_t N, int64_t K, int L, Geometry* g) {
+  if (!make_geometry(M, N, K, L, g)) return OZK_ERR_INVALID_ARG;
+  if (K > 131072) return OZK_ERR_UNSUPPORTED;  // 128 K <= 2^24 with |limb| <= 8
+  if (g->c_bits < 1) return OZK_ERR_UNSUPPORTED;
+  if (N > 65535 || g->Mp / 32 > 65535) return OZK_ERR_UNSUPPORTED;  // grid-dimension limits of the O(N^2) kernels
+  if (!g_ws.ptr) return OZK_ERR_WORKSPACE;
+  if (g_ws.bytes < g->total) return OZK_ERR_WORKSPACE;
+  return OZK_OK;
+}
+
+bool device_is_sm100() {
+  static int cached = -1;
+  if (cached < 0) {
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return false;
+    cached = (major == 10) ? 1 : 0;
+  }
+  return cached == 1;
+}
+
+ozk_status run_preprocess(const Geometry& g, const ModulusTable& mt, const double* A, int64_t lda, const double* B,
+                          int64_t ldb, int64_t* At_out, int64_t* Bt_out, cudaStream_t st) {
+  if (launch_build_lut(mt, g_ws.ptr + g.off_lut, st) != cudaSuccess) return OZK_ERR_CUDA;
+  if (launch_scan_and_shifts(g, A, lda, B, ldb, g_ws.ptr, st) != cudaSuccess) return OZK_ERR_CUDA;
+  if (launch_encode(g, mt, A, lda, B, ldb, g_ws.ptr, At_out, Bt_out, st) != cudaSuccess) return OZK_ERR_CUDA;
+  return OZK_OK;
+}
+
+}  // namespace
+}  // namespace ozk
+
+using namespace ozk;
+
+extern "C" {
+
+int ozk_get_moduli(int num_moduli, int* out) {
+  if (!out || num_moduli < 1 || num_moduli > OZK_MAX_MODULI) return OZK_ERR_INVALID_ARG;
+  return host_select_moduli(num_moduli, out) == num_moduli ? num_moduli : OZK_ERR_INVALID_ARG;
+}
+
+int ozk_capacity_bits(int64_t K, int num_moduli) {
+  if (K < 0 || num_moduli < 1 || num_moduli > OZK_MAX_MODULI) return OZK_ERR_INVALID_ARG;
+  const int c = host_capacity_bits(K, num_moduli);
+  return c >= 1 ? c : OZK_ERR_UNSUPPORTED;
+}
+
+ozk_status ozk_get_crt_constants(int num_moduli, uint32_t* P_words, uint32_t* weights) {
+  CrtTable ct;
+  if (!P_words || !weights || !host_build_crt_table(num_moduli, &ct)) return OZK_ERR_INVALID_ARG;
+  memcpy(P_words, ct.P, sizeof ct.P);
+  for (int l = 0; l < num_moduli; ++l) memcpy(weights + kCrtWords * l, ct.w[l], sizeof ct.w[l]);
+  return OZK_OK;
+}
+
+const char* ozk_status_string(ozk_status s) {
+  switch (s) {
+    case OZK_OK: return "ok";
+    case OZK_ERR_INVALID_ARG: return "invalid argument";
+    case OZK_ERR_UNSUPPORTED: return "unsupported size, modulus count or device";
+    case OZK_ERR_WORKSPACE: return "workspace missing or too small";
+    case OZK_ERR_CUDA: return "CUDA call failed";
+    case OZK_ERR_NONFINITE: return "non-finite input element";
+    case OZK_ERR_DEVICE_TIMEOUT: return "bounded device wait expired";
+    default: return "unknown status";
+  }
+}
+
+const char* ozk_version(void) { return "ozk 0.1 (sm_100a)"; }
+
+size_t ozk_dgemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int num_moduli) {
+  Geometry g;
+  return make_geometry(M, N, K, num_moduli, &g) ? g.total : 0;
+}
+
+ozk_status ozk_set_workspace(void* dev_ptr, size_t bytes) {
+  if (dev_ptr && (reinterpret_cast<uintptr_t>(dev_ptr) & 1023)) return OZK_ERR_INVALID_ARG;
+  g_ws.ptr = static_cast<uint8_t*>(dev_ptr);
+  g_ws.bytes = dev_ptr ? bytes : 0;
+  if (dev_ptr) {
+    if (bytes < sizeof(StatusBlock)) return OZK_ERR_WORKSPACE;
+    if (cudaMemset(dev_ptr, 0, sizeof(StatusBlock)) != cudaSuccess) return OZK_ERR_CUDA;
+  }
+  return OZK_OK;
+}
+
+ozk_status ozk_get_async_status(void* stream) {
+  if (!g_ws.ptr) return OZK_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaStreamSynchronize(st) != cudaSuccess) return OZK_ERR_CUDA;
+  StatusBlock sb;
+  if (cudaMemcpy(&sb, g_ws.ptr, sizeof sb, cudaMemcpyDeviceToHost) != cudaSuccess) return OZK_ERR_CUDA;
+  if (sb.code != 0) {
+    if (sb.code == OZK_ERR_DEVICE_TIMEOUT) fprintf(stderr, "ozk: bounded wait expired at 0x%x\n", sb.where);
+    cudaMemset(g_ws.ptr, 0, sizeof(StatusBlock));
+  }
+  return sb.code;
+}
+
+ozk_status ozk_stage_preprocess(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, const double* B,
+                                int64_t ldb, int num_moduli, int32_t* s_out, int32_t* t_out, int64_t* At_out,
+                                int64_t* Bt_out, void* stream) {
+  Geometry g;
+  ozk_status rc = check_common(M, N, K, num_moduli, &g);
+  if (rc != OZK_OK) return rc;
+  if (M == 0 || N == 0) return OZK_OK;
+  if ((K > 0 && (!A || !B)) || lda < (M > 1 ? M : 1) || ldb < (K > 1 ? K : 1)) return OZK_ERR_INVALID_ARG;
+  ModulusTable mt;
+  if (!host_build_modulus_table(num_moduli, &mt)) return OZK_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  rc = run_preprocess(g, mt, A, lda, B, ldb, At_out, Bt_out, st);
+  if (rc != OZK_OK) return rc;
+  if (s_out && cudaMemcpyAsync(s_out, g_ws.ptr + g.off_s, (size_t)M * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    return OZK_ERR_CUDA;
+  if (t_out && cudaMemcpyAsync(t_out, g_ws.ptr + g.off_t, (size_t)N * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    return OZK_ERR_CUDA;
+  return OZK_OK;
+}
+
+ozk_status ozk_stage_read_planes(char operand, int64_t M, int64_t N, int64_t K, int num_moduli, int l, int limb,
+                                 int8_t* out, void* stream) {
+  Geometry g;
+  ozk_status rc = check_common(M, N, K, num_moduli, &g);
+  if (rc != OZK_OK) return rc;
+  if (!out || l < 0 || l >= num_moduli || (limb != 0 && limb != 1) || (operand != 'A' && operand != 'B'))
+    return OZK_ERR_INVALID_ARG;
+  const bool a = operand == 'A';
+  const uint8_t* plane = g_ws.ptr + (a ? g.off_planes_a : g.off_planes_b) + (size_t)(2 * l + limb) * (a ? g.plane_bytes_a : g.plane_bytes_b);
+  return launch_decode_plane(plane, a ? M : N, K, g.Kp, out, static_cast<cudaStream_t>(stream)) == cudaSuccess ? OZK_OK
+                                                                                                                : OZK_ERR_CUDA;
+}
+
+ozk_status ozk_stage_residue_gemm(int64_t M, int64_t N, int64_t K, int num_moduli, uint8_t* residues_out, void* stream) {
+  Geometry g;
+  ozk_status rc = check_common(M, N, K, num_moduli, &g);
+  if (rc != OZK_OK) return rc;
+  if (M == 0 || N == 0) return OZK_OK;
+  if (!device_is_sm100()) return OZK_ERR_UNSUPPORTED;
+  ModulusTable mt;
+  if (!host_build_modulus_table(num_moduli, &mt)) return OZK_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  rc = gemm_residues(g, mt, g_ws.ptr, st);
+  if (rc != OZK_OK) return rc;
+  if (residues_out && launch_copy_residues(g, g_ws.ptr + g.off_res, residues_out, st) != cudaSuccess) return OZK_ERR_CUDA;
+  return OZK_OK;
+}
+
+ozk_status ozk_stage_crt(int64_t M, int64_t N, int64_t K, int num_moduli, const uint8_t* residues_in, const int32_t* s_in,
+                         const int32_t* t_in, double* C, int64_t ldc, uint32_t* x_out, void* stream) {
+  Geometry g;
+  ozk_status rc = check_common(M, N, K, num_moduli, &g);
+  if (rc != OZK_OK) return rc;
+  if (M == 0 || N == 0) return OZK_OK;
+  if (!C || ldc < M) return OZK_ERR_INVALID_ARG;
+  if ((residues_in != nullptr) != (s_in != nullptr) || (s_in != nullptr) != (t_in != nullptr)) return OZK_ERR_INVALID_ARG;
+  CrtTable ct;
+  if (!host_build_crt_table(num_moduli, &ct)) return OZK_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cudaError_t e;
+  if (residues_in)
+    e = launch_crt(g, ct, residues_in, M, (size_t)M * (size_t)N, s_in, t_in, C, ldc, x_out, st);
+  else
+    e = launch_crt(g, ct, g_ws.ptr + g.off_res, g.Mp, (size_t)g.Mp * (size_t)g.Np,
+                   reinterpret_cast<const int32_t*>(g_ws.ptr + g.off_s), reinterpret_cast<const int32_t*>(g_ws.ptr + g.off_t), C,
+                   ldc, x_out, st);
+  return e == cudaSuccess ? OZK_OK : OZK_ERR_CUDA;
+}
+
+ozk_status ozk_dgemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, const double* B, int64_t ldb, double* C,
+                     int64_t ldc, int num_moduli, void* stream) {
+  Geometry g;
+  ozk_status rc = check_common(M, N, K, num_moduli, &g);
+  if (rc != OZK_OK) return rc;
+  if (M == 0 || N == 0) return OZK_OK;
+  if (!C || ldc < M || (K > 0 && (!A || !B)) || lda < (M > 1 ? M : 1) || ldb < (K > 1 ? K : 1)) return OZK_ERR_INVALID_ARG;
+  if (!device_is_sm100()) return OZK_ERR_UNSUPPORTED;
+  ModulusTable mt;
+  CrtTable ct;
+  if (!host_build_modulus_table(num_moduli, &mt) || !host_build_crt_table(num_moduli, &ct)) return OZK_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  rc = run_preprocess(g, mt, A, lda, B, ldb, nullptr, nullptr, st);
+  if (rc != OZK_OK) return rc;
+  rc = gemm_residues(g, mt, g_ws.ptr, st);
+  if (rc != OZK_OK) return rc;
+  if (launch_crt(g, ct, g_ws.ptr + g.off_res, g.Mp, (size_t)g.Mp * (size_t)g.Np,
+                 reinterpret_cast<const int32_t*>(g_ws.ptr + g.off_s), reinterpret_cast<const int32_t*>(g_ws.ptr + g.off_t), C, ldc,
+                 nullptr, st) != cudaSuccess)
+    return OZK_ERR_CUDA;
+  return OZK_OK;
+}
+
+ozk_status ozk_stage_mma_probe(const uint8_t* P, const uint8_t* Q, int64_t K, int scale_byte, float* D, void* stream) {
+  if (!P || !Q || !D || K <= 0 || K % kTileKNibbles != 0) return OZK_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(P) & 15) || (reinterpret_cast<uintptr_t>(Q) & 15)) return OZK_ERR_INVALID_ARG;
+  if (!g_ws.ptr) return OZK_ERR_WORKSPACE;
+  if (!device_is_sm100()) return OZK_ERR_UNSUPPORTED;
+  return gemm_probe(P, Q, K, scale_byte, D, g_ws.ptr, static_cast<cudaStream_t>(stream));
+}
+
+// INT8 path: see ozk_igemm.cu
+}  // extern "C"

@@ -1,0 +1,80 @@
+// Shared declarations of the ozk library: layouts, parameter blocks, status word.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/ozk.h"
+
+namespace ozk {
+
+// ---- tiling constants ---------------------------------------------------------------
+constexpr int kTileRows = 128;       // rows of a limb plane covered by one GEMM tile (either operand)
+constexpr int kTileKNibbles = 256;   // k extent of one pipeline stage: 256 E2M1 nibbles = 128 bytes
+constexpr int kTileKBytes = 128;
+constexpr int kMaxModuli = OZK_MAX_MODULI;
+constexpr int kCrtWords = 6;         // 192-bit integers cover sum r_l w_l for all 27 moduli
+constexpr int kLutStride = 176;      // bytes reserved per modulus in the limb-pair table (m <= 169)
+
+// ---- status word (first bytes of the workspace) -------------------------------------
+struct StatusBlock {
+  int code;          // 0, OZK_ERR_NONFINITE or OZK_ERR_DEVICE_TIMEOUT (first writer wins on severity)
+  int where;         // which wait gave up (role * 256 + barrier id), for diagnostics
+  int pad[62];
+};
+
+// ---- problem geometry ---------------------------------------------------------------
+struct Geometry {
+  int64_t M, N, K;
+  int64_t Mp, Np, Kp;      // padded to 128 / 128 / 256
+  int L;
+  int c_bits;
+  // byte offsets into the workspace
+  size_t off_status, off_lut, off_amax_a, off_amax_b, off_s, off_t, off_planes_a, off_planes_b, off_res;
+  size_t plane_bytes_a, plane_bytes_b;   // one limb plane: rows_p * Kp / 2
+  size_t total;
+};
+
+static inline int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
+
+// ---- per-modulus constants handed to kernels by value --------------------------------
+struct ModulusTable {
+  int L;
+  int m[kMaxModuli];
+  uint32_t recip[kMaxModuli];      // floor(2^32 / m)
+  uint32_t pow18[kMaxModuli];      // 2^18 mod m
+  uint32_t pow36[kMaxModuli];      // 2^36 mod m
+};
+
+struct CrtTable {
+  int L;
+  int words;                               // 32-bit words needed for S = sum r_l w_l
+  int m[kMaxModuli];
+  uint32_t w[kMaxModuli][kCrtWords];       // w_l little endian
+  uint32_t P[kCrtWords];
+  uint32_t halfP[kCrtWords];               // floor(P / 2)
+  double inv_P;                            // 1 / P rounded to double
+};
+
+// host-side constant builders (ozk_tables.cu)
+int host_select_moduli(int count, int* out);
+int host_capacity_bits(int64_t K, int L);
+bool host_build_modulus_table(int L, ModulusTable* t);
+bool host_build_crt_table(int L, CrtTable* t);
+
+// kernels' launchers (each returns cudaError_t of the launch)
+cudaError_t launch_build_lut(const ModulusTable& mt, uint8_t* lut, cudaStream_t st);
+cudaError_t launch_scan_and_shifts(const Geometry& g, const double* A, int64_t lda, const double* B, int64_t ldb,
+                                   uint8_t* ws, cudaStream_t st);
+cudaError_t launch_encode(const Geometry& g, const ModulusTable& mt, const double* A, int64_t lda, const double* B,
+                          int64_t ldb, uint8_t* ws, int64_t* At_out, int64_t* Bt_out, cudaStream_t st);
+cudaError_t launch_decode_plane(const uint8_t* plane, int64_t rows, int64_t K, int64_t Kp, int8_t* out, cudaStream_t st);
+cudaError_t launch_crt(const Geometry& g, const CrtTable& ct, const uint8_t* res, int64_t res_ld, size_t res_stride,
+                       const int32_t* s, const int32_t* t, double* C, int64_t ldc, uint32_t* x_out, cudaStream_t st);
+cudaError_t launch_copy_residues(const Geometry& g, const uint8_t* res, uint8_t* out, cudaStream_t st);
+
+// limb GEMM (ozk_gemm.cu)
+ozk_status gemm_residues(const Geometry& g, const ModulusTable& mt, uint8_t* ws, cudaStream_t st);
+ozk_status gemm_probe(const uint8_t* P, const uint8_t* Q, int64_t K, int scale_byte, float* D, uint8_t* ws, cudaStream_t st);
+
+}  // namespace ozk

@@ -1,0 +1,356 @@
+// Preprocessing kernels (Section 4.2 shared-exponent conversion; Section 5.1 residues and
+// two-limb encoding; Section 6.2 fused decomposition with K-contiguous write-out).
+//
+//   build_lut         per modulus, for every residue one limb pair (c0, c1) as two E2M1 codes
+//   scan_rows/cols    max |.| over the rows of A / the columns of B (exponent scan)
+//   finalize_shifts   s_i = c - 1 - e_i, t_j likewise; flags NaN/Inf
+//   encode_cols       B-side planes: source is already K-contiguous
+//   encode_rows       A-side planes: source is M-contiguous, transposed through shared memory
+//
+// A limb plane is rows_p x Kp nibbles, K-contiguous, two nibbles per byte, the lower-k element
+// in the low nibble.  Plane (l, limb) of an operand starts at (2*l + limb) * plane_bytes.
+#include "ozk_common.cuh"
+
+namespace ozk {
+namespace {
+
+// Doubled E2M1 magnitudes in code order: code & 7 indexes this table, code & 8 is the sign.
+__device__ __constant__ int8_t kDoubledE2M1[8] = {0, 1, 2, 3, 4, 6, 8, 12};
+
+// ------------------------------------------------------------------------------------
+// Limb-pair table: for residue rho of modulus m, one byte (code(c1) << 4) | code(c0) with
+// c0 + 13 c1 = rho (mod m), both limbs in S, chosen to minimise max(|c0|,|c1|) then |c0|+|c1|.
+// ------------------------------------------------------------------------------------
+__global__ void build_lut_kernel(ModulusTable mt, uint8_t* __restrict__ lut) {
+  const int l = blockIdx.x;
+  const int m = mt.m[l];
+  for (int rho = threadIdx.x; rho < kLutStride; rho += blockDim.x) {
+    int best_key = 1 << 30, best_byte = 0;
+    if (rho < m) {
+      for (int i1 = 0; i1 < 16; ++i1) {
+        for (int i0 = 0; i0 < 16; ++i0) {
+          int c0 = kDoubledE2M1[i0 & 7] * ((i0 & 8) ? -1 : 1);
+          int c1 = kDoubledE2M1[i1 & 7] * ((i1 & 8) ? -1 : 1);
+          if ((i0 == 8) || (i1 == 8)) continue;  // skip the negative-zero codes
+          int v = c0 + 13 * c1 - rho;
+          if (v % m != 0) continue;
+          int a0 = abs(c0), a1 = abs(c1);
+          int key = max(a0, a1) * 64 + (a0 + a1);
+          if (key < best_key) {
+            best_key = key;
+            best_byte = (i1 << 4) | i0;
+          }
+        }
+      }
+    }
+    lut[l * kLutStride + rho] = (uint8_t)best_byte;
+  }
+}
+
+// ------------------------------------------------------------------------------------
+// Exponent scan.  |x| compares like its IEEE bit pattern with the sign cleared.
+// ------------------------------------------------------------------------------------
+__device__ __forceinline__ unsigned long long abs_bits(double v) {
+  return (unsigned long long)__double_as_longlong(v) & 0x7FFFFFFFFFFFFFFFull;
+}
+
+// A is M x K column-major: thread = row, loop over a slab of k; loads coalesce along rows.
+__global__ void __launch_bounds__(256) scan_rows_kernel(const double* __restrict__ A, int64_t lda, int64_t M, int64_t K,
+                                                        int kslab, unsigned long long* __restrict__ amax) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t k0 = (int64_t)blockIdx.y * kslab;
+  const int64_t k1 = min(K, k0 + (int64_t)kslab);
+  if (i >= M) return;
+  unsigned long long best = 0;
+  const double* p = A + i + k0 * lda;
+  int64_t k = k0;
+  for (; k + 8 <= k1; k += 8) {
+    unsigned long long b[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) b[u] = abs_bits(__ldg(p + u * lda));
+#pragma unroll
+    for (int u = 0; u < 8; ++u) best = max(best, b[u]);
+    p += 8 * lda;
+  }
+  for (; k < k1; ++k, p += lda) best = max(best, abs_bits(__ldg(p)));
+  if (best) atomicMax(amax + i, best);
+}
+
+// B is K x N column-major: block = (column, k slab); threads stride along k; warp-shuffle max.
+__global__ void __launch_bounds__(256) scan_cols_kernel(const double* __restrict__ B, int64_t ldb, int64_t K, int kslab,
+                                                        unsigned long long* __restrict__ amax) {
+  const int64_t j = blockIdx.x;
+  const int64_t k0 = (int64_t)blockIdx.y * kslab;
+  const int64_t k1 = min(K, k0 + (int64_t)kslab);
+  const double* col = B + j * ldb;
+  unsigned long long best = 0;
+  for (int64_t k = k0 + threadIdx.x; k < k1; k += blockDim.x) best = max(best, abs_bits(__ldg(col + k)));
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) best = max(best, __shfl_xor_sync(0xFFFFFFFFu, best, off));
+  if ((threadIdx.x & 31) == 0 && best) atomicMax(amax + j, best);
+}
+
+// e = floor(log2 |x|) from the bit pattern (subnormals included); shift = c - 1 - e; zero -> 0.
+__global__ void finalize_shifts_kernel(const unsigned long long* __restrict__ amax, int64_t n, int64_t n_pad, int c_bits,
+                                       int32_t* __restrict__ shifts, StatusBlock* __restrict__ status) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n_pad) return;
+  int32_t s = 0;
+  if (i < n) {
+    const unsigned long long b = amax[i];
+    if (b != 0) {
+      const int E = (int)(b >> 52);
+      if (E == 0x7FF) {
+        atomicMin(&status->code, (int)OZK_ERR_NONFINITE);
+      } else {
+        const int e = E ? E - 1023 : (63 - __clzll((long long)b)) - 1074;
+        s = c_bits - 1 - e;
+      }
+    }
+  }
+  shifts[i] = s;
+}
+
+// ------------------------------------------------------------------------------------
+// Integer conversion: round-to-nearest-even of x * 2^s on the significand (exact shift).
+// Returns the magnitude (<= 2^53); *neg receives the sign.
+// ------------------------------------------------------------------------------------
+__device__ __forceinline__ unsigned long long to_integer_magnitude(double x, int s, bool* neg) {
+  const unsigned long long bits = (unsigned long long)__double_as_longlong(x);
+  *neg = (bits >> 63) != 0;
+  const int E = (int)((bits >> 52) & 0x7FF);
+  unsigned long long mant = bits & 0x000FFFFFFFFFFFFFull;
+  if (E) mant |= 1ull << 52;
+  if (mant == 0) return 0;
+  const int sh = (E ? E : 1) - 1075 + s;  // x * 2^s = mant * 2^sh
+  if (sh >= 0) return sh > 52 ? 0 : mant << sh;  // sh > 0 only for subnormal x; |x 2^s| < 2^53 bounds it by 52
+  const int d = -sh;
+  if (d > 54) return 0;
+  const unsigned long long q = mant >> d;
+  const unsigned long long rem = mant & ((1ull << d) - 1);
+  const unsigned long long half = 1ull << (d - 1);
+  return q + ((rem > half) || (rem == half && (q & 1ull)) ? 1ull : 0ull);
+}
+
+// Eight consecutive-k integers of one plane row, split into 18-bit pieces, with sign masks.
+struct Piece8 {
+  uint32_t x0[8], x1[8], x2[8];
+  uint32_t sgn[8];  // 0x88 for negative values: flips the sign bit of both E2M1 codes
+};
+
+__device__ __forceinline__ void split8(const unsigned long long (&mag)[8], const bool (&neg)[8], Piece8& p) {
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    p.x0[e] = (uint32_t)(mag[e] & 0x3FFFFull);
+    p.x1[e] = (uint32_t)((mag[e] >> 18) & 0x3FFFFull);
+    p.x2[e] = (uint32_t)(mag[e] >> 36);
+    p.sgn[e] = neg[e] ? 0x88u : 0u;
+  }
+}
+
+// Residues of the eight values mod m_l and their limb codes packed as 8 nibbles per limb.
+// |a| = x2 2^36 + x1 2^18 + x0  =>  t = x2 (2^36 mod m) + x1 (2^18 mod m) + x0 < 2^27, then one
+// multiply-high reduction; limbs(-rho) = -limbs(rho) because S is symmetric.
+__device__ __forceinline__ void encode8(const Piece8& p, uint32_t m, uint32_t recip, uint32_t pow18, uint32_t pow36,
+                                        const uint8_t* __restrict__ lut_l, uint32_t& w0, uint32_t& w1) {
+  w0 = 0;
+  w1 = 0;
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    const uint32_t t = p.x2[e] * pow36 + p.x1[e] * pow18 + p.x0[e];
+    uint32_t r = t - __umulhi(t, recip) * m;
+    r = min(r, r - m);  // r in [0, 2m): the wrapped difference is larger unless r >= m
+    const uint32_t b = (uint32_t)lut_l[r] ^ p.sgn[e];
+    w0 |= (b & 0xFu) << (4 * e);
+    w1 |= (b >> 4) << (4 * e);
+  }
+}
+
+// ------------------------------------------------------------------------------------
+// B side: plane row = column j of B, source already K-contiguous.
+// Block = 256 threads = 2048 consecutive k of one column; thread = 8 consecutive k.
+// ------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) encode_cols_kernel(const double* __restrict__ B, int64_t ldb, int64_t N, int64_t K,
+                                                          int64_t Kp, ModulusTable mt, const uint8_t* __restrict__ lut,
+                                                          const int32_t* __restrict__ shifts, uint8_t* __restrict__ planes,
+                                                          size_t plane_bytes, int64_t* __restrict__ int_out) {
+  extern __shared__ uint8_t smem[];
+  for (int i = threadIdx.x; i < mt.L * kLutStride; i += blockDim.x) smem[i] = lut[i];
+  __syncthreads();
+  const int64_t j = blockIdx.x;
+  const int64_t k = ((int64_t)blockIdx.y * blockDim.x + threadIdx.x) * 8;
+  if (k >= Kp) return;
+  unsigned long long mag[8];
+  bool neg[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) mag[e] = 0, neg[e] = false;
+  if (j < N && k < K) {
+    const int s = shifts[j];
+    const double* src = B + j * ldb + k;
+    if (k + 8 <= K && ((reinterpret_cast<uintptr_t>(src) & 15) == 0)) {
+      const double2* s2 = reinterpret_cast<const double2*>(src);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const double2 v = __ldg(s2 + e);
+        mag[2 * e] = to_integer_magnitude(v.x, s, &neg[2 * e]);
+        mag[2 * e + 1] = to_integer_magnitude(v.y, s, &neg[2 * e + 1]);
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e)
+        if (k + e < K) mag[e] = to_integer_magnitude(__ldg(src + e), s, &neg[e]);
+    }
+    if (int_out) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e)
+        if (k + e < K) int_out[j * K + k + e] = neg[e] ? -(long long)mag[e] : (long long)mag[e];
+    }
+  }
+  Piece8 p;
+  split8(mag, neg, p);
+  uint8_t* dst = planes + (size_t)j * (size_t)(Kp / 2) + (size_t)(k / 2);
+  for (int l = 0; l < mt.L; ++l) {
+    uint32_t w0, w1;
+    encode8(p, (uint32_t)mt.m[l], mt.recip[l], mt.pow18[l], mt.pow36[l], smem + l * kLutStride, w0, w1);
+    *reinterpret_cast<uint32_t*>(dst + (size_t)(2 * l) * plane_bytes) = w0;
+    *reinterpret_cast<uint32_t*>(dst + (size_t)(2 * l + 1) * plane_bytes) = w1;
+  }
+}
+
+// ------------------------------------------------------------------------------------
+// A side: plane row = row i of A, source is M-contiguous.  Block = tile of 32 rows x 64 k.
+//   load    coalesced along rows into shared memory (k-major)
+//   encode  thread = (row, group of 8 k), warp = 32 rows of one group (conflict-free reads)
+//   store   staged through shared memory so that each plane row receives 32 contiguous bytes
+// ------------------------------------------------------------------------------------
+constexpr int kRowTile = 32;
+constexpr int kRowTileK = 64;
+constexpr int kStageStride = 9;  // words per staged row (8 used): odd stride avoids bank conflicts
+
+__global__ void __launch_bounds__(256) encode_rows_kernel(const double* __restrict__ A, int64_t lda, int64_t M, int64_t K,
+                                                          int64_t Kp, ModulusTable mt, const uint8_t* __restrict__ lut,
+                                                          const int32_t* __restrict__ shifts, uint8_t* __restrict__ planes,
+                                                          size_t plane_bytes, int64_t* __restrict__ int_out) {
+  extern __shared__ __align__(16) uint8_t smem[];
+  uint8_t* lut_s = smem;                                                        // L * kLutStride bytes
+  const int lut_bytes = (mt.L * kLutStride + 15) & ~15;
+  double* in_s = reinterpret_cast<double*>(smem + lut_bytes);                    // [64][32] doubles
+  uint32_t* out_s = reinterpret_cast<uint32_t*>(smem + lut_bytes);               // [2L][32][9] words, reuses in_s
+  const int t = threadIdx.x;
+  const int64_t i0 = (int64_t)blockIdx.x * kRowTile;
+  const int64_t k0 = (int64_t)blockIdx.y * kRowTileK;
+  for (int i = t; i < mt.L * kLutStride; i += blockDim.x) lut_s[i] = lut[i];
+  {
+    const int ti = t & 31, tk = t >> 5;
+    const int64_t i = i0 + ti;
+#pragma unroll
+    for (int n = 0; n < 8; ++n) {
+      const int64_t k = k0 + tk + 8 * n;
+      in_s[(tk + 8 * n) * kRowTile + ti] = (i < M && k < K) ? __ldg(A + i + k * lda) : 0.0;
+    }
+  }
+  __syncthreads();
+  const int r = t & 31, g = t >> 5;
+  unsigned long long mag[8];
+  bool neg[8];
+  {
+    const int64_t i = i0 + r;
+    const int s = shifts[i];  // shifts has Mp entries; padded rows hold 0
+#pragma unroll
+    for (int e = 0; e < 8; ++e) mag[e] = to_integer_magnitude(in_s[(8 * g + e) * kRowTile + r], s, &neg[e]);
+    if (int_out && i < M) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const int64_t k = k0 + 8 * g + e;
+        if (k < K) int_out[i + k * M] = neg[e] ? -(long long)mag[e] : (long long)mag[e];
+      }
+    }
+  }
+  __syncthreads();  // in_s is dead from here on; out_s takes its place
+  Piece8 p;
+  split8(mag, neg, p);
+  for (int l = 0; l < mt.L; ++l) {
+    uint32_t w0, w1;
+    encode8(p, (uint32_t)mt.m[l], mt.recip[l], mt.pow18[l], mt.pow36[l], lut_s + l * kLutStride, w0, w1);
+    out_s[((2 * l) * kRowTile + r) * kStageStride + g] = w0;
+    out_s[((2 * l + 1) * kRowTile + r) * kStageStride + g] = w1;
+  }
+  __syncthreads();
+  const int row = t >> 3, word = t & 7;
+  uint8_t* dst = planes + (size_t)(i0 + row) * (size_t)(Kp / 2) + (size_t)(k0 / 2) + 4 * word;
+  for (int pl = 0; pl < 2 * mt.L; ++pl)
+    *reinterpret_cast<uint32_t*>(dst + (size_t)pl * plane_bytes) = out_s[(pl * kRowTile + row) * kStageStride + word];
+}
+
+// Decodes one limb plane into doubled-E2M1 integers, out[r + k*rows] (test support).
+__global__ void decode_plane_kernel(const uint8_t* __restrict__ plane, int64_t rows, int64_t K, int64_t Kp,
+                                    int8_t* __restrict__ out) {
+  const int64_t r = (int64_t)blockIdx.y * blockDim.x + threadIdx.x;
+  const int64_t k = blockIdx.x;
+  if (r >= rows || k >= K) return;
+  const uint8_t byte = plane[(size_t)r * (size_t)(Kp / 2) + (size_t)(k / 2)];
+  const int code = (k & 1) ? (byte >> 4) : (byte & 0xF);
+  const int v = kDoubledE2M1[code & 7];
+  out[r + k * rows] = (int8_t)((code & 8) ? -v : v);
+}
+
+}  // namespace
+
+cudaError_t launch_build_lut(const ModulusTable& mt, uint8_t* lut, cudaStream_t st) {
+  build_lut_kernel<<<mt.L, 192, 0, st>>>(mt, lut);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_scan_and_shifts(const Geometry& g, const double* A, int64_t lda, const double* B, int64_t ldb,
+                                   uint8_t* ws, cudaStream_t st) {
+  auto* amax_a = reinterpret_cast<unsigned long long*>(ws + g.off_amax_a);
+  auto* amax_b = reinterpret_cast<unsigned long long*>(ws + g.off_amax_b);
+  auto* status = reinterpret_cast<StatusBlock*>(ws + g.off_status);
+  cudaError_t e = cudaMemsetAsync(amax_a, 0, (size_t)(g.Mp + g.Np) * sizeof(unsigned long long), st);
+  if (e != cudaSuccess) return e;
+  if (g.K > 0) {
+    const int kslab_a = 64;
+    dim3 ga((unsigned)((g.M + 255) / 256), (unsigned)((g.K + kslab_a - 1) / kslab_a));
+    scan_rows_kernel<<<ga, 256, 0, st>>>(A, lda, g.M, g.K, kslab_a, amax_a);
+    const int kslab_b = 2048;
+    dim3 gb((unsigned)g.N, (unsigned)((g.K + kslab_b - 1) / kslab_b));
+    scan_cols_kernel<<<gb, 256, 0, st>>>(B, ldb, g.K, kslab_b, amax_b);
+  }
+  finalize_shifts_kernel<<<(unsigned)((g.Mp + 255) / 256), 256, 0, st>>>(amax_a, g.M, g.Mp, g.c_bits,
+                                                                        reinterpret_cast<int32_t*>(ws + g.off_s), status);
+  finalize_shifts_kernel<<<(unsigned)((g.Np + 255) / 256), 256, 0, st>>>(amax_b, g.N, g.Np, g.c_bits,
+                                                                        reinterpret_cast<int32_t*>(ws + g.off_t), status);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_encode(const Geometry& g, const ModulusTable& mt, const double* A, int64_t lda, const double* B,
+                          int64_t ldb, uint8_t* ws, int64_t* At_out, int64_t* Bt_out, cudaStream_t st) {
+  const uint8_t* lut = ws + g.off_lut;
+  const int lut_bytes = (mt.L * kLutStride + 15) & ~15;
+  {
+    const size_t stage = (size_t)2 * mt.L * kRowTile * kStageStride * sizeof(uint32_t);
+    const size_t in_bytes = (size_t)kRowTileK * kRowTile * sizeof(double);
+    const size_t smem = lut_bytes + (stage > in_bytes ? stage : in_bytes);
+    cudaError_t e = cudaFuncSetAttribute(encode_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    dim3 grid((unsigned)(g.Mp / kRowTile), (unsigned)(g.Kp / kRowTileK));
+    encode_rows_kernel<<<grid, 256, smem, st>>>(A, lda, g.M, g.K, g.Kp, mt, lut, reinterpret_cast<const int32_t*>(ws + g.off_s),
+                                                ws + g.off_planes_a, g.plane_bytes_a, At_out);
+  }
+  {
+    dim3 grid((unsigned)g.Np, (unsigned)((g.Kp + 2047) / 2048));
+    encode_cols_kernel<<<grid, 256, lut_bytes, st>>>(B, ldb, g.N, g.K, g.Kp, mt, lut,
+                                                    reinterpret_cast<const int32_t*>(ws + g.off_t), ws + g.off_planes_b,
+                                                    g.plane_bytes_b, Bt_out);
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_decode_plane(const uint8_t* plane, int64_t rows, int64_t K, int64_t Kp, int8_t* out, cudaStream_t st) {
+  if (rows == 0 || K == 0) return cudaSuccess;
+  dim3 grid((unsigned)K, (unsigned)((rows + 127) / 128));
+  decode_plane_kernel<<<grid, 128, 0, st>>>(plane, rows, K, Kp, out);
+  return cudaGetLastError();
+}
+
+}  // namespace ozk

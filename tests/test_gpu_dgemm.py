@@ -1,0 +1,79 @@
+"""End-to-end parity of ozk_dgemm with the CPU oracle (bit for bit) and accuracy against fl(AB)."""
+import numpy as np
+import pytest
+
+from oracle import exact, ozaki2
+from paper_2608_06812_b200 import binding as ozk
+from paper_2608_06812_b200 import inputs
+from tests import gpu_util as gu
+
+pytestmark = pytest.mark.gpu
+
+
+def test_config1_256_cubed_L14_bit_exact_and_error_levels():
+    """M=N=K=256, phi=0.5, seeds 0/1: bit-exact against the oracle at 14 moduli; against the exact
+    fl(AB) the bound 1e-15 holds from 17 moduli on (14 moduli keep only 42 bits, Eq. 3)."""
+    A = inputs.lognormal_matrix(256, 256, 0.5, seed=0)
+    B = inputs.lognormal_matrix(256, 256, 0.5, seed=1)
+    F = exact.fl_matmul(A[:64], B[:, :64])
+    for L in (14, 17, 19):
+        C = gu.dgemm(A, B, L)
+        ref = ozaki2.dgemm(A, B, L)
+        assert gu.bits_equal(C, ref.C), f"L={L}"
+        err = exact.normwise_error(C[:64, :64], A[:64], B[:, :64], against_rounded=True)
+        if L >= 17:
+            assert err <= 1e-15
+    assert np.mean(gu.dgemm(A, B, 19)[:64, :64] == F) > 0.05   # many elements are the correctly rounded value itself
+
+
+@pytest.mark.parametrize("shape", [(1, 1, 1), (2, 3, 0), (130, 70, 300), (257, 129, 255), (128, 384, 1025), (640, 512, 768)])
+@pytest.mark.parametrize("L", [12, 19, 20])
+def test_ragged_shapes_bit_exact(shape, L):
+    M, N, K = shape
+    A = inputs.lognormal_matrix(M, K, 1.0, seed=10)
+    B = inputs.lognormal_matrix(K, N, 1.0, seed=11)
+    C = gu.dgemm(A, B, L, lda=M + 1, ldb=K + 7, ldc=M + 5)
+    assert gu.bits_equal(C, ozaki2.dgemm(A, B, L).C)
+
+
+@pytest.mark.parametrize("L", [2, 13, 15, 16, 18, 24, 27])
+def test_every_modulus_count_bit_exact(L):
+    A = inputs.lognormal_matrix(96, 200, 0.5, seed=0)
+    B = inputs.lognormal_matrix(200, 40, 0.5, seed=1)
+    assert gu.bits_equal(gu.dgemm(A, B, L), ozaki2.dgemm(A, B, L).C)
+
+
+def test_small_integers_give_the_exact_integer_product():
+    A = inputs.small_integer_matrix(200, 333, 1000, seed=1)
+    B = inputs.small_integer_matrix(333, 150, 1000, seed=2)
+    A[7, :] = 0.0
+    C = gu.dgemm(A, B, 19)
+    ref = (A.astype(np.int64) @ B.astype(np.int64)).astype(np.float64)
+    assert gu.bits_equal(C, ref)
+
+
+def test_paper_law_phi0_equals_fl_of_exact_product():
+    """Section 7.1: with one exponent per row/column the conversion is exact, so the output is
+    the exact product rounded once."""
+    A = inputs.exponent_spread_matrix(64, 2048, 0, seed=0)
+    B = inputs.exponent_spread_matrix(2048, 48, 0, seed=1)
+    assert gu.bits_equal(gu.dgemm(A, B, 19), exact.fl_matmul(A, B))
+
+
+def test_wide_exponent_range_and_extremes_bit_exact():
+    A = inputs.lognormal_matrix(64, 128, 4.0, seed=0)
+    B = inputs.lognormal_matrix(128, 64, 4.0, seed=1)
+    A[0, :] *= 2.0 ** 500
+    A[1, :] *= 2.0 ** -500
+    B[:, 0] *= 2.0 ** 400
+    B[:, 1] *= 2.0 ** -520                       # products reach the subnormal range
+    A[2, :] = 0.0
+    C = gu.dgemm(A, B, 19)
+    assert gu.bits_equal(C, ozaki2.dgemm(A, B, 19).C)
+
+
+def test_invalid_arguments():
+    gu.ensure_workspace(1 << 20)
+    assert ozk.ozk_dgemm(8, 8, 8, None, 8, None, 8, None, 8, 19, 0) == ozk.OZK_ERR_INVALID_ARG      # null pointers
+    assert ozk.ozk_dgemm(4096, 4096, 4096, 1024, 4096, 1024, 4096, 1024, 4096, 19, 0) == ozk.OZK_ERR_WORKSPACE
+    assert ozk.ozk_dgemm(0, 8, 8, None, 1, None, 8, None, 1, 19, 0) == ozk.OZK_OK                   # empty result
