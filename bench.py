@@ -1,0 +1,334 @@
+#!/usr/bin/env python
+"""Benchmark of the emulated DGEMM hot path (Ozaki scheme II on FP4 tensor cores).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--size 16384] [--moduli 19]
+    python bench.py --impl reference ...     # times the CPU oracle on a bounded sample
+
+One step = one ozk_dgemm (exponent scan, limb encoding, limb GEMM, CRT) over one pair of
+seeded synthetic FP64 matrices.  `value` is the whole-job effective FP64 rate 2MNK/t with the
+inputs resident in HBM; `e2e` is the same metric through the C ABI with host buffers, the
+host-to-device copies of A and B and the device-to-host copy of C inside the timed region.
+With N > 1 every rank runs an independent replica of the same problem (the path has no
+exchange step); the time is the maximum over ranks and the value the sum of the work.
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "effective FP64 TFLOPS (2MNK/t), Ozaki scheme II on FP4, end to end incl. preprocessing"
+UNIT = "TFLOP/s"
+PAPER_TOTAL_TFLOPS = {4096: 10.81, 8192: 13.52, 16384: 15.26}   # the paper's end-to-end numbers, L = 19, other GPU
+FP4_PER_BF16 = 4.0                                               # nominal dense FP4 : BF16 ratio on B200
+KERNELS_PER_STEP = 9   # lut, scan_rows, scan_cols, 2 x finalize, encode_rows, encode_cols, limb GEMM, CRT
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--size", type=int, default=16384, help="M = N = K")
+    ap.add_argument("--moduli", type=int, default=19)
+    ap.add_argument("--phi", type=float, default=1.0)
+    ap.add_argument("--impl", default="ozk", choices=["ozk", "reference"])
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-fp64-context", action="store_true")
+    return ap.parse_args()
+
+
+def workload_name(n: int, L: int, phi: float) -> str:
+    return f"M=N=K={n} FP64 square, (U-0.5)*exp({phi:g}*N(0,1)), seeds 0/1, Ozaki-II {L} moduli"
+
+
+# ---------------------------------------------------------------------------------------------
+# measured peaks, clocks
+# ---------------------------------------------------------------------------------------------
+def measured_peaks() -> dict:
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return {"source": "measured", "hbm_gbs": d["hbm_gbs"], "bf16_burst": d["bf16_tflops"],
+                "bf16_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"])}
+    return {"source": "fallback", "hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0}
+
+
+class ClockSampler:
+    """nvidia-smi clock and throttle-reason samples while the timed region runs."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.file = None
+
+    def start(self):
+        try:
+            self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.gpu_index)], stdout=self.file, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.file.flush()
+        rows = [r.split(", ") for r in open(self.file.name).read().strip().splitlines() if r.strip()]
+        os.unlink(self.file.name)
+        sm, smax, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            if len(r) < 9:
+                continue
+            try:
+                sm.append(float(r[1])); smax.append(float(r[2])); power.append(float(r[3]))
+            except ValueError:
+                continue
+            for name, flag in zip(names, r[5:9]):
+                if flag.strip().lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(smax), "power_w_max": max(power),
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ---------------------------------------------------------------------------------------------
+# CPU oracle legs
+# ---------------------------------------------------------------------------------------------
+def oracle_sample_tflops(A: np.ndarray, B: np.ndarray, L: int, block: int, repeats: int = 1) -> tuple[float, float, str, int]:
+    """Times the CPU oracle, as it stands, on a block x block corner of the output (full K).
+    Returns (TFLOP/s, seconds per run, description of the sample, threads used)."""
+    from oracle import ozaki2
+    M, K = A.shape
+    b = min(block, M, B.shape[1])
+    As, Bs = np.ascontiguousarray(A[:b]), np.ascontiguousarray(B[:, :b])
+    best = float("inf")
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        ozaki2.dgemm(As, Bs, L)
+        best = min(best, time.perf_counter() - t0)
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    sample = f"oracle.ozaki2.dgemm on the {b}x{b} leading output block, full K={K} ({2.0 * b * b * K:.3g} flop-equivalents)"
+    return 2.0 * b * b * K / best / 1e12, best, sample, threads
+
+
+def run_reference(args, rank: int, world: int) -> None:
+    """--impl reference: the CPU oracle on this arm's workload, rank 0 only."""
+    if rank != 0:
+        return
+    from paper_2608_06812_b200 import inputs
+    n, L = args.size, args.moduli
+    block = 128
+    A = inputs.lognormal_matrix(block, n, args.phi, seed=0)          # 128 rows / columns of the workload's law and seeds
+    B = inputs.lognormal_matrix(n, block, args.phi, seed=1)
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample_tflops(A, B, L, block)
+    secs = []
+    for _ in range(args.steps):
+        tf, s, sample, threads = oracle_sample_tflops(A, B, L, block)
+        secs.append(s)
+    t = statistics.mean(secs)
+    value = 2.0 * block * block * n / t / 1e12
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * t, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "int64/f64 (CPU oracle)", "data": "synthetic",
+            "config": {"workload": workload_name(n, L, args.phi), "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------------
+# multi-rank reduction (replicas): max of the times, sum of the work
+# ---------------------------------------------------------------------------------------------
+def reduce_over_ranks(ms_per_step: float, flops_per_step: float, dist=None, device=None) -> tuple[float, float]:
+    """Returns (max over ranks of ms_per_step, sum over ranks of flops_per_step)."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return ms_per_step, flops_per_step
+    import torch
+    t = torch.tensor([ms_per_step], dtype=torch.float64, device=device)
+    f = torch.tensor([flops_per_step], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(f, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(f.item())
+
+
+# ---------------------------------------------------------------------------------------------
+# the GPU arm
+# ---------------------------------------------------------------------------------------------
+def run_ozk(args, rank: int, local_rank: int, world: int) -> None:
+    import torch
+    import torch.distributed as dist
+    from paper_2608_06812_b200 import binding as ozk
+    from paper_2608_06812_b200 import inputs
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the product path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1 and not dist.is_initialized():
+        dist.init_process_group("nccl", device_id=dev)
+
+    n, L = args.size, args.moduli
+    M = N = K = n
+    stream = torch.cuda.current_stream().cuda_stream
+    A = inputs.lognormal_matrix(M, K, args.phi, seed=0)
+    B = inputs.lognormal_matrix(K, N, args.phi, seed=1)
+    # column-major storage = the transpose in C order
+    hA = torch.from_numpy(np.ascontiguousarray(A.T)).pin_memory()
+    hB = torch.from_numpy(np.ascontiguousarray(B.T)).pin_memory()
+    hC = torch.empty((N, M), dtype=torch.float64).pin_memory()
+    dA, dB = hA.to(dev), hB.to(dev)
+    dC = torch.empty((N, M), dtype=torch.float64, device=dev)
+    ws_bytes = ozk.ozk_dgemm_workspace_bytes(M, N, K, L)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    ozk.check(ozk.ozk_set_workspace(ws.data_ptr(), ws.numel()), "ozk_set_workspace")
+    ozk.check(ozk.ozk_stage_timing_enable(True), "ozk_stage_timing_enable")
+
+    def step():
+        ozk.check(ozk.ozk_dgemm(M, N, K, dA.data_ptr(), M, dB.data_ptr(), K, dC.data_ptr(), M, L, stream), "ozk_dgemm")
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    ozk.check(ozk.ozk_get_async_status(stream), "ozk_get_async_status")
+
+    # ---- device-resident timing: exactly `steps` steps between two barriers -----------------
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    stage_acc = np.zeros(3)
+    barrier()
+    ev[0].record()
+    for i in range(args.steps):
+        step()
+        ev[i + 1].record()
+        # per-stage CUDA events recorded by the library on this stream, read live inside the timed
+        # region (the read waits for this step's last event; a step is >100 ms, the wait adds microseconds)
+        stage_acc += np.array(ozk.ozk_stage_timing_read())
+    barrier()
+    total_ms = ev[0].elapsed_time(ev[args.steps])
+    clocks = sampler.stop() if rank == 0 else None
+    ozk.check(ozk.ozk_get_async_status(stream), "ozk_get_async_status")
+    per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
+    stage_acc /= args.steps
+    ms_per_step = total_ms / args.steps
+    flops = 2.0 * M * N * K
+
+    # ---- end to end with host buffers -----------------------------------------------------
+    e2e = None
+    if not args.no_e2e:
+        def e2e_step():
+            dA.copy_(hA, non_blocking=True)
+            dB.copy_(hB, non_blocking=True)
+            step()
+            hC.copy_(dC, non_blocking=True)
+        e2e_step()
+        barrier()
+        t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+        t0.record()
+        for _ in range(args.steps):
+            e2e_step()
+        t1.record()
+        barrier()
+        e2e_ms = t0.elapsed_time(t1) / args.steps
+        e2e_ms, e2e_flops = reduce_over_ranks(e2e_ms, flops, dist if world > 1 else None, dev)
+        e2e = {"value": e2e_flops / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
+               "h2d_bytes_per_step": int(hA.numel() * 8 + hB.numel() * 8), "d2h_bytes_per_step": int(hC.numel() * 8)}
+
+    ms_max, flops_all = reduce_over_ranks(ms_per_step, flops, dist if world > 1 else None, dev)
+    value = flops_all / (ms_max * 1e-3) / 1e12
+
+    if rank != 0:
+        return
+    peaks = measured_peaks()
+    gemm_ms = float(stage_acc[1])
+    fp4_flops_exec = 2.0 * 4 * L * M * N * K             # 4 limb products per modulus are executed
+    fp4_flops_req = 2.0 * (4 * L - 1) * M * N * K        # the 13^2 term of modulus 169 is not required
+    achieved = fp4_flops_exec / (gemm_ms * 1e-3) / 1e12
+    peak = peaks["bf16_sustained"] * FP4_PER_BF16
+    roofline = {"bound": "tensor", "kernel": "residue_gemm_kernel", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                "frac": achieved / peak, "traffic": None,
+                "peak_source": f"{peaks['source']} bf16 sustained {peaks['bf16_sustained']:.1f} TFLOP/s x {FP4_PER_BF16:g} (nominal FP4:BF16)",
+                "achieved_required_count": fp4_flops_req / (gemm_ms * 1e-3) / 1e12,
+                "frac_of_burst_peak": achieved / (peaks["bf16_burst"] * FP4_PER_BF16),
+                "frac_of_nominal_9000": achieved / 9000.0, "ms_per_launch": gemm_ms}
+    pre_bytes = (16 + L) * (M * K + K * N)               # scan read + convert read + one byte (two nibbles) per modulus
+    crt_bytes = (L + 8) * M * N
+    stages = {"preprocess_ms": float(stage_acc[0]), "limb_gemm_ms": gemm_ms, "crt_ms": float(stage_acc[2]),
+              "preprocess_gbs": pre_bytes / (stage_acc[0] * 1e-3) / 1e9, "crt_gbs": crt_bytes / (stage_acc[2] * 1e-3) / 1e9,
+              "hbm_peak_gbs": peaks["hbm_gbs"], "per_step_ms": per_step}
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": ms_max, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": (value / world / PAPER_TOTAL_TFLOPS[n]) if (n in PAPER_TOTAL_TFLOPS and L == 19) else None,
+            "dtype": "fp4_e2m1 (fp32 accumulate, integer CRT)", "data": "synthetic",
+            "config": {"workload": workload_name(n, L, args.phi), "l2": "inputs (2 x %.2f GiB) larger than L2" % (M * K * 8 / 2 ** 30),
+                       "parallelism": "replicas" if world > 1 else "single GPU", "moduli": L},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": KERNELS_PER_STEP * args.steps, "roofline": roofline, "stages": stages}
+
+    if not args.no_fp64_context:
+        try:
+            x = torch.matmul(dA, dB)                      # native FP64 GEMM on the same GPU: context only
+            torch.cuda.synchronize()
+            t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+            t0.record(); x = torch.matmul(dA, dB); t1.record(); torch.cuda.synchronize()
+            line["native_fp64_tflops_context"] = flops / (t0.elapsed_time(t1) * 1e-3) / 1e12
+            del x
+        except Exception as exc:                          # out of memory on small boxes: context is optional
+            line["native_fp64_tflops_context"] = f"unavailable: {type(exc).__name__}"
+    if not args.no_cpu_baseline:
+        tf, secs, sample, threads = oracle_sample_tflops(A, B, L, 256)
+        line["cpu_baseline"] = {"value": tf, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample, "seconds": secs}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    args = parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+    run_ozk(args, rank, local_rank, world)
+    if world > 1:
+        import torch.distributed as dist
+        if dist.is_initialized():
+            dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -153,6 +153,14 @@ ozk_status ozk_stage_crt(int64_t M, int64_t N, int64_t K, int num_moduli,
                          const uint8_t* residues_in, const int32_t* s_in, const int32_t* t_in,
                          double* C, int64_t ldc, uint32_t* x_out, void* stream);
 
+/* Measurement aid (the paper times its stages with CUDA events, Section 6.1): when enabled,
+ * ozk_dgemm records four CUDA events on its stream, before stage 1 and after each of the three
+ * stages.  Enabling creates the events (a host-side allocation; do it outside timed regions).
+ * ozk_stage_timing_read() synchronises on the last event and writes the milliseconds of
+ * preprocessing, limb GEMM and reconstruction of the most recent ozk_dgemm to ms3[0..2] (host). */
+ozk_status ozk_stage_timing_enable(int enable);
+ozk_status ozk_stage_timing_read(float* ms3);
+
 /* One tcgen05.mma.kind::mxf4.block_scale instruction sequence on caller-supplied packed
  * E2M1 operands, used to pin the hardware byte formats (nibble order, E2M1 codes, UE8M0
  * scale byte, FP32 accumulator exactness): D[128 x 128] (FP32, row-major, device) =

@@ -43,6 +43,8 @@ SIGNATURES = {
     "ozk_stage_residue_gemm": (c_int, [c_int64, c_int64, c_int64, c_int, c_void_p, c_void_p]),
     "ozk_stage_crt": (c_int, [c_int64, c_int64, c_int64, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_int64,
                               c_void_p, c_void_p]),
+    "ozk_stage_timing_enable": (c_int, [c_int]),
+    "ozk_stage_timing_read": (c_int, [c_void_p]),
     "ozk_stage_mma_probe": (c_int, [c_void_p, c_void_p, c_int64, c_int, c_void_p, c_void_p]),
 }
 
@@ -145,3 +147,13 @@ def ozk_stage_crt(M, N, K, num_moduli, residues_in, s_in, t_in, C, ldc, x_out=No
 
 def ozk_stage_mma_probe(P, Q, K, scale_byte, D, stream=0) -> int:
     return lib().ozk_stage_mma_probe(P, Q, K, scale_byte, D, stream)
+
+
+def ozk_stage_timing_enable(enable: bool) -> int:
+    return lib().ozk_stage_timing_enable(1 if enable else 0)
+
+
+def ozk_stage_timing_read() -> tuple[float, float, float]:
+    ms = (ctypes.c_float * 3)()
+    check(lib().ozk_stage_timing_read(ms), "ozk_stage_timing_read")
+    return float(ms[0]), float(ms[1]), float(ms[2])

@@ -15,6 +15,17 @@ Workspace g_ws;
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+struct StageTiming {
+  bool enabled = false;
+  bool recorded = false;
+  cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
+};
+StageTiming g_timing;
+
+void mark(int i, cudaStream_t st) {
+  if (g_timing.enabled) cudaEventRecord(g_timing.ev[i], st);
+}
+
 // Workspace layout for an (M, N, K, L) problem.  Returns false on invalid sizes.
 bool make_geometry(int64_t M, int64_t N, int64_t K, int L, Geometry* g) {
   if (M < 0 || N < 0 || K < 0 || L < OZK_MIN_MODULI || L > OZK_MAX_MODULI) return false;
@@ -233,14 +244,38 @@ ozk_status ozk_dgemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t l
   CrtTable ct;
   if (!host_build_modulus_table(num_moduli, &mt) || !host_build_crt_table(num_moduli, &ct)) return OZK_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  mark(0, st);
   rc = run_preprocess(g, mt, A, lda, B, ldb, nullptr, nullptr, st);
   if (rc != OZK_OK) return rc;
+  mark(1, st);
   rc = gemm_residues(g, mt, g_ws.ptr, st);
   if (rc != OZK_OK) return rc;
+  mark(2, st);
   if (launch_crt(g, ct, g_ws.ptr + g.off_res, g.Mp, (size_t)g.Mp * (size_t)g.Np,
                  reinterpret_cast<const int32_t*>(g_ws.ptr + g.off_s), reinterpret_cast<const int32_t*>(g_ws.ptr + g.off_t), C, ldc,
                  nullptr, st) != cudaSuccess)
     return OZK_ERR_CUDA;
+  mark(3, st);
+  g_timing.recorded = g_timing.enabled;
+  return OZK_OK;
+}
+
+ozk_status ozk_stage_timing_enable(int enable) {
+  if (enable && !g_timing.ev[0]) {
+    for (int i = 0; i < 4; ++i)
+      if (cudaEventCreate(&g_timing.ev[i]) != cudaSuccess) return OZK_ERR_CUDA;
+  }
+  g_timing.enabled = enable != 0;
+  g_timing.recorded = false;
+  return OZK_OK;
+}
+
+ozk_status ozk_stage_timing_read(float* ms3) {
+  if (!ms3) return OZK_ERR_INVALID_ARG;
+  if (!g_timing.recorded) return OZK_ERR_INVALID_ARG;
+  if (cudaEventSynchronize(g_timing.ev[3]) != cudaSuccess) return OZK_ERR_CUDA;
+  for (int i = 0; i < 3; ++i)
+    if (cudaEventElapsedTime(&ms3[i], g_timing.ev[i], g_timing.ev[i + 1]) != cudaSuccess) return OZK_ERR_CUDA;
   return OZK_OK;
 }
 
