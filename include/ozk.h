@@ -153,6 +153,26 @@ ozk_status ozk_stage_crt(int64_t M, int64_t N, int64_t K, int num_moduli,
                          const uint8_t* residues_in, const int32_t* s_in, const int32_t* t_in,
                          double* C, int64_t ldc, uint32_t* x_out, void* stream);
 
+/* The paper has no counterpart to this entry point.  It is for callers that cannot allocate
+ * device memory and so cannot provide the workspace the calls above need: code running under a
+ * framework whose allocator owns all device memory and forbids raw cudaMalloc (which synchronises
+ * the device), plug-ins inside latency-critical loops, processes that have no free memory left.
+ * It computes what stage 1 computes first, the row shifts s_i = c - 1 - e_i of A
+ * (c = ozk_capacity_bits(K, num_moduli), Section 4.2), and keeps its only scratch, one 64-bit
+ * maximum per row, in a fixed array inside the library image: OZK_NOALLOC_MAX_ROWS rows,
+ * 512 KiB, resident on every GPU that loads the library until the process exits.  Neither this
+ * call nor anything it calls allocates or frees memory.
+ *   A: M x K column-major FP64 (device), lda >= M.  s_out: M int32 (device).  An all-zero row
+ *   gets 0; a row containing NaN or Inf gets INT32_MIN (there is no status word to report it).
+ *   M > OZK_NOALLOC_MAX_ROWS, or K beyond the limits of ozk_dgemm -> OZK_ERR_UNSUPPORTED.
+ * The first call on each device looks up the device address of the array (with that device
+ * current); make that first call before starting any stream capture.  Every call uses the same
+ * array and finds the previous call's contents in it: the rows it needs are cleared on `stream`
+ * first, and two calls whose work overlaps on the GPU (different streams, no ordering) race. */
+enum { OZK_NOALLOC_MAX_ROWS = 65536 };
+ozk_status ozk_row_shifts_noalloc(int64_t M, int64_t K, const double* A, int64_t lda, int num_moduli,
+                                  int32_t* s_out, void* stream);
+
 /* Measurement aid (the paper times its stages with CUDA events, Section 6.1): when enabled,
  * ozk_dgemm records four CUDA events on its stream, before stage 1 and after each of the three
  * stages.  Enabling creates the events (a host-side allocation; do it outside timed regions).
