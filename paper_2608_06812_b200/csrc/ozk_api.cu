@@ -94,6 +94,10 @@ ozk_status run_preprocess(const Geometry& g, const ModulusTable& mt, const doubl
 }
 
 }  // namespace
+
+uint8_t* workspace_ptr() { return g_ws.ptr; }
+size_t workspace_bytes() { return g_ws.bytes; }
+
 }  // namespace ozk
 
 using namespace ozk;
@@ -287,5 +291,4 @@ ozk_status ozk_stage_mma_probe(const uint8_t* P, const uint8_t* Q, int64_t K, in
   return gemm_probe(P, Q, K, scale_byte, D, g_ws.ptr, static_cast<cudaStream_t>(stream));
 }
 
-// INT8 path: see ozk_igemm.cu
 }  // extern "C"

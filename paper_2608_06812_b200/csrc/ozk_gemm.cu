@@ -1,19 +1,23 @@
-// Limb GEMM with residue composition in the epilogue (Section 5.1: ab = a0 b0 + 13 (a0 b1 + a1 b0)
-// + 13^2 a1 b1 (mod m); Section 6.4: all moduli in one launch, three accumulators per modulus,
-// nothing but the residues written to memory; Lemma 3: every FP32 partial sum is an exact integer).
+// Limb GEMM on the FP4 tensor cores (tcgen05.mma kind::mxf4, block-scaled E2M1, FP32 accumulators
+// in tensor memory), with the recombination of the limb products in the epilogue.
 //
-// One persistent CTA per SM walks a static list of work items (modulus l, tile of 128 columns
-// of C, tile of 128 rows of C).  The tensor-core "row" side (TMEM lanes) holds the B-matrix
-// limbs p0, p1 (plane rows = columns j of C) and the "column" side the A-matrix limbs q0, q1
-// (plane rows = rows i of C), so a thread of the epilogue owns one j and consecutive i, which is
-// the column-major order of the residue matrices and of C.
+//   DGEMM path   Section 5.1: ab = a0 b0 + 13 (a0 b1 + a1 b0) + 13^2 a1 b1 (mod m); Section 6.4: all
+//                moduli in one launch, three accumulators per modulus, only residues reach memory;
+//                Lemma 3: every FP32 partial sum is an exact integer.
+//   INT8 path    Section 3 / Eq. 1 with p = q = 3: nine limb products in five groups i + j = g,
+//                C = sum_g 13^g G_g as int32.
 //
-// Per 64-nibble K step two N = 256 instructions do the four limb products:
-//     D[  0..255] += p0 * [q0 ; q1]    -> columns   0..127: p0 q0,  128..255: p0 q1
-//     D[128..383] += p1 * [q0 ; q1]    -> columns 128..255: p1 q0,  256..383: p1 q1
-// so columns 128..255 accumulate the two cross terms of weight 13 in one accumulator.
+// One persistent CTA per SM walks a static list of work items (plane group l, tile of 128 columns
+// of C, tile of W rows of C).  The tensor-core row side (TMEM lanes) holds the B-matrix limbs p_i
+// (plane rows = columns j of C) and the column side the A-matrix limbs q_j (plane rows = rows i of
+// C), so an epilogue thread owns one j and consecutive i: the column-major order of C.
 //
-// Warp roles: 0 = TMA producer, 1 = MMA issuer (owns the TMEM allocation), 2..5 = epilogue.
+// The limb tiles q_0 .. q_{NQ-1} of a stage are adjacent in shared memory, so ONE instruction per
+// row-side limb does all its products:  D[W*i .. W*i + NQ*W) += p_i * [q_0 ; ... ; q_{NQ-1}].
+// Group g = i + j therefore accumulates in TMEM columns [W*g, W*g + W): the cross terms that share
+// a power of 13 land in the same accumulator (NP + NQ - 1 accumulators for NP * NQ products).
+//
+// Warp roles: 0 = TMA producer, 1 = MMA issuer (owns the TMEM allocation), 2.. = epilogue.
 // Every wait is bounded; on expiry the CTA records OZK_ERR_DEVICE_TIMEOUT, drains and returns.
 #include "ozk_common.cuh"
 #include "ozk_ptx.cuh"
@@ -23,33 +27,26 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kStages = 3;
-constexpr int kOperandTileBytes = kTileRows * kTileKBytes;  // 16 KiB: 128 rows x 128 bytes
-constexpr int kStageBytes = 4 * kOperandTileBytes;          // p0, p1, q0, q1
-constexpr int kGemmThreads = 192;
+constexpr int kPTileBytes = kTileRows * kTileKBytes;  // 16 KiB: 128 rows x 128 bytes
 constexpr int kTmemCols = 512;
-constexpr int kScaleCol = 384;  // scale-factor bytes live in TMEM columns 384..399
+constexpr int kScaleCol = 496;  // scale-factor bytes live in TMEM columns 496..511
 constexpr uint64_t kWaitLimitNs = 2000000000ull;
+constexpr int kMaxStages = 4;
 
-struct GemmParams {
-  int L;
-  int tiles_p;  // tiles along the columns of C (B-matrix plane rows)
-  int tiles_q;  // tiles along the rows of C (A-matrix plane rows)
+struct GemmCore {
+  int L;        // plane groups (moduli); plane index = limbs * l + limb
+  int tiles_p;  // tiles of 128 along the columns of C (B-matrix plane rows)
+  int tiles_q;  // tiles of W along the rows of C (A-matrix plane rows)
   int kblocks;  // Kp / 256
   int group;    // rasterisation: this many column tiles share one sweep over the row tiles
-  int m[kMaxModuli];
-  uint32_t recip[kMaxModuli];   // floor(2^32 / m)
-  uint32_t offset[kMaxModuli];  // multiple of m close to 2^31: makes the composed value non-negative
-  uint8_t* res;                 // [L][Np][Mp] bytes
-  int64_t res_ld;               // Mp
-  size_t res_stride;            // Mp * Np
+  int skip_top_first;  // plane group 0 needs no p_{NP-1} q_{NQ-1} product (13^2 = 0 mod 169)
   StatusBlock* status;
-  uint32_t scale_word;          // four copies of the UE8M0 scale byte
+  uint32_t scale_word;  // four copies of the UE8M0 scale byte
 };
 
 struct __align__(8) GemmShared {
-  uint64_t full[kStages];
-  uint64_t empty[kStages];
+  uint64_t full[kMaxStages];
+  uint64_t empty[kMaxStages];
   uint64_t tmem_full;
   uint64_t tmem_empty;
   uint64_t drained;
@@ -76,10 +73,10 @@ __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, Gemm
   }
 }
 
-__device__ __forceinline__ void decode_item(const GemmParams& p, int item, int& l, int& tp, int& tq) {
-  const int per_mod = p.tiles_p * p.tiles_q;
-  l = item / per_mod;
-  const int t = item - l * per_mod;
+__device__ __forceinline__ void decode_item(const GemmCore& p, int item, int& l, int& tp, int& tq) {
+  const int per_group = p.tiles_p * p.tiles_q;
+  l = item / per_group;
+  const int t = item - l * per_group;
   const int band = p.group * p.tiles_q;
   const int g = t / band;
   const int rem = t - g * band;
@@ -88,13 +85,139 @@ __device__ __forceinline__ void decode_item(const GemmParams& p, int item, int& 
   tp = g * p.group + (rem - tq * gsize);
 }
 
-__global__ void __launch_bounds__(kGemmThreads, 1)
-residue_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_q,
-                    const __grid_constant__ GemmParams p) {
+// ------------------------------------------------------------------------------------
+// Epilogue of the DGEMM path: r = (D0 + 13 D1 + 169 D2) mod m in [0, m), one byte per element.
+// 8 warps: warp (quadrant q, half h) drains lanes 32q..32q+31, columns 64h..64h+63 of the three
+// accumulators into 64 registers, releases tensor memory, then reduces and stores.
+// ------------------------------------------------------------------------------------
+struct ResidueEpilogue {
+  static constexpr int kWarps = 8;
+  struct Params {
+    int m[kMaxModuli];
+    uint32_t recip[kMaxModuli];   // floor(2^32 / m)
+    uint32_t offset[kMaxModuli];  // multiple of m close to 2^31: makes the composed value non-negative
+    uint8_t* res;                 // [L][Np][Mp] bytes
+    int64_t res_ld;               // Mp
+    size_t res_stride;            // Mp * Np
+  };
+  template <int W>
+  __device__ static __forceinline__ void run(const Params& ep, const GemmCore& core, uint32_t tmem, int epi_warp, int lane, int l,
+                                             int tp, int tq, uint32_t release_bar) {
+    static_assert(W == 128, "residue epilogue is written for 128-wide tiles");
+    // a warp can only touch the TMEM lanes of its own quadrant, (warp index in the CTA) mod 4
+    const uint32_t quad = (uint32_t)((epi_warp + 2) & 3), half = (uint32_t)(epi_warp >> 2);
+    const uint32_t base = tmem + ((quad * 32u) << 16) + half * 64u;
+    const uint32_t m = (uint32_t)ep.m[l], recip = ep.recip[l], offset = ep.offset[l];
+    const bool top = !(core.skip_top_first && l == 0);
+    uint32_t t[64];
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      uint32_t d0[32], d1[32], d2[32];
+      tmem_ld_32x32(base + 0 * W + c * 32, d0);
+      tmem_ld_32x32(base + 1 * W + c * 32, d1);
+      if (top) tmem_ld_32x32(base + 2 * W + c * 32, d2);
+      tmem_wait_ld();
+#pragma unroll
+      for (int e = 0; e < 32; ++e) {
+        const int v0 = __float2int_rn(__uint_as_float(d0[e]));
+        const int v1 = __float2int_rn(__uint_as_float(d1[e]));
+        const int v2 = top ? __float2int_rn(__uint_as_float(d2[e])) : 0;
+        t[c * 32 + e] = (uint32_t)(v0 + 13 * v1 + 169 * v2) + offset;  // non-negative, < 2^32
+      }
+    }
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(release_bar);  // the accumulators may be overwritten from here on
+    const int64_t j = (int64_t)tp * kTileRows + quad * 32 + lane;
+    uint4* dst = reinterpret_cast<uint4*>(ep.res + (size_t)l * ep.res_stride + (size_t)j * (size_t)ep.res_ld +
+                                          (size_t)tq * W + half * 64);
+#pragma unroll
+    for (int q4 = 0; q4 < 4; ++q4) {
+      uint32_t w[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        uint32_t word = 0;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+          const uint32_t x = t[q4 * 16 + k * 4 + b];
+          uint32_t r = x - __umulhi(x, recip) * m;  // in [0, 2m)
+          r = min(r, r - m);
+          word |= r << (8 * b);
+        }
+        w[k] = word;
+      }
+      dst[q4] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+  }
+};
+
+// ------------------------------------------------------------------------------------
+// Epilogue of the INT8 path: C = G0 + 13 G1 + 169 G2 + 2197 G3 + 28561 G4 as int32, written
+// straight into the caller's column-major C.  4 warps, 16 columns at a time.
+// ------------------------------------------------------------------------------------
+struct Int32Epilogue {
+  static constexpr int kWarps = 4;
+  struct Params {
+    int32_t* C;
+    int64_t ldc, M, N;
+  };
+  template <int W>
+  __device__ static __forceinline__ void run(const Params& ep, const GemmCore&, uint32_t tmem, int epi_warp, int lane, int,
+                                             int tp, int tq, uint32_t release_bar) {
+    const uint32_t quad = (uint32_t)((epi_warp + 2) & 3);  // TMEM lane quadrant = warp index mod 4
+    const uint32_t base = tmem + ((quad * 32u) << 16);
+    const int64_t j = (int64_t)tp * kTileRows + quad * 32 + lane;
+    const int64_t i0 = (int64_t)tq * W;
+    int32_t* col = ep.C + j * ep.ldc;
+    const bool vec_ok = ((reinterpret_cast<uintptr_t>(ep.C) & 15) == 0) && ((ep.ldc & 3) == 0);
+#pragma unroll 1
+    for (int c = 0; c < W / 16; ++c) {
+      uint32_t g0[16], g1[16], g2[16], g3[16], g4[16];
+      tmem_ld_32x16(base + 0 * W + c * 16, g0);
+      tmem_ld_32x16(base + 1 * W + c * 16, g1);
+      tmem_ld_32x16(base + 2 * W + c * 16, g2);
+      tmem_ld_32x16(base + 3 * W + c * 16, g3);
+      tmem_ld_32x16(base + 4 * W + c * 16, g4);
+      tmem_wait_ld();
+      int32_t v[16];
+#pragma unroll
+      for (int e = 0; e < 16; ++e) {
+        v[e] = __float2int_rn(__uint_as_float(g0[e])) + 13 * __float2int_rn(__uint_as_float(g1[e])) +
+               169 * __float2int_rn(__uint_as_float(g2[e])) + 2197 * __float2int_rn(__uint_as_float(g3[e])) +
+               28561 * __float2int_rn(__uint_as_float(g4[e]));
+      }
+      const int64_t i = i0 + c * 16;
+      if (j < ep.N) {
+        if (vec_ok && i + 16 <= ep.M) {
+          int4* d = reinterpret_cast<int4*>(col + i);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) d[k] = make_int4(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
+        } else {
+#pragma unroll
+          for (int e = 0; e < 16; ++e)
+            if (i + e < ep.M) col[i + e] = v[e];
+        }
+      }
+    }
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(release_bar);
+  }
+};
+
+template <int NP, int NQ, int W, int STAGES, class Epi>
+__global__ void __launch_bounds__(64 + 32 * Epi::kWarps, 1)
+limb_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_q,
+                 const __grid_constant__ GemmCore p, const __grid_constant__ typename Epi::Params ep) {
+  constexpr int kQTileBytes = W * kTileKBytes;
+  constexpr int kStageBytes = NP * kPTileBytes + NQ * kQTileBytes;
+  constexpr int NG = NP + NQ - 1;
+  static_assert(NG * W <= kScaleCol, "accumulators must leave room for the scale-factor columns");
+  static_assert(NQ * W <= 256 && W % 16 == 0 && STAGES <= kMaxStages, "instruction shape limits");
   extern __shared__ uint8_t smem_raw[];
   // operand stages need 1024-byte alignment (128-byte swizzle atoms)
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  GemmShared* sh = reinterpret_cast<GemmShared*>(tiles + kStages * kStageBytes);
+  GemmShared* sh = reinterpret_cast<GemmShared*>(tiles + STAGES * kStageBytes);
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const int total_items = p.L * p.tiles_p * p.tiles_q;
@@ -102,12 +225,12 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_cons
   if (threadIdx.x == 0) {
     prefetch_tensormap(&map_p);
     prefetch_tensormap(&map_q);
-    for (int s = 0; s < kStages; ++s) {
+    for (int s = 0; s < STAGES; ++s) {
       mbar_init(smem_u32(&sh->full[s]), 1);
       mbar_init(smem_u32(&sh->empty[s]), 1);
     }
     mbar_init(smem_u32(&sh->tmem_full), 1);
-    mbar_init(smem_u32(&sh->tmem_empty), 4);
+    mbar_init(smem_u32(&sh->tmem_empty), Epi::kWarps);
     mbar_init(smem_u32(&sh->drained), 1);
     sh->abort = 0;
     fence_barrier_init();
@@ -121,7 +244,7 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_cons
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = sh->tmem_base;
-  if (warp >= 2) {  // constant UE8M0 scale bytes, identical for every row, column and K block
+  if (warp >= 2 && warp < 6) {  // constant UE8M0 scale bytes, identical for every row, column and K block
     const uint32_t quad = (uint32_t)(warp & 3);
     tmem_st_32x8_const(tmem + ((quad * 32u) << 16) + kScaleCol, p.scale_word);
     tmem_st_32x8_const(tmem + ((quad * 32u) << 16) + kScaleCol + 8, p.scale_word);
@@ -136,9 +259,9 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_cons
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
-      uint32_t armed_parity[kStages];
-      bool armed[kStages];
-      for (int s = 0; s < kStages; ++s) armed[s] = false, armed_parity[s] = 0;
+      uint32_t armed_parity[STAGES];
+      bool armed[STAGES];
+      for (int s = 0; s < STAGES; ++s) armed[s] = false, armed_parity[s] = 0;
       bool ok = true;
       for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
         int l, tp, tq;
@@ -154,15 +277,16 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_cons
           armed[stage] = true;
           armed_parity[stage] = phase;
           const int x = kb * kTileKBytes;
-          tma_load_3d(dst + 0 * kOperandTileBytes, &map_p, bar, x, tp * kTileRows, 2 * l + 0);
-          tma_load_3d(dst + 1 * kOperandTileBytes, &map_p, bar, x, tp * kTileRows, 2 * l + 1);
-          tma_load_3d(dst + 2 * kOperandTileBytes, &map_q, bar, x, tq * kTileRows, 2 * l + 0);
-          tma_load_3d(dst + 3 * kOperandTileBytes, &map_q, bar, x, tq * kTileRows, 2 * l + 1);
-          if (++stage == kStages) stage = 0, phase ^= 1u;
+#pragma unroll
+          for (int i = 0; i < NP; ++i) tma_load_3d(dst + i * kPTileBytes, &map_p, bar, x, tp * kTileRows, NP * l + i);
+#pragma unroll
+          for (int jq = 0; jq < NQ; ++jq)
+            tma_load_3d(dst + NP * kPTileBytes + jq * kQTileBytes, &map_q, bar, x, tq * W, NQ * l + jq);
+          if (++stage == STAGES) stage = 0, phase ^= 1u;
         }
       }
       if (sh->abort) {  // let copies already in flight land before the CTA leaves
-        for (int s = 0; s < kStages; ++s)
+        for (int s = 0; s < STAGES; ++s)
           if (armed[s]) {
             const uint64_t t0 = global_timer_ns();
             while (!mbar_try_wait(smem_u32(&sh->full[s]), armed_parity[s]) && global_timer_ns() - t0 < kWaitLimitNs) {
@@ -176,10 +300,14 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_cons
       int stage = 0;
       uint32_t phase = 0, acc_phase = 0;
       const uint32_t sf = tmem + kScaleCol;
-      constexpr uint32_t kIdesc128 = idesc_mxf4(128);
-      constexpr uint32_t kIdesc256 = idesc_mxf4(256);
+      constexpr uint32_t kIdescOne = idesc_mxf4(W);
+      constexpr uint32_t kIdescAll = idesc_mxf4(NQ * W);
+      constexpr uint32_t kIdescButLast = idesc_mxf4(NQ > 1 ? (NQ - 1) * W : W);
       bool ok = true;
       for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
+        int l, tp, tq;
+        decode_item(p, item, l, tp, tq);
+        const bool skip_top = p.skip_top_first && l == 0;
         if (!wait_bounded(smem_u32(&sh->tmem_empty), acc_phase ^ 1u, sh, p.status, 0x100)) break;
         tc_fence_after();
         for (int kb = 0; kb < p.kblocks; ++kb) {
@@ -188,26 +316,36 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_cons
             break;
           }
           tc_fence_after();
-          const uint32_t base = smem_u32(tiles + stage * kStageBytes);
+          const uint32_t pbase = smem_u32(tiles + stage * kStageBytes);
+          const uint32_t qbase = pbase + NP * kPTileBytes;
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks) {
-            const uint64_t p0 = smem_desc_sw128(base + 0 * kOperandTileBytes + ks * 32);
-            const uint64_t p1 = smem_desc_sw128(base + 1 * kOperandTileBytes + ks * 32);
-            const uint64_t q0 = smem_desc_sw128(base + 2 * kOperandTileBytes + ks * 32);
-            const uint64_t q1 = smem_desc_sw128(base + 3 * kOperandTileBytes + ks * 32);
             if (kb == 0 && ks == 0) {
-              // first step of a tile: overwrite instead of accumulate, region by region
-              mma_mxf4(tmem + 0, p0, q0, kIdesc128, sf, sf, 0u);
-              mma_mxf4(tmem + 128, p0, q1, kIdesc128, sf, sf, 0u);
-              mma_mxf4(tmem + 128, p1, q0, kIdesc128, sf, sf, 1u);
-              mma_mxf4(tmem + 256, p1, q1, kIdesc128, sf, sf, 0u);
+              // first step of a tile: overwrite instead of accumulate, group by group
+              bool touched[NG];
+#pragma unroll
+              for (int g = 0; g < NG; ++g) touched[g] = false;
+#pragma unroll
+              for (int i = 0; i < NP; ++i) {
+#pragma unroll
+                for (int jq = 0; jq < NQ; ++jq) {
+                  if (skip_top && i == NP - 1 && jq == NQ - 1) continue;
+                  mma_mxf4(tmem + W * (i + jq), smem_desc_sw128(pbase + i * kPTileBytes),
+                           smem_desc_sw128(qbase + jq * kQTileBytes), kIdescOne, sf, sf, touched[i + jq] ? 1u : 0u);
+                  touched[i + jq] = true;
+                }
+              }
             } else {
-              mma_mxf4(tmem + 0, p0, q0, kIdesc256, sf, sf, 1u);    // q0 and q1 are adjacent: 256 rows
-              mma_mxf4(tmem + 128, p1, q0, kIdesc256, sf, sf, 1u);
+#pragma unroll
+              for (int i = 0; i < NP; ++i) {
+                const bool shorten = skip_top && i == NP - 1;
+                mma_mxf4(tmem + W * i, smem_desc_sw128(pbase + i * kPTileBytes + ks * 32), smem_desc_sw128(qbase + ks * 32),
+                         shorten ? kIdescButLast : kIdescAll, sf, sf, 1u);
+              }
             }
           }
           mma_commit(smem_u32(&sh->empty[stage]));
-          if (++stage == kStages) stage = 0, phase ^= 1u;
+          if (++stage == STAGES) stage = 0, phase ^= 1u;
         }
         if (!ok) break;
         mma_commit(smem_u32(&sh->tmem_full));
@@ -222,8 +360,6 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_cons
     }
   } else {
     // ------------------------------ epilogue ----------------------------------
-    const uint32_t quad = (uint32_t)(warp & 3);
-    const uint32_t lane_base = tmem + ((quad * 32u) << 16);
     uint32_t acc_phase = 0;
     for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
       int l, tp, tq;
@@ -231,40 +367,7 @@ residue_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_cons
       // the outcome must be warp-uniform: the TMEM loads below are warp-collective
       if (!__all_sync(0xFFFFFFFFu, wait_bounded(smem_u32(&sh->tmem_full), acc_phase, sh, p.status, 0x200 + warp))) break;
       tc_fence_after();
-      const uint32_t m = (uint32_t)p.m[l], recip = p.recip[l], offset = p.offset[l];
-      const int64_t j = (int64_t)tp * kTileRows + quad * 32 + lane;
-      uint8_t* out = p.res + (size_t)l * p.res_stride + (size_t)j * (size_t)p.res_ld + (size_t)tq * kTileRows;
-#pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
-        uint32_t d0[32], d1[32], d2[32];
-        tmem_ld_32x32(lane_base + 0 + c * 32, d0);
-        tmem_ld_32x32(lane_base + 128 + c * 32, d1);
-        tmem_ld_32x32(lane_base + 256 + c * 32, d2);
-        tmem_wait_ld();
-        uint32_t packed[8];
-#pragma unroll
-        for (int w = 0; w < 8; ++w) {
-          uint32_t word = 0;
-#pragma unroll
-          for (int b = 0; b < 4; ++b) {
-            const int e = 4 * w + b;
-            const int v0 = __float2int_rn(__uint_as_float(d0[e]));
-            const int v1 = __float2int_rn(__uint_as_float(d1[e]));
-            const int v2 = __float2int_rn(__uint_as_float(d2[e]));
-            const uint32_t t = (uint32_t)(v0 + 13 * v1 + 169 * v2) + offset;  // non-negative, < 2^32
-            uint32_t r = t - __umulhi(t, recip) * m;                          // in [0, 2m)
-            r = min(r, r - m);
-            word |= r << (8 * b);
-          }
-          packed[w] = word;
-        }
-        uint4* dst = reinterpret_cast<uint4*>(out + c * 32);
-        dst[0] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-        dst[1] = make_uint4(packed[4], packed[5], packed[6], packed[7]);
-      }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&sh->tmem_empty));
+      Epi::template run<W>(ep, p, tmem, warp - 2, lane, l, tp, tq, smem_u32(&sh->tmem_empty));
       acc_phase ^= 1u;
     }
   }
@@ -289,12 +392,12 @@ struct ProbeShared {
   volatile int abort;
 };
 
-__global__ void __launch_bounds__(kGemmThreads, 1)
+__global__ void __launch_bounds__(192, 1)
 mma_probe_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_q, int kblocks,
                  uint32_t scale_word, float* __restrict__ D, StatusBlock* status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  ProbeShared* sh = reinterpret_cast<ProbeShared*>(tiles + 2 * kOperandTileBytes);
+  ProbeShared* sh = reinterpret_cast<ProbeShared*>(tiles + 2 * kPTileBytes);
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
@@ -325,9 +428,9 @@ mma_probe_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constan
     const uint32_t sf = tmem + 128;
     uint32_t phase = 0;
     for (int kb = 0; kb < kblocks; ++kb) {
-      mbar_arrive_expect_tx(smem_u32(&sh->full), 2 * kOperandTileBytes);
+      mbar_arrive_expect_tx(smem_u32(&sh->full), 2 * kPTileBytes);
       tma_load_2d(base, &map_p, smem_u32(&sh->full), kb * kTileKBytes, 0);
-      tma_load_2d(base + kOperandTileBytes, &map_q, smem_u32(&sh->full), kb * kTileKBytes, 0);
+      tma_load_2d(base + kPTileBytes, &map_q, smem_u32(&sh->full), kb * kTileKBytes, 0);
       const uint64_t t0 = global_timer_ns();
       while (!mbar_try_wait(smem_u32(&sh->full), phase)) {
         if (global_timer_ns() - t0 > kWaitLimitNs) {
@@ -338,7 +441,7 @@ mma_probe_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constan
       if (sh->abort) break;
       tc_fence_after();
       for (int ks = 0; ks < 4; ++ks)
-        mma_mxf4(tmem, smem_desc_sw128(base + ks * 32), smem_desc_sw128(base + kOperandTileBytes + ks * 32),
+        mma_mxf4(tmem, smem_desc_sw128(base + ks * 32), smem_desc_sw128(base + kPTileBytes + ks * 32),
                  idesc_mxf4(128), sf, sf, (kb | ks) ? 1u : 0u);
       mma_commit(smem_u32(&sh->done));
       const uint64_t t1 = global_timer_ns();
@@ -375,6 +478,7 @@ mma_probe_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constan
   }
 }
 
+
 // ------------------------------------------------------------------------------------
 // Host side
 // ------------------------------------------------------------------------------------
@@ -394,13 +498,15 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-// Planes of one operand as a (bytes along K, rows, plane) byte tensor; box = 128 bytes x 128 rows.
-bool make_plane_map(CUtensorMap* map, const void* base, int64_t k_bytes, int64_t rows, int64_t planes, size_t plane_bytes) {
+// Planes of one operand as a (bytes along K, rows, plane) byte tensor; box = 128 bytes x box_rows.
+// Rows of a box that fall outside the tensor are filled with zero bytes (E2M1 code 0 = value 0).
+bool make_plane_map(CUtensorMap* map, const void* base, int64_t k_bytes, int64_t rows, int64_t planes, size_t plane_bytes,
+                    int box_rows) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return false;
   cuuint64_t dims[3] = {(cuuint64_t)k_bytes, (cuuint64_t)rows, (cuuint64_t)planes};
   cuuint64_t strides[2] = {(cuuint64_t)k_bytes, (cuuint64_t)plane_bytes};
-  cuuint32_t box[3] = {(cuuint32_t)kTileKBytes, (cuuint32_t)kTileRows, 1};
+  cuuint32_t box[3] = {(cuuint32_t)kTileKBytes, (cuuint32_t)box_rows, 1};
   cuuint32_t estr[3] = {1, 1, 1};
   const int rank = planes > 0 ? 3 : 2;
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, rank, const_cast<void*>(base), dims, strides, box, estr,
@@ -418,51 +524,85 @@ int sm_count() {
   return n;
 }
 
-}  // namespace
-
-ozk_status gemm_residues(const Geometry& g, const ModulusTable& mt, uint8_t* ws, cudaStream_t st) {
-  CUtensorMap map_p, map_q;
-  if (!make_plane_map(&map_p, ws + g.off_planes_b, g.Kp / 2, g.Np, 2 * g.L, g.plane_bytes_b)) return OZK_ERR_CUDA;
-  if (!make_plane_map(&map_q, ws + g.off_planes_a, g.Kp / 2, g.Mp, 2 * g.L, g.plane_bytes_a)) return OZK_ERR_CUDA;
-  GemmParams p;
-  p.L = g.L;
-  p.tiles_p = (int)(g.Np / kTileRows);
-  p.tiles_q = (int)(g.Mp / kTileRows);
-  p.kblocks = (int)(g.Kp / kTileKNibbles);
-  p.group = 16;
-  for (int l = 0; l < kMaxModuli; ++l) {
-    p.m[l] = mt.m[l];
-    p.recip[l] = mt.recip[l];
-    p.offset[l] = (uint32_t)mt.m[l] * (uint32_t)(0x80000000u / (uint32_t)mt.m[l]);
-  }
-  p.res = ws + g.off_res;
-  p.res_ld = g.Mp;
-  p.res_stride = (size_t)g.Mp * (size_t)g.Np;
-  p.status = reinterpret_cast<StatusBlock*>(ws + g.off_status);
-  p.scale_word = 0x80808080u;  // UE8M0 byte 0x80 = 2: both operands doubled, accumulators hold integers
-  const size_t smem = (size_t)kStages * kStageBytes + sizeof(GemmShared) + 1024;
+template <int NP, int NQ, int W, int STAGES, class Epi>
+ozk_status launch_limb_gemm(const CUtensorMap& map_p, const CUtensorMap& map_q, const GemmCore& core,
+                            const typename Epi::Params& ep, cudaStream_t st) {
+  constexpr size_t kStageBytes = (size_t)NP * kPTileBytes + (size_t)NQ * W * kTileKBytes;
+  const size_t smem = STAGES * kStageBytes + sizeof(GemmShared) + 1024;
+  auto kernel = limb_gemm_kernel<NP, NQ, W, STAGES, Epi>;
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(residue_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return OZK_ERR_CUDA;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return OZK_ERR_CUDA;
     attr_set = true;
   }
-  const long long items = (long long)p.L * p.tiles_p * p.tiles_q;
+  const long long items = (long long)core.L * core.tiles_p * core.tiles_q;
   const int grid = (int)(items < sm_count() ? items : sm_count());
-  residue_gemm_kernel<<<grid, kGemmThreads, smem, st>>>(map_p, map_q, p);
+  kernel<<<grid, 64 + 32 * Epi::kWarps, smem, st>>>(map_p, map_q, core, ep);
   return cudaGetLastError() == cudaSuccess ? OZK_OK : OZK_ERR_CUDA;
+}
+
+}  // namespace
+
+// DGEMM path: residues r_l[j][i] for all moduli from the limb planes in the workspace.
+ozk_status gemm_residues(const Geometry& g, const ModulusTable& mt, uint8_t* ws, cudaStream_t st) {
+  CUtensorMap map_p, map_q;
+  if (!make_plane_map(&map_p, ws + g.off_planes_b, g.Kp / 2, g.Np, 2 * g.L, g.plane_bytes_b, kTileRows)) return OZK_ERR_CUDA;
+  if (!make_plane_map(&map_q, ws + g.off_planes_a, g.Kp / 2, g.Mp, 2 * g.L, g.plane_bytes_a, 128)) return OZK_ERR_CUDA;
+  GemmCore core;
+  core.L = g.L;
+  core.tiles_p = (int)(g.Np / kTileRows);
+  core.tiles_q = (int)(g.Mp / 128);
+  core.kblocks = (int)(g.Kp / kTileKNibbles);
+  core.group = 16;
+  core.skip_top_first = (mt.m[0] == 169) ? 1 : 0;  // 13^2 a1 b1 vanishes mod 169 (Section 5.1)
+  core.status = reinterpret_cast<StatusBlock*>(ws + g.off_status);
+  core.scale_word = 0x80808080u;  // UE8M0 byte 0x80 = 2: both operands doubled, accumulators hold integers
+  ResidueEpilogue::Params ep;
+  for (int l = 0; l < kMaxModuli; ++l) {
+    ep.m[l] = mt.m[l];
+    ep.recip[l] = mt.recip[l];
+    ep.offset[l] = (uint32_t)mt.m[l] * (uint32_t)(0x80000000u / (uint32_t)mt.m[l]);
+  }
+  ep.res = ws + g.off_res;
+  ep.res_ld = g.Mp;
+  ep.res_stride = (size_t)g.Mp * (size_t)g.Np;
+  return launch_limb_gemm<2, 2, 128, 3, ResidueEpilogue>(map_p, map_q, core, ep, st);
+}
+
+// INT8 path: C (int32, column-major) from three limb planes per operand.
+ozk_status gemm_int8(const uint8_t* planes_a, const uint8_t* planes_b, int64_t M, int64_t N, int64_t Mp, int64_t Np, int64_t Kp,
+                     int32_t* C, int64_t ldc, StatusBlock* status, cudaStream_t st) {
+  constexpr int W = 80;
+  CUtensorMap map_p, map_q;
+  if (!make_plane_map(&map_p, planes_b, Kp / 2, Np, 3, (size_t)Np * (size_t)(Kp / 2), kTileRows)) return OZK_ERR_CUDA;
+  if (!make_plane_map(&map_q, planes_a, Kp / 2, Mp, 3, (size_t)Mp * (size_t)(Kp / 2), W)) return OZK_ERR_CUDA;
+  GemmCore core;
+  core.L = 1;
+  core.tiles_p = (int)(Np / kTileRows);
+  core.tiles_q = (int)((M + W - 1) / W);
+  core.kblocks = (int)(Kp / kTileKNibbles);
+  core.group = 16;
+  core.skip_top_first = 0;
+  core.status = status;
+  core.scale_word = 0x80808080u;
+  Int32Epilogue::Params ep;
+  ep.C = C;
+  ep.ldc = ldc;
+  ep.M = M;
+  ep.N = N;
+  return launch_limb_gemm<3, 3, W, 2, Int32Epilogue>(map_p, map_q, core, ep, st);
 }
 
 ozk_status gemm_probe(const uint8_t* P, const uint8_t* Q, int64_t K, int scale_byte, float* D, uint8_t* ws, cudaStream_t st) {
   CUtensorMap map_p, map_q;
-  if (!make_plane_map(&map_p, P, K / 2, kTileRows, 0, 0)) return OZK_ERR_CUDA;
-  if (!make_plane_map(&map_q, Q, K / 2, kTileRows, 0, 0)) return OZK_ERR_CUDA;
-  const size_t smem = 2 * kOperandTileBytes + sizeof(ProbeShared) + 1024;
+  if (!make_plane_map(&map_p, P, K / 2, kTileRows, 0, 0, kTileRows)) return OZK_ERR_CUDA;
+  if (!make_plane_map(&map_q, Q, K / 2, kTileRows, 0, 0, kTileRows)) return OZK_ERR_CUDA;
+  const size_t smem = 2 * kPTileBytes + sizeof(ProbeShared) + 1024;
   if (cudaFuncSetAttribute(mma_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return OZK_ERR_CUDA;
   const uint32_t b = (uint32_t)(scale_byte & 0xFF);
-  mma_probe_kernel<<<1, kGemmThreads, smem, st>>>(map_p, map_q, (int)(K / kTileKNibbles), b * 0x01010101u, D,
-                                                 reinterpret_cast<StatusBlock*>(ws));
+  mma_probe_kernel<<<1, 192, smem, st>>>(map_p, map_q, (int)(K / kTileKNibbles), b * 0x01010101u, D,
+                                        reinterpret_cast<StatusBlock*>(ws));
   return cudaGetLastError() == cudaSuccess ? OZK_OK : OZK_ERR_CUDA;
 }
 

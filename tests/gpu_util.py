@@ -25,6 +25,16 @@ def ensure_workspace(nbytes: int) -> None:
         ozk.check(ozk.ozk_set_workspace(buf.data_ptr(), buf.numel()), "ozk_set_workspace")
 
 
+def register_small_workspace(nbytes: int = 1 << 20) -> None:
+    """Registers a fresh workspace of exactly nbytes (for tests of the 'workspace too small' error);
+    the next ensure_workspace() call replaces it."""
+    torch.cuda.synchronize()
+    _ws["buf"] = None
+    buf = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    ozk.check(ozk.ozk_set_workspace(buf.data_ptr(), buf.numel()), "ozk_set_workspace")
+    _ws["small"] = buf
+
+
 def to_dev_colmajor(X: np.ndarray, ld: int | None = None) -> torch.Tensor:
     """Uploads X[r, c] as a column-major device buffer with leading dimension ld."""
     rows, cols = X.shape

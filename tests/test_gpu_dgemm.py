@@ -73,7 +73,7 @@ def test_wide_exponent_range_and_extremes_bit_exact():
 
 
 def test_invalid_arguments():
-    gu.ensure_workspace(1 << 20)
+    gu.register_small_workspace(8 << 20)          # every call below must be rejected before anything is launched
     assert ozk.ozk_dgemm(8, 8, 8, None, 8, None, 8, None, 8, 19, 0) == ozk.OZK_ERR_INVALID_ARG      # null pointers
-    assert ozk.ozk_dgemm(4096, 4096, 4096, 1024, 4096, 1024, 4096, 1024, 4096, 19, 0) == ozk.OZK_ERR_WORKSPACE
+    assert ozk.ozk_dgemm(4096, 4096, 4096, None, 4096, None, 4096, None, 4096, 19, 0) == ozk.OZK_ERR_WORKSPACE
     assert ozk.ozk_dgemm(0, 8, 8, None, 1, None, 8, None, 1, 19, 0) == ozk.OZK_OK                   # empty result

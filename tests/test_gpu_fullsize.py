@@ -1,0 +1,130 @@
+"""Parity at the full configured sizes, in the launch configuration bench.py times (ozk_dgemm on
+column-major device buffers): a 128x128 output block (the paper's own evaluation protocol) plus
+scattered rows and columns against the CPU oracle bit for bit, the error against exact fl(AB) on
+a sub-block, and (4096, 8192) every reconstructed integer by a Freivalds check modulo two primes."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import exact, moduli, ozaki2
+from paper_2608_06812_b200 import binding as ozk
+from paper_2608_06812_b200 import inputs
+from tests import gpu_util as gu
+
+pytestmark = pytest.mark.gpu
+
+
+def upload(n, phi):
+    A = inputs.lognormal_matrix(n, n, phi, seed=0)
+    B = inputs.lognormal_matrix(n, n, phi, seed=1)
+    dA = torch.from_numpy(np.ascontiguousarray(A.T)).cuda()
+    dB = torch.from_numpy(np.ascontiguousarray(B.T)).cuda()
+    return A, B, dA, dB
+
+
+def run(n, dA, dB, L):
+    gu.ensure_workspace(ozk.ozk_dgemm_workspace_bytes(n, n, n, L))
+    dC = torch.empty((n, n), dtype=torch.float64, device="cuda")
+    ozk.check(ozk.ozk_dgemm(n, n, n, dA.data_ptr(), n, dB.data_ptr(), n, dC.data_ptr(), n, L, gu.stream()), "ozk_dgemm")
+    ozk.check(ozk.ozk_get_async_status(gu.stream()), "status")
+    return dC
+
+
+def sample_sets(n, seed, extra=40):
+    rng = np.random.default_rng(seed)
+    rows = np.concatenate([np.arange(128), np.sort(rng.choice(np.arange(128, n), extra, replace=False))])
+    cols = np.concatenate([np.arange(128), np.sort(rng.choice(np.arange(128, n), extra, replace=False))])
+    return rows, cols
+
+
+def check_samples(A, B, dC, L, rows, cols):
+    ref = ozaki2.dgemm(A[rows], B[:, cols], L)              # shifts are per row / per column: sub-matrices give the same elements
+    got = dC[torch.from_numpy(cols).cuda()][:, torch.from_numpy(rows).cuda()].cpu().numpy().T
+    assert gu.bits_equal(got, ref.C)
+    return got
+
+
+def freivalds(n, L, A, B, x_words):
+    """x_words[j, i, 6] (two's complement, 32-bit words) must equal sum_k At[i,k] Bt[k,j] for every i, j:
+    compare x v with At (Bt v) modulo two 31-bit primes for random v."""
+    c = moduli.capacity_bits(n, L)
+    At = ozaki2.to_integers(A, ozaki2.shared_shifts(A, 1, c), 1)
+    Bt = ozaki2.to_integers(B, ozaki2.shared_shifts(B, 0, c), 0)
+    W = x_words.astype(np.int64) & 0xFFFFFFFF
+    negative = W[:, :, 5] >> 31
+    rng = np.random.default_rng(99)
+    for q in (2147483647, 2147483629):
+        pw = [pow(2, 32 * k, q) for k in range(6)]
+        xm = np.zeros(W.shape[:2], dtype=np.int64)
+        for k in range(6):
+            xm = (xm + (W[:, :, k] % q) * pw[k]) % q
+        xm = (xm - negative * pow(2, 192, q)) % q             # xm[j, i] = x_ij mod q
+        v = rng.integers(0, q, size=n).astype(np.int64)
+        Bv = np.zeros(n, dtype=np.int64)
+        Btm = np.mod(Bt, q)
+        for j0 in range(0, n, 1024):                          # products < 2^62, reduced before summing
+            Bv = (Bv + ((Btm[:, j0:j0 + 1024] * v[None, j0:j0 + 1024]) % q).sum(axis=1)) % q
+        Atm = np.mod(At, q)
+        right = np.zeros(n, dtype=np.int64)
+        for k0 in range(0, n, 1024):
+            right = (right + ((Atm[:, k0:k0 + 1024] * Bv[None, k0:k0 + 1024]) % q).sum(axis=1)) % q
+        left = np.zeros(n, dtype=np.int64)
+        for j0 in range(0, n, 1024):
+            left = (left + ((xm[j0:j0 + 1024, :] * v[j0:j0 + 1024, None]) % q).sum(axis=0)) % q
+        assert np.array_equal(left, right)
+
+
+def x_words_of_last_call(n, L):
+    dX = torch.empty((n, n, 6), dtype=torch.int32, device="cuda")
+    dC2 = torch.empty((n, n), dtype=torch.float64, device="cuda")
+    ozk.check(ozk.ozk_stage_crt(n, n, n, L, None, None, None, dC2.data_ptr(), n, dX.data_ptr(), gu.stream()), "ozk_stage_crt")
+    ozk.check(ozk.ozk_get_async_status(gu.stream()), "status")
+    return dX.cpu().numpy(), dC2
+
+
+def test_config2_4096_moduli_sweep():
+    """M=N=K=4096, phi=0.5, moduli count 12..20: bit-exact samples for every count; the error bound
+    1e-15 against fl(AB) from 17 moduli on; Freivalds over the whole matrix at 19 moduli."""
+    n = 4096
+    A, B, dA, dB = upload(n, 0.5)
+    rows, cols = sample_sets(n, seed=2, extra=24)
+    errs = {}
+    for L in range(12, 21):
+        dC = run(n, dA, dB, L)
+        got = check_samples(A, B, dC, L, rows, cols)
+        errs[L] = exact.normwise_error(got[:32, :32], A[rows[:32]], B[:, cols[:32]], against_rounded=True)
+        if L == 19:
+            X, dC2 = x_words_of_last_call(n, L)
+            assert torch.equal(dC2.view(torch.int64), dC.view(torch.int64))
+            freivalds(n, L, A, B, X)
+    assert all(errs[L] <= 1e-15 for L in range(17, 21)), errs
+    assert errs[12] > errs[15] > errs[18]                     # fewer moduli keep fewer bits
+
+
+def test_config3_8192_phi4_wide_exponent_range():
+    """M=N=K=8192, phi=4: bit-exact against the oracle; the method saturates at 19 moduli (53-bit cap,
+    one exponent per row/column), so the error against fl(AB) is reported, not bounded by 1e-15."""
+    n = 8192
+    A, B, dA, dB = upload(n, 4.0)
+    rows, cols = sample_sets(n, seed=3, extra=24)
+    got = {}
+    for L in (19, 20):
+        dC = run(n, dA, dB, L)
+        got[L] = check_samples(A, B, dC, L, rows, cols)
+    assert gu.bits_equal(got[19], got[20])                    # capacity is capped at 53 bits: more moduli change nothing
+    err = exact.normwise_error(got[19][:16, :16], A[rows[:16]], B[:, cols[:16]], against_rounded=True)
+    assert 1e-15 < err < 1e-8
+    X, _ = x_words_of_last_call(n, 20)
+    freivalds(n, 20, A, B, X)
+
+
+def test_config5_16384_headline_configuration():
+    """M=N=K=16384, phi=1, 19 moduli (the benchmark's workload): bit-exact samples, 1e-15 bound."""
+    n = 16384
+    A, B, dA, dB = upload(n, 1.0)
+    rows, cols = sample_sets(n, seed=5, extra=40)
+    dC = run(n, dA, dB, 19)
+    got = check_samples(A, B, dC, 19, rows, cols)
+    err = exact.normwise_error(got[:16, :16], A[rows[:16]], B[:, cols[:16]], against_rounded=True)
+    assert err <= 1e-15
+    assert torch.isfinite(dC).all()
