@@ -157,7 +157,10 @@ def round_scaled_to_double(x: int, shift: int) -> float:
         return 0.0
     if shift >= 0:
         return x / (1 << shift)
-    return float(x << (-shift))
+    try:
+        return float(x << (-shift))
+    except OverflowError:            # beyond the FP64 range: IEEE 754 round-to-nearest gives +-infinity
+        return math.copysign(math.inf, x)
 
 
 @dataclass

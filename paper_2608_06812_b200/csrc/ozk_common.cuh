@@ -14,7 +14,7 @@ constexpr int kTileKNibbles = 256;   // k extent of one pipeline stage: 256 E2M1
 constexpr int kTileKBytes = 128;
 constexpr int kMaxModuli = OZK_MAX_MODULI;
 constexpr int kCrtWords = 6;         // 192-bit integers cover sum r_l w_l for all 27 moduli
-constexpr int kLutStride = 176;      // bytes reserved per modulus in the limb-pair table (m <= 169)
+constexpr int kLutStride = 352;      // 16-bit entries per modulus in the limb-pair table: residues 0 .. 2m-1, m <= 169
 
 // ---- status word (first bytes of the workspace) -------------------------------------
 struct StatusBlock {
@@ -54,6 +54,8 @@ struct CrtTable {
   uint32_t P[kCrtWords];
   uint32_t halfP[kCrtWords];               // floor(P / 2)
   double inv_P;                            // 1 / P rounded to double
+  double q_scale;                          // (2^96 / P) (1 - 2^-30): quotient estimate from the words above bit 96
+  int p_bits;                              // bit length of P
 };
 
 // registered workspace (ozk_api.cu)

@@ -197,6 +197,219 @@ __global__ void __launch_bounds__(256) crt_kernel(CrtTable ct, const uint8_t* __
   }
 }
 
+
+// ------------------------------------------------------------------------------------
+// Fast variant for aligned inputs: one thread reconstructs four consecutive rows i of one column j.
+//   * residues come in as one 32-bit load per modulus (four bytes = four rows)
+//   * S = sum r_l w_l is accumulated limb by limb in independent 64-bit sums (r < 2^8, w limb < 2^32,
+//     at most 27 terms: no carries until the end), one multiply-add per (modulus, limb)
+//   * the rounding builds the FP64 bit pattern directly (normalise, 53 bits, round bit, sticky); a
+//     result in the subnormal range takes the general routine above
+// ------------------------------------------------------------------------------------
+template <int NW>
+__device__ __forceinline__ double round_scaled_fast(const uint32_t (&mag)[NW], int shift) {
+  // top non-zero word and the two words below it
+  int top = -1;
+#pragma unroll
+  for (int i = 0; i < NW; ++i)
+    if (mag[i]) top = i;
+  if (top < 0) return 0.0;
+  uint32_t w2 = 0, w1 = 0, w0 = 0, rest = 0;
+#pragma unroll
+  for (int i = 0; i < NW; ++i) {
+    if (i == top) w2 = mag[i];
+    if (i == top - 1) w1 = mag[i];
+    if (i == top - 2) w0 = mag[i];
+    if (i < top - 2) rest |= mag[i];
+  }
+  const int lz = __clz(w2);
+  const int bitlen = 32 * top + 32 - lz;
+  const int e_out = bitlen - 1 - shift;  // value in [2^e_out, 2^(e_out+1))
+  if (e_out < -1022 || e_out > 1023) return round_scaled<NW>(mag, shift);  // subnormal or overflowing: general path
+  // 64-bit window with the value's top bit at bit 63: the top 64 bits of (w2:w1:w0) << lz
+  const uint32_t h1 = __funnelshift_l(w1, w2, lz), h0 = __funnelshift_l(w0, w1, lz);
+  const unsigned long long h = ((unsigned long long)h1 << 32) | h0;
+  const uint32_t below = (w0 << lz) | rest;  // everything under the window (for lz = 0 all of w0)
+  unsigned long long mant = h >> 11;         // 53 bits, leading one at bit 52
+  const bool round_bit = ((h >> 10) & 1ull) != 0ull;
+  const bool sticky = ((h & 0x3FFull) != 0ull) || (below != 0u);
+  if (round_bit && (sticky || (mant & 1ull))) ++mant;
+  // exponent field and mantissa in one addition: the leading one adds 1 to the exponent field, and a
+  // carry out of the mantissa (mant = 2^53) moves the result to the next binade (or to infinity)
+  return __longlong_as_double((long long)(((unsigned long long)(e_out + 1022) << 52) + mant));
+}
+
+
+// Lean reconstruction for 2^100 <= P < 2^126 (16 to 19 moduli): the weighted sum S (five words)
+// arrives as four 64-bit column sums; everything after the quotient estimate is 128-bit arithmetic
+// written as explicit carry chains.
+//   q  = floor((S >> 96) * (2^96 / P) * (1 - 2^-30))  is the true quotient or one below it, so
+//   x  = S - q P  lies in [0, 2P) and fits 128 bits; one conditional subtraction brings it below P.
+__device__ __forceinline__ double reconstruct_lean(const unsigned long long (&acc)[4], const CrtTable& ct, int shift) {
+  const uint32_t a0l = (uint32_t)acc[0], a0h = (uint32_t)(acc[0] >> 32), a1l = (uint32_t)acc[1], a1h = (uint32_t)(acc[1] >> 32);
+  const uint32_t a2l = (uint32_t)acc[2], a2h = (uint32_t)(acc[2] >> 32), a3l = (uint32_t)acc[3], a3h = (uint32_t)(acc[3] >> 32);
+  uint32_t S1, S2, S3, S4;
+  asm("add.cc.u32 %0, %4, %5;\n\t"
+      "addc.cc.u32 %1, %6, %7;\n\t"
+      "addc.cc.u32 %2, %8, %9;\n\t"
+      "addc.u32 %3, %10, 0;"
+      : "=r"(S1), "=r"(S2), "=r"(S3), "=r"(S4)
+      : "r"(a0h), "r"(a1l), "r"(a1h), "r"(a2l), "r"(a2h), "r"(a3l), "r"(a3h));
+  const uint32_t S0 = a0l;
+  const unsigned long long top = ((unsigned long long)S4 << 32) | S3;
+  const uint32_t q = __double2uint_rz(__ull2double_rz(top) * ct.q_scale);
+  const unsigned long long m0 = (unsigned long long)q * ct.P[0];
+  const unsigned long long m1 = (unsigned long long)q * ct.P[1] + (m0 >> 32);
+  const unsigned long long m2 = (unsigned long long)q * ct.P[2] + (m1 >> 32);
+  const unsigned long long m3 = (unsigned long long)q * ct.P[3] + (m2 >> 32);
+  uint32_t x0, x1, x2, x3;
+  asm("sub.cc.u32 %0, %4, %8;\n\t"
+      "subc.cc.u32 %1, %5, %9;\n\t"
+      "subc.cc.u32 %2, %6, %10;\n\t"
+      "subc.u32 %3, %7, %11;"
+      : "=r"(x0), "=r"(x1), "=r"(x2), "=r"(x3)
+      : "r"(S0), "r"(S1), "r"(S2), "r"(S3), "r"((uint32_t)m0), "r"((uint32_t)m1), "r"((uint32_t)m2), "r"((uint32_t)m3));
+  const uint32_t P0 = ct.P[0], P1 = ct.P[1], P2 = ct.P[2], P3 = ct.P[3];
+  uint32_t d0, d1, d2, d3, below;  // d = x - P; below = all ones if x < P
+  asm("sub.cc.u32 %0, %5, %9;\n\t"
+      "subc.cc.u32 %1, %6, %10;\n\t"
+      "subc.cc.u32 %2, %7, %11;\n\t"
+      "subc.cc.u32 %3, %8, %12;\n\t"
+      "subc.u32 %4, 0, 0;"
+      : "=r"(d0), "=r"(d1), "=r"(d2), "=r"(d3), "=r"(below)
+      : "r"(x0), "r"(x1), "r"(x2), "r"(x3), "r"(P0), "r"(P1), "r"(P2), "r"(P3));
+  if (!below) x0 = d0, x1 = d1, x2 = d2, x3 = d3;
+  uint32_t e0, e1, e2, e3;  // e = P - x
+  asm("sub.cc.u32 %0, %4, %8;\n\t"
+      "subc.cc.u32 %1, %5, %9;\n\t"
+      "subc.cc.u32 %2, %6, %10;\n\t"
+      "subc.u32 %3, %7, %11;"
+      : "=r"(e0), "=r"(e1), "=r"(e2), "=r"(e3)
+      : "r"(P0), "r"(P1), "r"(P2), "r"(P3), "r"(x0), "r"(x1), "r"(x2), "r"(x3));
+  uint32_t u0, u1, u2, u3, over;  // halfP - x borrows exactly when x > P/2
+  asm("sub.cc.u32 %0, %5, %9;\n\t"
+      "subc.cc.u32 %1, %6, %10;\n\t"
+      "subc.cc.u32 %2, %7, %11;\n\t"
+      "subc.cc.u32 %3, %8, %12;\n\t"
+      "subc.u32 %4, 0, 0;"
+      : "=r"(u0), "=r"(u1), "=r"(u2), "=r"(u3), "=r"(over)
+      : "r"(ct.halfP[0]), "r"(ct.halfP[1]), "r"(ct.halfP[2]), "r"(ct.halfP[3]), "r"(x0), "r"(x1), "r"(x2), "r"(x3));
+  uint32_t mag[4];
+  mag[0] = over ? e0 : x0;
+  mag[1] = over ? e1 : x1;
+  mag[2] = over ? e2 : x2;
+  mag[3] = over ? e3 : x3;
+  const double r = round_scaled_fast<4>(mag, shift);
+  return over ? -r : r;
+}
+
+template <int WW, int NW, bool LEAN>
+__global__ void __launch_bounds__(256) crt4_kernel(const __grid_constant__ CrtTable ct, const uint8_t* __restrict__ res,
+                                                   int64_t res_ld, size_t res_stride, const int32_t* __restrict__ s,
+                                                   const int32_t* __restrict__ t, int64_t M, int64_t N,
+                                                   double* __restrict__ C, int64_t ldc) {
+  const int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  if (i >= M) return;
+  for (int64_t j = blockIdx.y; j < N; j += gridDim.y) {
+    const uint8_t* rp = res + (size_t)j * (size_t)res_ld + (size_t)i;
+    unsigned long long acc[4][WW];
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+#pragma unroll
+      for (int k = 0; k < WW; ++k) acc[e][k] = 0ull;
+    // all residue loads are issued before the first use: 19..27 independent 128-byte requests per
+    // warp in flight instead of one (the streams of the moduli are 'res_stride' bytes apart)
+    uint32_t r4[kMaxModuli];
+#pragma unroll
+    for (int l = 0; l < kMaxModuli; ++l)
+      r4[l] = (l < ct.L) ? __ldg(reinterpret_cast<const uint32_t*>(rp + (size_t)l * res_stride)) : 0u;
+#pragma unroll
+    for (int l = 0; l < kMaxModuli; ++l) {
+      if (l < ct.L) {
+#pragma unroll
+        for (int k = 0; k < WW; ++k) {
+          const uint32_t w = ct.w[l][k];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) acc[e][k] += (unsigned long long)((r4[l] >> (8 * e)) & 0xFFu) * w;
+        }
+      }
+    }
+    const int tj = t[j];
+    const int4 s4 = *reinterpret_cast<const int4*>(s + i);
+    const int sh[4] = {s4.x + tj, s4.y + tj, s4.z + tj, s4.w + tj};
+    double out[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      if constexpr (LEAN) {
+        static_assert(!LEAN || (WW == 4 && NW == 5), "the lean tail is written for 4 weight words, 5 sum words");
+        unsigned long long a4[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) a4[k] = acc[e][k < WW ? k : 0];
+        out[e] = reconstruct_lean(a4, ct, sh[e]);
+        continue;
+      }
+      uint32_t S[NW];
+      unsigned long long carry = 0ull;
+#pragma unroll
+      for (int k = 0; k < NW; ++k) {
+        const unsigned long long v = (k < WW ? acc[e][k] : 0ull) + carry;
+        S[k] = (uint32_t)v;
+        carry = v >> 32;
+      }
+      // quotient estimate from the three top words (truncation error << 1), exact correction
+      double Sd = (double)S[NW - 1];
+      if (NW >= 2) Sd = Sd * 4294967296.0 + (double)S[NW - 2];
+      if (NW >= 3) Sd = Sd * 4294967296.0 + (double)S[NW - 3];
+      if (NW > 3) Sd *= __longlong_as_double((long long)(1023 + 32 * (NW - 3)) << 52);
+      const uint32_t q = (uint32_t)(Sd * ct.inv_P);
+      uint32_t borrow = 0, mc = 0;
+#pragma unroll
+      for (int k = 0; k < NW; ++k) {
+        const unsigned long long prod = (unsigned long long)q * ct.P[k] + mc;
+        mc = (uint32_t)(prod >> 32);
+        const unsigned long long d = (unsigned long long)S[k] - (uint32_t)prod - borrow;
+        S[k] = (uint32_t)d;
+        borrow = (uint32_t)(d >> 63);
+      }
+      uint32_t signw = 0u - mc - borrow;
+#pragma unroll 1
+      for (int it = 0; it < 2 && signw != 0; ++it) {
+        uint32_t c2 = 0;
+#pragma unroll
+        for (int k = 0; k < NW; ++k) {
+          const unsigned long long v = (unsigned long long)S[k] + ct.P[k] + c2;
+          S[k] = (uint32_t)v;
+          c2 = (uint32_t)(v >> 32);
+        }
+        signw += c2;
+      }
+#pragma unroll 1
+      for (int it = 0; it < 2 && ge<NW>(S, ct.P); ++it) sub_in_place<NW>(S, ct.P);
+      bool neg = false;
+      if (gt<NW>(S, ct.halfP)) {
+        uint32_t tmp[NW];
+#pragma unroll
+        for (int k = 0; k < NW; ++k) tmp[k] = ct.P[k];
+        sub_in_place<NW>(tmp, S);
+#pragma unroll
+        for (int k = 0; k < NW; ++k) S[k] = tmp[k];
+        neg = true;
+      }
+      const double mag = round_scaled_fast<NW>(S, sh[e]);
+      out[e] = neg ? -mag : mag;
+    }
+    double* dst = C + i + j * ldc;
+    if (i + 4 <= M && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0)) {
+      reinterpret_cast<double2*>(dst)[0] = make_double2(out[0], out[1]);
+      reinterpret_cast<double2*>(dst)[1] = make_double2(out[2], out[3]);
+    } else {
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+        if (i + e < M) dst[e] = out[e];
+    }
+  }
+}
+
 __global__ void copy_residues_kernel(const uint8_t* __restrict__ res, int64_t Mp, size_t res_stride, int64_t M, int64_t N,
                                      uint8_t* __restrict__ out) {
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -211,6 +424,28 @@ __global__ void copy_residues_kernel(const uint8_t* __restrict__ res, int64_t Mp
 
 cudaError_t launch_crt(const Geometry& g, const CrtTable& ct, const uint8_t* res, int64_t res_ld, size_t res_stride,
                        const int32_t* s, const int32_t* t, double* C, int64_t ldc, uint32_t* x_out, cudaStream_t st) {
+  // weight words actually used, and whether the four-row kernel's vector loads are legal here
+  int ww = 1;
+  for (int l = 0; l < ct.L; ++l)
+    for (int k = 0; k < kCrtWords; ++k)
+      if (ct.w[l][k] && k + 1 > ww) ww = k + 1;
+  const bool s_padded = (const void*)s == (const void*)(workspace_ptr() + g.off_s);  // the workspace copy has Mp entries
+  const bool fast = !x_out && (res_ld % 4 == 0) && (res_stride % 4 == 0) && ((reinterpret_cast<uintptr_t>(res) & 3) == 0) &&
+                    ((reinterpret_cast<uintptr_t>(s) & 15) == 0) && (g.M % 4 == 0 || s_padded);
+  if (fast) {
+    dim3 grid((unsigned)((g.M + 1023) / 1024), (unsigned)(g.N < 65535 ? g.N : 65535));
+#define OZK_CRT4(WW, NW) crt4_kernel<WW, NW, false><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc)
+    if (ct.words <= 5 && ww <= 4 && ct.p_bits >= 101 && ct.p_bits <= 126)
+      crt4_kernel<4, 5, true><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc);
+    else if (ct.words == 5 && ww <= 4) OZK_CRT4(4, 5);
+    else if (ct.words <= 2) OZK_CRT4(2, 2);
+    else if (ct.words == 3) OZK_CRT4(3, 3);
+    else if (ct.words == 4) OZK_CRT4(4, 4);
+    else if (ct.words == 5) OZK_CRT4(5, 5);
+    else OZK_CRT4(6, 6);
+#undef OZK_CRT4
+    return cudaGetLastError();
+  }
   dim3 grid((unsigned)((g.M + 255) / 256), (unsigned)g.N);
   switch (ct.words) {
     case 2: crt_kernel<2><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, C, ldc, x_out); break;

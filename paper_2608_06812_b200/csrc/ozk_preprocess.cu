@@ -1,7 +1,7 @@
 // Preprocessing kernels (Section 4.2 shared-exponent conversion; Section 5.1 residues and
 // two-limb encoding; Section 6.2 fused decomposition with K-contiguous write-out).
 //
-//   build_lut         per modulus, for every residue one limb pair (c0, c1) as two E2M1 codes
+//   build_lut         per modulus, for every x in [0, 2m) one limb pair (c0, c1) as two E2M1 codes
 //   scan_rows/cols    max |.| over the rows of A / the columns of B (exponent scan)
 //   finalize_shifts   s_i = c - 1 - e_i, t_j likewise; flags NaN/Inf
 //   encode_cols       B-side planes: source is already K-contiguous
@@ -18,32 +18,34 @@ namespace {
 __device__ __constant__ int8_t kDoubledE2M1[8] = {0, 1, 2, 3, 4, 6, 8, 12};
 
 // ------------------------------------------------------------------------------------
-// Limb-pair table: for residue rho of modulus m, one byte (code(c1) << 4) | code(c0) with
-// c0 + 13 c1 = rho (mod m), both limbs in S, chosen to minimise max(|c0|,|c1|) then |c0|+|c1|.
+// Limb-pair table: for modulus m and every x in [0, 2m) one 16-bit entry holding the E2M1 codes of a
+// limb pair (c0, c1) with c0 + 13 c1 = x (mod m): code(c0) in bits 0..3, code(c1) in bits 8..11.
+// Both limbs are in S and the pair minimises max(|c0|,|c1|), then |c0|+|c1|.  The range 2m lets the
+// encoder skip the last conditional subtraction of its modular reduction.
 // ------------------------------------------------------------------------------------
-__global__ void build_lut_kernel(ModulusTable mt, uint8_t* __restrict__ lut) {
+__global__ void build_lut_kernel(ModulusTable mt, uint16_t* __restrict__ lut) {
   const int l = blockIdx.x;
   const int m = mt.m[l];
-  for (int rho = threadIdx.x; rho < kLutStride; rho += blockDim.x) {
-    int best_key = 1 << 30, best_byte = 0;
-    if (rho < m) {
+  for (int x = threadIdx.x; x < kLutStride; x += blockDim.x) {
+    int best_key = 1 << 30, best = 0;
+    if (x < 2 * m) {
+      const int rho = x % m;
       for (int i1 = 0; i1 < 16; ++i1) {
         for (int i0 = 0; i0 < 16; ++i0) {
-          int c0 = kDoubledE2M1[i0 & 7] * ((i0 & 8) ? -1 : 1);
-          int c1 = kDoubledE2M1[i1 & 7] * ((i1 & 8) ? -1 : 1);
           if ((i0 == 8) || (i1 == 8)) continue;  // skip the negative-zero codes
-          int v = c0 + 13 * c1 - rho;
-          if (v % m != 0) continue;
-          int a0 = abs(c0), a1 = abs(c1);
-          int key = max(a0, a1) * 64 + (a0 + a1);
+          const int c0 = kDoubledE2M1[i0 & 7] * ((i0 & 8) ? -1 : 1);
+          const int c1 = kDoubledE2M1[i1 & 7] * ((i1 & 8) ? -1 : 1);
+          if ((c0 + 13 * c1 - rho) % m != 0) continue;
+          const int a0 = abs(c0), a1 = abs(c1);
+          const int key = max(a0, a1) * 64 + (a0 + a1);
           if (key < best_key) {
             best_key = key;
-            best_byte = (i1 << 4) | i0;
+            best = (i1 << 8) | i0;
           }
         }
       }
     }
-    lut[l * kLutStride + rho] = (uint8_t)best_byte;
+    lut[l * kLutStride + x] = (uint16_t)best;
   }
 }
 
@@ -135,7 +137,7 @@ __device__ __forceinline__ unsigned long long to_integer_magnitude(double x, int
 // Eight consecutive-k integers of one plane row, split into 18-bit pieces, with sign masks.
 struct Piece8 {
   uint32_t x0[8], x1[8], x2[8];
-  uint32_t sgn[8];  // 0x88 for negative values: flips the sign bit of both E2M1 codes
+  uint32_t sgn[8];  // 0x0808 for negative values: flips the sign bit of both E2M1 codes of a table entry
 };
 
 __device__ __forceinline__ void split8(const unsigned long long (&mag)[8], const bool (&neg)[8], Piece8& p) {
@@ -144,26 +146,33 @@ __device__ __forceinline__ void split8(const unsigned long long (&mag)[8], const
     p.x0[e] = (uint32_t)(mag[e] & 0x3FFFFull);
     p.x1[e] = (uint32_t)((mag[e] >> 18) & 0x3FFFFull);
     p.x2[e] = (uint32_t)(mag[e] >> 36);
-    p.sgn[e] = neg[e] ? 0x88u : 0u;
+    p.sgn[e] = neg[e] ? 0x0808u : 0u;
   }
 }
 
 // Residues of the eight values mod m_l and their limb codes packed as 8 nibbles per limb.
-// |a| = x2 2^36 + x1 2^18 + x0  =>  t = x2 (2^36 mod m) + x1 (2^18 mod m) + x0 < 2^27, then one
-// multiply-high reduction; limbs(-rho) = -limbs(rho) because S is symmetric.
+// |a| = x2 2^36 + x1 2^18 + x0  =>  t = x2 (2^36 mod m) + x1 (2^18 mod m) + x0 < 2^27; one multiply-high
+// gives x = t - floor'(t/m) m in [0, 2m), which indexes the table directly; limbs(-rho) = -limbs(rho)
+// because S is symmetric.  Two neighbouring k share a byte: entry(even k) | entry(odd k) << 4 has the
+// byte of limb 0 in bits 0..7 and the byte of limb 1 in bits 8..15.
 __device__ __forceinline__ void encode8(const Piece8& p, uint32_t m, uint32_t recip, uint32_t pow18, uint32_t pow36,
-                                        const uint8_t* __restrict__ lut_l, uint32_t& w0, uint32_t& w1) {
-  w0 = 0;
-  w1 = 0;
+                                        const uint16_t* __restrict__ lut_l, uint32_t& w0, uint32_t& w1) {
+  uint32_t pair[4];
 #pragma unroll
-  for (int e = 0; e < 8; ++e) {
-    const uint32_t t = p.x2[e] * pow36 + p.x1[e] * pow18 + p.x0[e];
-    uint32_t r = t - __umulhi(t, recip) * m;
-    r = min(r, r - m);  // r in [0, 2m): the wrapped difference is larger unless r >= m
-    const uint32_t b = (uint32_t)lut_l[r] ^ p.sgn[e];
-    w0 |= (b & 0xFu) << (4 * e);
-    w1 |= (b >> 4) << (4 * e);
+  for (int h = 0; h < 4; ++h) {
+    uint32_t v[2];
+#pragma unroll
+    for (int o = 0; o < 2; ++o) {
+      const int e = 2 * h + o;
+      const uint32_t t = p.x2[e] * pow36 + p.x1[e] * pow18 + p.x0[e];
+      const uint32_t x = t - __umulhi(t, recip) * m;
+      v[o] = (uint32_t)lut_l[x] ^ p.sgn[e];
+    }
+    pair[h] = v[0] | (v[1] << 4);
   }
+  const uint32_t t0 = pair[0] | (pair[1] << 16), t1 = pair[2] | (pair[3] << 16);
+  w0 = __byte_perm(t0, t1, 0x6420);
+  w1 = __byte_perm(t0, t1, 0x7531);
 }
 
 // ------------------------------------------------------------------------------------
@@ -171,14 +180,19 @@ __device__ __forceinline__ void encode8(const Piece8& p, uint32_t m, uint32_t re
 // Block = 256 threads = 2048 consecutive k of one column; thread = 8 consecutive k.
 // ------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) encode_cols_kernel(const double* __restrict__ B, int64_t ldb, int64_t N, int64_t K,
-                                                          int64_t Kp, ModulusTable mt, const uint8_t* __restrict__ lut,
+                                                          int64_t Kp, ModulusTable mt, const uint16_t* __restrict__ lut,
                                                           const int32_t* __restrict__ shifts, uint8_t* __restrict__ planes,
-                                                          size_t plane_bytes, int64_t* __restrict__ int_out) {
-  extern __shared__ uint8_t smem[];
-  for (int i = threadIdx.x; i < mt.L * kLutStride; i += blockDim.x) smem[i] = lut[i];
+                                                          size_t plane_bytes, int64_t* __restrict__ int_out, int reps) {
+  extern __shared__ __align__(16) uint16_t lut_s[];
+  {  // the table is copied once per block and reused for `reps` chunks of 2048 k
+    const uint4* src = reinterpret_cast<const uint4*>(lut);
+    uint4* dst = reinterpret_cast<uint4*>(lut_s);
+    for (int i = threadIdx.x; i < mt.L * kLutStride / 8; i += blockDim.x) dst[i] = src[i];
+  }
   __syncthreads();
   const int64_t j = blockIdx.x;
-  const int64_t k = ((int64_t)blockIdx.y * blockDim.x + threadIdx.x) * 8;
+  for (int rep = 0; rep < reps; ++rep) {
+  const int64_t k = (((int64_t)blockIdx.y * reps + rep) * blockDim.x + threadIdx.x) * 8;
   if (k >= Kp) return;
   unsigned long long mag[8];
   bool neg[8];
@@ -211,9 +225,10 @@ __global__ void __launch_bounds__(256) encode_cols_kernel(const double* __restri
   uint8_t* dst = planes + (size_t)j * (size_t)(Kp / 2) + (size_t)(k / 2);
   for (int l = 0; l < mt.L; ++l) {
     uint32_t w0, w1;
-    encode8(p, (uint32_t)mt.m[l], mt.recip[l], mt.pow18[l], mt.pow36[l], smem + l * kLutStride, w0, w1);
+    encode8(p, (uint32_t)mt.m[l], mt.recip[l], mt.pow18[l], mt.pow36[l], lut_s + l * kLutStride, w0, w1);
     *reinterpret_cast<uint32_t*>(dst + (size_t)(2 * l) * plane_bytes) = w0;
     *reinterpret_cast<uint32_t*>(dst + (size_t)(2 * l + 1) * plane_bytes) = w1;
+  }
   }
 }
 
@@ -228,18 +243,25 @@ constexpr int kRowTileK = 64;
 constexpr int kStageStride = 9;  // words per staged row (8 used): odd stride avoids bank conflicts
 
 __global__ void __launch_bounds__(256) encode_rows_kernel(const double* __restrict__ A, int64_t lda, int64_t M, int64_t K,
-                                                          int64_t Kp, ModulusTable mt, const uint8_t* __restrict__ lut,
+                                                          int64_t Kp, ModulusTable mt, const uint16_t* __restrict__ lut,
                                                           const int32_t* __restrict__ shifts, uint8_t* __restrict__ planes,
-                                                          size_t plane_bytes, int64_t* __restrict__ int_out) {
+                                                          size_t plane_bytes, int64_t* __restrict__ int_out, int reps) {
   extern __shared__ __align__(16) uint8_t smem[];
-  uint8_t* lut_s = smem;                                                        // L * kLutStride bytes
-  const int lut_bytes = (mt.L * kLutStride + 15) & ~15;
+  uint16_t* lut_s = reinterpret_cast<uint16_t*>(smem);                          // L * kLutStride entries
+  const int lut_bytes = (mt.L * kLutStride * (int)sizeof(uint16_t) + 15) & ~15;
   double* in_s = reinterpret_cast<double*>(smem + lut_bytes);                    // [64][32] doubles
   uint32_t* out_s = reinterpret_cast<uint32_t*>(smem + lut_bytes);               // [2L][32][9] words, reuses in_s
   const int t = threadIdx.x;
   const int64_t i0 = (int64_t)blockIdx.x * kRowTile;
-  const int64_t k0 = (int64_t)blockIdx.y * kRowTileK;
-  for (int i = t; i < mt.L * kLutStride; i += blockDim.x) lut_s[i] = lut[i];
+  {  // the table is copied once per block and reused for `reps` tiles along k
+    const uint4* src = reinterpret_cast<const uint4*>(lut);
+    uint4* dst = reinterpret_cast<uint4*>(lut_s);
+    for (int i = t; i < mt.L * kLutStride / 8; i += blockDim.x) dst[i] = src[i];
+  }
+  for (int rep = 0; rep < reps; ++rep) {
+  const int64_t k0 = ((int64_t)blockIdx.y * reps + rep) * kRowTileK;
+  if (k0 >= Kp) break;  // uniform over the block
+  if (rep) __syncthreads();  // the previous tile's staged output has been written out
   {
     const int ti = t & 31, tk = t >> 5;
     const int64_t i = i0 + ti;
@@ -280,6 +302,7 @@ __global__ void __launch_bounds__(256) encode_rows_kernel(const double* __restri
   uint8_t* dst = planes + (size_t)(i0 + row) * (size_t)(Kp / 2) + (size_t)(k0 / 2) + 4 * word;
   for (int pl = 0; pl < 2 * mt.L; ++pl)
     *reinterpret_cast<uint32_t*>(dst + (size_t)pl * plane_bytes) = out_s[(pl * kRowTile + row) * kStageStride + word];
+  }
 }
 
 // Decodes one limb plane into doubled-E2M1 integers, out[r + k*rows] (test support).
@@ -297,7 +320,7 @@ __global__ void decode_plane_kernel(const uint8_t* __restrict__ plane, int64_t r
 }  // namespace
 
 cudaError_t launch_build_lut(const ModulusTable& mt, uint8_t* lut, cudaStream_t st) {
-  build_lut_kernel<<<mt.L, 192, 0, st>>>(mt, lut);
+  build_lut_kernel<<<mt.L, 384, 0, st>>>(mt, reinterpret_cast<uint16_t*>(lut));
   return cudaGetLastError();
 }
 
@@ -325,23 +348,25 @@ cudaError_t launch_scan_and_shifts(const Geometry& g, const double* A, int64_t l
 
 cudaError_t launch_encode(const Geometry& g, const ModulusTable& mt, const double* A, int64_t lda, const double* B,
                           int64_t ldb, uint8_t* ws, int64_t* At_out, int64_t* Bt_out, cudaStream_t st) {
-  const uint8_t* lut = ws + g.off_lut;
-  const int lut_bytes = (mt.L * kLutStride + 15) & ~15;
+  const uint16_t* lut = reinterpret_cast<const uint16_t*>(ws + g.off_lut);
+  const int lut_bytes = (mt.L * kLutStride * (int)sizeof(uint16_t) + 15) & ~15;
   {
     const size_t stage = (size_t)2 * mt.L * kRowTile * kStageStride * sizeof(uint32_t);
     const size_t in_bytes = (size_t)kRowTileK * kRowTile * sizeof(double);
     const size_t smem = lut_bytes + (stage > in_bytes ? stage : in_bytes);
     cudaError_t e = cudaFuncSetAttribute(encode_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    dim3 grid((unsigned)(g.Mp / kRowTile), (unsigned)(g.Kp / kRowTileK));
+    const int reps = 4;
+    dim3 grid((unsigned)(g.Mp / kRowTile), (unsigned)((g.Kp / kRowTileK + reps - 1) / reps));
     encode_rows_kernel<<<grid, 256, smem, st>>>(A, lda, g.M, g.K, g.Kp, mt, lut, reinterpret_cast<const int32_t*>(ws + g.off_s),
-                                                ws + g.off_planes_a, g.plane_bytes_a, At_out);
+                                                ws + g.off_planes_a, g.plane_bytes_a, At_out, reps);
   }
   {
-    dim3 grid((unsigned)g.Np, (unsigned)((g.Kp + 2047) / 2048));
+    const int reps = 4;
+    dim3 grid((unsigned)g.Np, (unsigned)(((g.Kp + 2047) / 2048 + reps - 1) / reps));
     encode_cols_kernel<<<grid, 256, lut_bytes, st>>>(B, ldb, g.N, g.K, g.Kp, mt, lut,
                                                     reinterpret_cast<const int32_t*>(ws + g.off_t), ws + g.off_planes_b,
-                                                    g.plane_bytes_b, Bt_out);
+                                                    g.plane_bytes_b, Bt_out, reps);
   }
   return cudaGetLastError();
 }

@@ -184,6 +184,8 @@ bool host_build_crt_table(int L, CrtTable* t) {
   Big h = big_div_small(P, 2, nullptr);
   for (int i = 0; i < kCrtWords; ++i) t->halfP[i] = h.w[i];
   t->inv_P = 1.0 / big_to_double(P);
+  t->q_scale = ldexp(t->inv_P, 96) * (1.0 - ldexp(1.0, -30));
+  t->p_bits = big_bits(P);
   return true;
 }
 

@@ -139,6 +139,10 @@ def test_single_rounding_against_bit_level_rne():
     assert ozaki2.round_scaled_to_double(3, 1075) == 2 * 2.0 ** -1074
     assert ozaki2.round_scaled_to_double(1, 1075) == 0.0
     assert ozaki2.round_scaled_to_double(-5, 1) == -2.5
+    # overflow follows IEEE 754 round-to-nearest: the largest finite double, then infinity
+    assert ozaki2.round_scaled_to_double(2 ** 53 - 1, -(1023 - 52)) == float.fromhex("0x1.fffffffffffffp+1023")
+    assert ozaki2.round_scaled_to_double(2 ** 54 - 1, -(1023 - 53)) == math.inf
+    assert ozaki2.round_scaled_to_double(-3, -1100) == -math.inf
 
 
 # ---- fl(AB) --------------------------------------------------------------------------------
