@@ -117,6 +117,19 @@ ozk_status ozk_igemm_i8(int64_t M, int64_t N, int64_t K,
                         const int8_t* B, int64_t ldb,
                         int32_t* C, int64_t ldc, void* stream);
 
+/* Emulated DGEMM by Ozaki scheme I on the same limbs (Section 4; Fig. 2; Eq. 1; Lemma 2): the
+ * integer-converted inputs (c = 53 bits, Section 4.2) are decomposed into p = q = 15 greedy base-13
+ * E2M1 limbs, the limb products are aggregated along the anti-diagonals i + j = g, weighted by 13^g
+ * in multiword integers, scaled back and rounded once.  The result equals ozk_dgemm with 19 moduli
+ * bit for bit (both are the exact product of the same converted integers rounded once, Section 7.1).
+ * Arguments and layout as ozk_dgemm.  K <= 87381 (three products of magnitude <= 64 share an FP32
+ * accumulator).  Workspace: 15 + 16 limb planes and 20 int64 block values per element of C. */
+size_t ozk_dgemm_oz1_workspace_bytes(int64_t M, int64_t N, int64_t K);
+ozk_status ozk_dgemm_oz1(int64_t M, int64_t N, int64_t K,
+                         const double* A, int64_t lda,
+                         const double* B, int64_t ldb,
+                         double* C, int64_t ldc, void* stream);
+
 /* ---------------------------------------------------------------------------------------
  * Staged entry points: the same kernels one stage at a time, used by the parity tests.
  * They use the registered workspace exactly as ozk_dgemm does.

@@ -37,6 +37,8 @@ SIGNATURES = {
     "ozk_get_async_status": (c_int, [c_void_p]),
     "ozk_dgemm": (c_int, [c_int64, c_int64, c_int64, c_void_p, c_int64, c_void_p, c_int64, c_void_p, c_int64, c_int, c_void_p]),
     "ozk_igemm_i8": (c_int, [c_int64, c_int64, c_int64, c_void_p, c_int64, c_void_p, c_int64, c_void_p, c_int64, c_void_p]),
+    "ozk_dgemm_oz1_workspace_bytes": (c_size_t, [c_int64, c_int64, c_int64]),
+    "ozk_dgemm_oz1": (c_int, [c_int64, c_int64, c_int64, c_void_p, c_int64, c_void_p, c_int64, c_void_p, c_int64, c_void_p]),
     "ozk_stage_preprocess": (c_int, [c_int64, c_int64, c_int64, c_void_p, c_int64, c_void_p, c_int64, c_int,
                                      c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "ozk_stage_read_planes": (c_int, [c_char, c_int64, c_int64, c_int64, c_int, c_int, c_int, c_void_p, c_void_p]),
@@ -164,3 +166,11 @@ def ozk_row_shifts_noalloc(M, K, A, lda, num_moduli, s_out, stream=0) -> int:
     """Row shifts of A without any workspace: the scratch is a fixed 512 KiB array inside the
     library (at most 65536 rows), for callers that may not allocate device memory."""
     return lib().ozk_row_shifts_noalloc(M, K, A, lda, num_moduli, s_out, stream)
+
+
+def ozk_dgemm_oz1_workspace_bytes(M: int, N: int, K: int) -> int:
+    return lib().ozk_dgemm_oz1_workspace_bytes(M, N, K)
+
+
+def ozk_dgemm_oz1(M, N, K, A, lda, B, ldb, C, ldc, stream=0) -> int:
+    return lib().ozk_dgemm_oz1(M, N, K, A, lda, B, ldb, C, ldc, stream)

@@ -40,6 +40,7 @@ struct GemmCore {
   int kblocks;  // Kp / 256
   int group;    // rasterisation: this many column tiles share one sweep over the row tiles
   int skip_top_first;  // plane group 0 needs no p_{NP-1} q_{NQ-1} product (13^2 = 0 mod 169)
+  int q_groups;        // 0: both operands use plane group l; n > 0: row side uses l / n, column side l % n
   StatusBlock* status;
   uint32_t scale_word;  // four copies of the UE8M0 scale byte
 };
@@ -205,6 +206,57 @@ struct Int32Epilogue {
   }
 };
 
+
+// ------------------------------------------------------------------------------------
+// Epilogue of the scheme-I passes (Eq. 1): one pass multiplies NP = 4 row-side limbs with NQ = 3
+// column-side limbs; its six accumulators G_0..G_5 (anti-diagonals of the 4 x 3 block) are combined
+// as V = sum_g 13^g G_g in int64 (|G_g| <= 3 * 64 * K, 13^5 < 2^19) and stored per pass; a separate
+// reduction kernel adds the passes with their powers of 13.  4 warps, 16 columns at a time.
+// ------------------------------------------------------------------------------------
+struct Int64BlockEpilogue {
+  static constexpr int kWarps = 4;
+  struct Params {
+    long long* out;      // [passes][Np][ld] int64
+    int64_t ld;          // rows per column of a pass (multiple of the tile width)
+    size_t pass_stride;  // Np * ld
+  };
+  template <int W>
+  __device__ static __forceinline__ void run(const Params& ep, const GemmCore&, uint32_t tmem, int epi_warp, int lane, int l,
+                                             int tp, int tq, uint32_t release_bar) {
+    const uint32_t quad = (uint32_t)((epi_warp + 2) & 3);  // TMEM lane quadrant = warp index mod 4
+    const uint32_t base = tmem + ((quad * 32u) << 16);
+    const int64_t j = (int64_t)tp * kTileRows + quad * 32 + lane;
+    long long* col = ep.out + (size_t)l * ep.pass_stride + (size_t)j * (size_t)ep.ld + (size_t)tq * W;
+#pragma unroll 1
+    for (int c = 0; c < W / 16; ++c) {
+      uint32_t g0[16], g1[16], g2[16], g3[16], g4[16], g5[16];
+      tmem_ld_32x16(base + 0 * W + c * 16, g0);
+      tmem_ld_32x16(base + 1 * W + c * 16, g1);
+      tmem_ld_32x16(base + 2 * W + c * 16, g2);
+      tmem_ld_32x16(base + 3 * W + c * 16, g3);
+      tmem_ld_32x16(base + 4 * W + c * 16, g4);
+      tmem_ld_32x16(base + 5 * W + c * 16, g5);
+      tmem_wait_ld();
+      longlong2* dst = reinterpret_cast<longlong2*>(col + c * 16);
+#pragma unroll
+      for (int e = 0; e < 16; e += 2) {
+        long long v[2];
+#pragma unroll
+        for (int o = 0; o < 2; ++o) {
+          const long long a0 = __float2int_rn(__uint_as_float(g0[e + o])), a1 = __float2int_rn(__uint_as_float(g1[e + o]));
+          const long long a2 = __float2int_rn(__uint_as_float(g2[e + o])), a3 = __float2int_rn(__uint_as_float(g3[e + o]));
+          const long long a4 = __float2int_rn(__uint_as_float(g4[e + o])), a5 = __float2int_rn(__uint_as_float(g5[e + o]));
+          v[o] = a0 + 13ll * a1 + 169ll * a2 + 2197ll * a3 + 28561ll * a4 + 371293ll * a5;
+        }
+        dst[e / 2] = make_longlong2(v[0], v[1]);
+      }
+    }
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(release_bar);
+  }
+};
+
 template <int NP, int NQ, int W, int STAGES, class Epi>
 __global__ void __launch_bounds__(64 + 32 * Epi::kWarps, 1)
 limb_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_q,
@@ -266,6 +318,7 @@ limb_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constan
       for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
         int l, tp, tq;
         decode_item(p, item, l, tp, tq);
+        const int lp = p.q_groups ? l / p.q_groups : l, lq = p.q_groups ? l % p.q_groups : l;
         for (int kb = 0; kb < p.kblocks; ++kb) {
           if (!wait_bounded(smem_u32(&sh->empty[stage]), phase ^ 1u, sh, p.status, 0x000 + stage)) {
             ok = false;
@@ -278,10 +331,10 @@ limb_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constan
           armed_parity[stage] = phase;
           const int x = kb * kTileKBytes;
 #pragma unroll
-          for (int i = 0; i < NP; ++i) tma_load_3d(dst + i * kPTileBytes, &map_p, bar, x, tp * kTileRows, NP * l + i);
+          for (int i = 0; i < NP; ++i) tma_load_3d(dst + i * kPTileBytes, &map_p, bar, x, tp * kTileRows, NP * lp + i);
 #pragma unroll
           for (int jq = 0; jq < NQ; ++jq)
-            tma_load_3d(dst + NP * kPTileBytes + jq * kQTileBytes, &map_q, bar, x, tq * W, NQ * l + jq);
+            tma_load_3d(dst + NP * kPTileBytes + jq * kQTileBytes, &map_q, bar, x, tq * W, NQ * lq + jq);
           if (++stage == STAGES) stage = 0, phase ^= 1u;
         }
       }
@@ -555,6 +608,7 @@ ozk_status gemm_residues(const Geometry& g, const ModulusTable& mt, uint8_t* ws,
   core.kblocks = (int)(g.Kp / kTileKNibbles);
   core.group = 16;
   core.skip_top_first = (mt.m[0] == 169) ? 1 : 0;  // 13^2 a1 b1 vanishes mod 169 (Section 5.1)
+  core.q_groups = 0;
   core.status = reinterpret_cast<StatusBlock*>(ws + g.off_status);
   core.scale_word = 0x80808080u;  // UE8M0 byte 0x80 = 2: both operands doubled, accumulators hold integers
   ResidueEpilogue::Params ep;
@@ -583,6 +637,7 @@ ozk_status gemm_int8(const uint8_t* planes_a, const uint8_t* planes_b, int64_t M
   core.kblocks = (int)(Kp / kTileKNibbles);
   core.group = 16;
   core.skip_top_first = 0;
+  core.q_groups = 0;
   core.status = status;
   core.scale_word = 0x80808080u;
   Int32Epilogue::Params ep;
@@ -591,6 +646,31 @@ ozk_status gemm_int8(const uint8_t* planes_a, const uint8_t* planes_b, int64_t M
   ep.M = M;
   ep.N = N;
   return launch_limb_gemm<3, 3, W, 2, Int32Epilogue>(map_p, map_q, core, ep, st);
+}
+
+// Scheme-I passes: 16 row-side limb planes (the 16th all zero) in 4 groups of 4, 15 column-side planes in
+// 5 groups of 3; pass l = 5 * (row group) + (column group) writes its int64 block value to out[l].
+ozk_status gemm_oz1_passes(const uint8_t* planes_a, const uint8_t* planes_b, int64_t Mp, int64_t Np, int64_t Kp, int64_t M,
+                           long long* out, int64_t out_ld, StatusBlock* status, cudaStream_t st) {
+  constexpr int W = 80;
+  CUtensorMap map_p, map_q;
+  if (!make_plane_map(&map_p, planes_b, Kp / 2, Np, 16, (size_t)Np * (size_t)(Kp / 2), kTileRows)) return OZK_ERR_CUDA;
+  if (!make_plane_map(&map_q, planes_a, Kp / 2, Mp, 15, (size_t)Mp * (size_t)(Kp / 2), W)) return OZK_ERR_CUDA;
+  GemmCore core;
+  core.L = 20;
+  core.tiles_p = (int)(Np / kTileRows);
+  core.tiles_q = (int)((M + W - 1) / W);
+  core.kblocks = (int)(Kp / kTileKNibbles);
+  core.group = 16;
+  core.skip_top_first = 0;
+  core.q_groups = 5;
+  core.status = status;
+  core.scale_word = 0x80808080u;
+  Int64BlockEpilogue::Params ep;
+  ep.out = out;
+  ep.ld = out_ld;
+  ep.pass_stride = (size_t)Np * (size_t)out_ld;
+  return launch_limb_gemm<4, 3, W, 2, Int64BlockEpilogue>(map_p, map_q, core, ep, st);
 }
 
 ozk_status gemm_probe(const uint8_t* P, const uint8_t* Q, int64_t K, int scale_byte, float* D, uint8_t* ws, cudaStream_t st) {

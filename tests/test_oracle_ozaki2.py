@@ -232,3 +232,20 @@ def test_config1_law_error_levels():
     errs = {L: exact.normwise_error(ozaki2.dgemm(A, B, L).C, A, B, against_rounded=True) for L in (14, 17, 19)}
     assert errs[19] <= 1e-15 and errs[17] <= 1e-15
     assert errs[14] > errs[17] >= errs[19] * 0.999
+
+
+# ---- scheme I (Section 4) ---------------------------------------------------------------------
+def test_scheme1_equals_integer_product_and_scheme2_bit_for_bit():
+    """Section 7.1: both schemes compute the exact product of the same converted integers and round
+    once, so their outputs agree bit for bit; c = floor(log2 min(X_15, 2^53)) = 53."""
+    from oracle import ozaki1
+    assert ozaki1.capacity_bits_oz1(15) == 53 and ozaki1.capacity_bits_oz1(14) == 50
+    rng = np.random.default_rng(21)
+    A = (rng.random((9, 70)) - 0.5) * np.exp(2 * rng.standard_normal((9, 70)))
+    B = (rng.random((70, 7)) - 0.5) * np.exp(2 * rng.standard_normal((70, 7)))
+    A[3, :] = 0.0
+    C1, X1, At, Bt = ozaki1.dgemm(A, B)
+    ref = np.dot(At.astype(object), Bt.astype(object))
+    assert all(int(X1[idx]) == int(ref[idx]) for idx in np.ndindex(*X1.shape))
+    C2 = ozaki2.dgemm(A, B, 19).C
+    assert np.array_equal(C1.view(np.uint64), C2.view(np.uint64))
