@@ -44,6 +44,8 @@ def parse_args():
     ap.add_argument("--moduli", type=int, default=19)
     ap.add_argument("--phi", type=float, default=1.0)
     ap.add_argument("--impl", default="ozk", choices=["ozk", "reference"])
+    ap.add_argument("--scheme", default="oz2", choices=["oz2", "oz1"],
+                    help="oz2 = Ozaki scheme II (the headline path); oz1 = Ozaki scheme I, 15 x 15 limbs")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-fp64-context", action="store_true")
@@ -207,13 +209,17 @@ def run_ozk(args, rank: int, local_rank: int, world: int) -> None:
     hC = torch.empty((N, M), dtype=torch.float64).pin_memory()
     dA, dB = hA.to(dev), hB.to(dev)
     dC = torch.empty((N, M), dtype=torch.float64, device=dev)
-    ws_bytes = ozk.ozk_dgemm_workspace_bytes(M, N, K, L)
+    oz1 = args.scheme == "oz1"
+    ws_bytes = ozk.ozk_dgemm_oz1_workspace_bytes(M, N, K) if oz1 else ozk.ozk_dgemm_workspace_bytes(M, N, K, L)
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
     ozk.check(ozk.ozk_set_workspace(ws.data_ptr(), ws.numel()), "ozk_set_workspace")
-    ozk.check(ozk.ozk_stage_timing_enable(True), "ozk_stage_timing_enable")
+    ozk.check(ozk.ozk_stage_timing_enable(not oz1), "ozk_stage_timing_enable")
 
     def step():
-        ozk.check(ozk.ozk_dgemm(M, N, K, dA.data_ptr(), M, dB.data_ptr(), K, dC.data_ptr(), M, L, stream), "ozk_dgemm")
+        if oz1:
+            ozk.check(ozk.ozk_dgemm_oz1(M, N, K, dA.data_ptr(), M, dB.data_ptr(), K, dC.data_ptr(), M, stream), "ozk_dgemm_oz1")
+        else:
+            ozk.check(ozk.ozk_dgemm(M, N, K, dA.data_ptr(), M, dB.data_ptr(), K, dC.data_ptr(), M, L, stream), "ozk_dgemm")
 
     def barrier():
         torch.cuda.synchronize()
@@ -238,7 +244,8 @@ def run_ozk(args, rank: int, local_rank: int, world: int) -> None:
         ev[i + 1].record()
         # per-stage CUDA events recorded by the library on this stream, read live inside the timed
         # region (the read waits for this step's last event; a step is >100 ms, the wait adds microseconds)
-        stage_acc += np.array(ozk.ozk_stage_timing_read())
+        if not oz1:
+            stage_acc += np.array(ozk.ozk_stage_timing_read())
     barrier()
     total_ms = ev[0].elapsed_time(ev[args.steps])
     clocks = sampler.stop() if rank == 0 else None
@@ -275,8 +282,19 @@ def run_ozk(args, rank: int, local_rank: int, world: int) -> None:
     if rank != 0:
         return
     peaks = measured_peaks()
+    if oz1:
+        line = {"metric": METRIC.replace("scheme II", "scheme I (15 x 15 limbs)"), "value": value, "unit": UNIT, "n_gpus": world,
+                "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_max, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "fp4_e2m1 (fp32 accumulate, multiword integer reduction)",
+                "data": "synthetic", "config": {"workload": workload_name(n, L, args.phi).replace(f"Ozaki-II {L} moduli", "Ozaki-I p=q=15"),
+                                                "l2": "inputs larger than L2" if M * K * 8 > (126 << 20) else "inputs fit L2"},
+                "clocks": clocks, "e2e": e2e, "gpu_launches": 8 * args.steps,
+                "fp4_tflops_executed_240_products": 2.0 * 240 * M * N * K / (ms_max * 1e-3) / 1e12, "per_step_ms": per_step}
+        print(json.dumps(line), flush=True)
+        return
     gemm_ms = float(stage_acc[1])
-    fp4_flops_exec = 2.0 * 4 * L * M * N * K             # 4 limb products per modulus are executed
+    executed = 4 * L - 1 if ozk.ozk_get_moduli(L)[0] == 169 else 4 * L   # the 13^2 term of modulus 169 is skipped
+    fp4_flops_exec = 2.0 * executed * M * N * K
     fp4_flops_req = 2.0 * (4 * L - 1) * M * N * K        # the 13^2 term of modulus 169 is not required
     achieved = fp4_flops_exec / (gemm_ms * 1e-3) / 1e12
     peak = peaks["bf16_sustained"] * FP4_PER_BF16

@@ -1,5 +1,6 @@
 // C-ABI entry points of the ozk library: argument checks, workspace layout, stage sequencing.
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include "ozk_common.cuh"
@@ -160,6 +161,8 @@ ozk_status ozk_get_async_status(void* stream) {
   if (cudaStreamSynchronize(st) != cudaSuccess) return OZK_ERR_CUDA;
   StatusBlock sb;
   if (cudaMemcpy(&sb, g_ws.ptr, sizeof sb, cudaMemcpyDeviceToHost) != cudaSuccess) return OZK_ERR_CUDA;
+  if (getenv("OZK_DEBUG_TIMING"))
+    fprintf(stderr, "ozk dbg: mma thread total %d, wait tmem_empty %d, wait full %d (x256 clk)\n", sb.pad[0], sb.pad[1], sb.pad[2]);
   if (sb.code != 0) {
     if (sb.code == OZK_ERR_DEVICE_TIMEOUT) fprintf(stderr, "ozk: bounded wait expired at 0x%x\n", sb.where);
     cudaMemset(g_ws.ptr, 0, sizeof(StatusBlock));

@@ -19,6 +19,9 @@
 //
 // Warp roles: 0 = TMA producer, 1 = MMA issuer (owns the TMEM allocation), 2.. = epilogue.
 // Every wait is bounded; on expiry the CTA records OZK_ERR_DEVICE_TIMEOUT, drains and returns.
+#include <stdio.h>
+#include <stdlib.h>
+
 #include "ozk_common.cuh"
 #include "ozk_ptx.cuh"
 
@@ -41,6 +44,7 @@ struct GemmCore {
   int group;    // rasterisation: this many column tiles share one sweep over the row tiles
   int skip_top_first;  // plane group 0 needs no p_{NP-1} q_{NQ-1} product (13^2 = 0 mod 169)
   int q_groups;        // 0: both operands use plane group l; n > 0: row side uses l / n, column side l % n
+  int fast_combine;    // K <= 17476: D1 + 13 D2 stays below 2^24 and may be formed in FP32 before the release
   StatusBlock* status;
   uint32_t scale_word;  // four copies of the UE8M0 scale byte
 };
@@ -86,21 +90,99 @@ __device__ __forceinline__ void decode_item(const GemmCore& p, int item, int& l,
   tp = g * p.group + (rem - tq * gsize);
 }
 
+
+// Drains the three accumulators of 64 columns (lanes of this warp's quadrant) and hands tensor memory
+// back as early as possible.  With `fast` the only work before the release is one exact FP32
+// multiply-add per element, u = D1 + 13 D2 (|u| <= 128 K + 13 * 64 K < 2^24 for K <= 17476); the
+// conversions, the rest of the weighted sum and the reduction mod m run after the release and
+// overlap the next tile's main loop.  Returns t = D0 + 13 D1 + 169 D2 + offset (non-negative).
+template <bool kFast, bool kZeroTop>
+__device__ __forceinline__ void drain_and_release(uint32_t base, int W, bool top, uint32_t offset, uint32_t release_bar,
+                                                  bool release_remote, int lane, uint32_t (&t)[64]) {
+  uint32_t u[kFast ? 64 : 1];
+#pragma unroll
+  for (int c = 0; c < 2; ++c) {
+    uint32_t d1[32], d2[32];
+    tmem_ld_32x32(base + 1 * W + c * 32, d1);
+    if (top) tmem_ld_32x32(base + 2 * W + c * 32, d2);
+    if constexpr (kFast) {
+      tmem_wait_ld();
+#pragma unroll
+      for (int e = 0; e < 32; ++e)
+        u[c * 32 + e] = top ? __float_as_uint(fmaf(__uint_as_float(d2[e]), 13.0f, __uint_as_float(d1[e]))) : d1[e];
+      uint32_t d0[32];
+      tmem_ld_32x32(base + 0 * W + c * 32, d0);
+      tmem_wait_ld();
+#pragma unroll
+      for (int e = 0; e < 32; ++e) t[c * 32 + e] = d0[e];  // raw FP32 bits until after the release
+    } else {
+      uint32_t d0[32];
+      tmem_ld_32x32(base + 0 * W + c * 32, d0);
+      tmem_wait_ld();
+#pragma unroll
+      for (int e = 0; e < 32; ++e) {
+        const int a0 = __float2int_rn(__uint_as_float(d0[e]));
+        const int a1 = __float2int_rn(__uint_as_float(d1[e]));
+        const int a2 = top ? __float2int_rn(__uint_as_float(d2[e])) : 0;
+        t[c * 32 + e] = (uint32_t)(a0 + 13 * a1 + 169 * a2) + offset;  // non-negative, < 2^32
+      }
+    }
+  }
+  if constexpr (kZeroTop) {
+    tmem_st_32x32_const(base + 2 * W, 0u);
+    tmem_st_32x32_const(base + 2 * W + 32, 0u);
+    tmem_wait_st();
+  }
+  tc_fence_before();
+  __syncwarp();
+  if (lane == 0) {
+    if (release_remote) mbar_arrive_cluster(release_bar); else mbar_arrive(release_bar);
+  }
+  if constexpr (kFast) {
+#pragma unroll
+    for (int e = 0; e < 64; ++e)
+      t[e] = (uint32_t)(__float2int_rn(__uint_as_float(t[e])) + 13 * __float2int_rn(__uint_as_float(u[e]))) + offset;
+  }
+}
+
+// Reduces 64 composed values mod m (one multiply-high each, result in [0, m)) and stores them as bytes.
+__device__ __forceinline__ void reduce_and_store(const uint32_t (&t)[64], uint32_t m, uint32_t recip, uint4* dst) {
+#pragma unroll
+  for (int q4 = 0; q4 < 4; ++q4) {
+    uint32_t w[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      uint32_t word = 0;
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {
+        const uint32_t x = t[q4 * 16 + k * 4 + b];
+        uint32_t r = x - __umulhi(x, recip) * m;  // in [0, 2m)
+        r = min(r, r - m);
+        word |= r << (8 * b);
+      }
+      w[k] = word;
+    }
+    dst[q4] = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+}
+
 // ------------------------------------------------------------------------------------
 // Epilogue of the DGEMM path: r = (D0 + 13 D1 + 169 D2) mod m in [0, m), one byte per element.
 // 8 warps: warp (quadrant q, half h) drains lanes 32q..32q+31, columns 64h..64h+63 of the three
 // accumulators into 64 registers, releases tensor memory, then reduces and stores.
 // ------------------------------------------------------------------------------------
-struct ResidueEpilogue {
-  static constexpr int kWarps = 8;
-  struct Params {
+struct ResidueParams {
     int m[kMaxModuli];
     uint32_t recip[kMaxModuli];   // floor(2^32 / m)
     uint32_t offset[kMaxModuli];  // multiple of m close to 2^31: makes the composed value non-negative
     uint8_t* res;                 // [L][Np][Mp] bytes
     int64_t res_ld;               // Mp
     size_t res_stride;            // Mp * Np
-  };
+};
+template <bool kFast>
+struct ResidueEpilogue {
+  static constexpr int kWarps = 8;
+  using Params = ResidueParams;
   template <int W>
   __device__ static __forceinline__ void run(const Params& ep, const GemmCore& core, uint32_t tmem, int epi_warp, int lane, int l,
                                              int tp, int tq, uint32_t release_bar) {
@@ -111,44 +193,11 @@ struct ResidueEpilogue {
     const uint32_t m = (uint32_t)ep.m[l], recip = ep.recip[l], offset = ep.offset[l];
     const bool top = !(core.skip_top_first && l == 0);
     uint32_t t[64];
-#pragma unroll
-    for (int c = 0; c < 2; ++c) {
-      uint32_t d0[32], d1[32], d2[32];
-      tmem_ld_32x32(base + 0 * W + c * 32, d0);
-      tmem_ld_32x32(base + 1 * W + c * 32, d1);
-      if (top) tmem_ld_32x32(base + 2 * W + c * 32, d2);
-      tmem_wait_ld();
-#pragma unroll
-      for (int e = 0; e < 32; ++e) {
-        const int v0 = __float2int_rn(__uint_as_float(d0[e]));
-        const int v1 = __float2int_rn(__uint_as_float(d1[e]));
-        const int v2 = top ? __float2int_rn(__uint_as_float(d2[e])) : 0;
-        t[c * 32 + e] = (uint32_t)(v0 + 13 * v1 + 169 * v2) + offset;  // non-negative, < 2^32
-      }
-    }
-    tc_fence_before();
-    __syncwarp();
-    if (lane == 0) mbar_arrive(release_bar);  // the accumulators may be overwritten from here on
+    drain_and_release<kFast, false>(base, W, top, offset, release_bar, false, lane, t);
     const int64_t j = (int64_t)tp * kTileRows + quad * 32 + lane;
     uint4* dst = reinterpret_cast<uint4*>(ep.res + (size_t)l * ep.res_stride + (size_t)j * (size_t)ep.res_ld +
                                           (size_t)tq * W + half * 64);
-#pragma unroll
-    for (int q4 = 0; q4 < 4; ++q4) {
-      uint32_t w[4];
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        uint32_t word = 0;
-#pragma unroll
-        for (int b = 0; b < 4; ++b) {
-          const uint32_t x = t[q4 * 16 + k * 4 + b];
-          uint32_t r = x - __umulhi(x, recip) * m;  // in [0, 2m)
-          r = min(r, r - m);
-          word |= r << (8 * b);
-        }
-        w[k] = word;
-      }
-      dst[q4] = make_uint4(w[0], w[1], w[2], w[3]);
-    }
+    reduce_and_store(t, m, recip, dst);
   }
 };
 
@@ -357,17 +406,22 @@ limb_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constan
       constexpr uint32_t kIdescAll = idesc_mxf4(NQ * W);
       constexpr uint32_t kIdescButLast = idesc_mxf4(NQ > 1 ? (NQ - 1) * W : W);
       bool ok = true;
+      long long dbg_t0 = clock64(), dbg_empty = 0, dbg_full = 0;
       for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
         int l, tp, tq;
         decode_item(p, item, l, tp, tq);
         const bool skip_top = p.skip_top_first && l == 0;
+        long long dbg_a = clock64();
         if (!wait_bounded(smem_u32(&sh->tmem_empty), acc_phase ^ 1u, sh, p.status, 0x100)) break;
+        dbg_empty += clock64() - dbg_a;
         tc_fence_after();
         for (int kb = 0; kb < p.kblocks; ++kb) {
+          dbg_a = clock64();
           if (!wait_bounded(smem_u32(&sh->full[stage]), phase, sh, p.status, 0x110 + stage)) {
             ok = false;
             break;
           }
+          dbg_full += clock64() - dbg_a;
           tc_fence_after();
           const uint32_t pbase = smem_u32(tiles + stage * kStageBytes);
           const uint32_t qbase = pbase + NP * kPTileBytes;
@@ -404,6 +458,11 @@ limb_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constan
         mma_commit(smem_u32(&sh->tmem_full));
         acc_phase ^= 1u;
       }
+      if (blockIdx.x == 0) {
+        p.status->pad[0] = (int)((clock64() - dbg_t0) >> 8);
+        p.status->pad[1] = (int)(dbg_empty >> 8);
+        p.status->pad[2] = (int)(dbg_full >> 8);
+      }
       if (sh->abort) {  // wait for the tensor pipe to go idle before TMEM is released
         mma_commit(smem_u32(&sh->drained));
         const uint64_t t0 = global_timer_ns();
@@ -431,6 +490,175 @@ limb_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constan
   if (warp == 1) {
     __syncwarp();
     tmem_dealloc(tmem, kTmemCols);
+  }
+}
+
+
+// ------------------------------------------------------------------------------------
+// DGEMM path on CTA pairs (cta_group::2).  Two CTAs of a cluster (one TPC) work on a 256 x 128
+// output tile: each holds 128 of the 256 TMEM lanes (columns j of C) and loads its own p0, p1 tiles;
+// the 256 stacked column-side rows [q0 ; q1] are split between them, the leader keeps q0 and its
+// peer q1, and the tensor core reads both halves.  Per stage a CTA therefore loads 48 KiB instead
+// of 64 KiB and its shared memory feeds 64 instead of 96 bytes per clock to the MMA.
+// The leader's MMA thread issues for the pair; byte counts of both CTAs' TMA loads arrive on the
+// leader's "full" barrier; commits are multicast to the barriers of both CTAs.
+// Accumulator columns 256..383 are zeroed by the epilogue before a tile starts, so the first
+// K step can run p0 with "overwrite" and p1 with "accumulate" (the cross-term columns 128..255
+// need both).  All four products are executed for every modulus (for m = 169 the 13^2 term
+// cancels in the reduction).
+// ------------------------------------------------------------------------------------
+constexpr int kPairStages = 4;
+constexpr int kPairStageBytes = 3 * kPTileBytes;  // p0, p1 and this CTA's half of [q0 ; q1]
+constexpr int kPairThreads = 64 + 32 * 8;
+
+template <bool kFast>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
+residue_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_q,
+                         const __grid_constant__ GemmCore p, const __grid_constant__ ResidueParams ep) {
+  constexpr int W = 128;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  GemmShared* sh = reinterpret_cast<GemmShared*>(tiles + kPairStages * kPairStageBytes);
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+  const int total_items = p.L * p.tiles_p * p.tiles_q;  // tiles_p counts 256-wide column tiles here
+
+  if (threadIdx.x == 0) {
+    prefetch_tensormap(&map_p);
+    prefetch_tensormap(&map_q);
+    for (int s = 0; s < kPairStages; ++s) {
+      mbar_init(smem_u32(&sh->full[s]), 1);   // used in the leader only
+      mbar_init(smem_u32(&sh->empty[s]), 1);
+    }
+    mbar_init(smem_u32(&sh->tmem_full), 1);
+    mbar_init(smem_u32(&sh->tmem_empty), 16);  // 8 epilogue warps of each CTA; used in the leader only
+    mbar_init(smem_u32(&sh->drained), 1);
+    sh->abort = 0;
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(smem_u32(&sh->tmem_base), kTmemCols);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = sh->tmem_base;
+  if (warp >= 2) {
+    const uint32_t quad = (uint32_t)(warp & 3), half = (uint32_t)((warp - 2) >> 2);
+    const uint32_t lane_base = tmem + ((quad * 32u) << 16);
+    if (half == 0) {  // constant UE8M0 scale bytes
+      tmem_st_32x8_const(lane_base + kScaleCol, p.scale_word);
+      tmem_st_32x8_const(lane_base + kScaleCol + 8, p.scale_word);
+    }
+    tmem_st_32x32_const(lane_base + 2 * W + half * 64, 0u);  // accumulator of the 13^2 term starts at zero
+    tmem_st_32x32_const(lane_base + 2 * W + half * 64 + 32, 0u);
+    tmem_wait_st();
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_arrive();  // the peer's barriers are initialised before anything is sent to them
+  cluster_wait();
+  tc_fence_after();
+
+  if (warp == 0) {
+    // ------------------------------ TMA producer (both CTAs) ------------------------------
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int item = pair; item < total_items && ok; item += npairs) {
+        int l, tp, tq;
+        decode_item(p, item, l, tp, tq);
+        for (int kb = 0; kb < p.kblocks; ++kb) {
+          if (!wait_bounded(smem_u32(&sh->empty[stage]), phase ^ 1u, sh, p.status, 0x300 + stage)) {
+            ok = false;
+            break;
+          }
+          const uint32_t leader_full = map_to_cta(smem_u32(&sh->full[stage]), 0);
+          const uint32_t dst = smem_u32(tiles + stage * kPairStageBytes);
+          if (rank == 0) mbar_arrive_expect_tx(smem_u32(&sh->full[stage]), 2 * kPairStageBytes);
+          const int x = kb * kTileKBytes;
+          const int prow = (2 * tp + (int)rank) * kTileRows;
+          tma_load_3d_pair(dst + 0 * kPTileBytes, &map_p, leader_full, x, prow, 2 * l + 0);
+          tma_load_3d_pair(dst + 1 * kPTileBytes, &map_p, leader_full, x, prow, 2 * l + 1);
+          tma_load_3d_pair(dst + 2 * kPTileBytes, &map_q, leader_full, x, tq * W, 2 * l + (int)rank);
+          if (++stage == kPairStages) stage = 0, phase ^= 1u;
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer (leader only) ------------------------------
+    if (lane == 0 && rank == 0) {
+      int stage = 0;
+      uint32_t phase = 0, acc_phase = 0;
+      const uint32_t sf = tmem + kScaleCol;
+      constexpr uint32_t kIdesc = idesc_mxf4_pair(2 * W);
+      bool ok = true;
+      for (int item = pair; item < total_items && ok; item += npairs) {
+        if (!wait_bounded(smem_u32(&sh->tmem_empty), acc_phase ^ 1u, sh, p.status, 0x400)) break;
+        tc_fence_after();
+        for (int kb = 0; kb < p.kblocks; ++kb) {
+          if (!wait_bounded(smem_u32(&sh->full[stage]), phase, sh, p.status, 0x410 + stage)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t base = smem_u32(tiles + stage * kPairStageBytes);
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks) {
+            const uint64_t q = smem_desc_sw128(base + 2 * kPTileBytes + ks * 32);
+            mma_mxf4_pair(tmem + 0, smem_desc_sw128(base + 0 * kPTileBytes + ks * 32), q, kIdesc, sf, sf,
+                          (kb == 0 && ks == 0) ? 0u : 1u);
+            mma_mxf4_pair(tmem + W, smem_desc_sw128(base + 1 * kPTileBytes + ks * 32), q, kIdesc, sf, sf, 1u);
+          }
+          mma_commit_pair(smem_u32(&sh->empty[stage]), (uint16_t)3);
+          if (++stage == kPairStages) stage = 0, phase ^= 1u;
+        }
+        if (!ok) break;
+        mma_commit_pair(smem_u32(&sh->tmem_full), (uint16_t)3);
+        acc_phase ^= 1u;
+      }
+      if (sh->abort) {
+        mma_commit_pair(smem_u32(&sh->drained), (uint16_t)1);
+        const uint64_t t0 = global_timer_ns();
+        while (!mbar_try_wait(smem_u32(&sh->drained), 0u) && global_timer_ns() - t0 < kWaitLimitNs) {
+        }
+      }
+    }
+  } else {
+    // ------------------------------ epilogue (both CTAs) ----------------------------------
+    const uint32_t quad = (uint32_t)(warp & 3), half = (uint32_t)((warp - 2) >> 2);
+    const uint32_t base = tmem + ((quad * 32u) << 16) + half * 64u;
+    const uint32_t leader_empty = map_to_cta(smem_u32(&sh->tmem_empty), 0);
+    uint32_t acc_phase = 0;
+    for (int item = pair; item < total_items; item += npairs) {
+      int l, tp, tq;
+      decode_item(p, item, l, tp, tq);
+      if (!__all_sync(0xFFFFFFFFu, wait_bounded(smem_u32(&sh->tmem_full), acc_phase, sh, p.status, 0x500 + warp))) break;
+      tc_fence_after();
+      const uint32_t m = (uint32_t)ep.m[l], recip = ep.recip[l], offset = ep.offset[l];
+      uint32_t t[64];
+      drain_and_release<kFast, true>(base, W, true, offset, leader_empty, true, lane, t);
+      const int64_t j = (int64_t)(2 * tp + (int)rank) * kTileRows + quad * 32 + lane;
+      uint4* dst = reinterpret_cast<uint4*>(ep.res + (size_t)l * ep.res_stride + (size_t)j * (size_t)ep.res_ld +
+                                            (size_t)tq * W + half * 64);
+      reduce_and_store(t, m, recip, dst);
+      acc_phase ^= 1u;
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  cluster_arrive();  // neither CTA leaves while the other may still signal its barriers
+  cluster_wait();
+  tc_fence_after();
+  if (warp == 1) {
+    __syncwarp();
+    tmem_dealloc_pair(tmem, kTmemCols);
   }
 }
 
@@ -577,6 +805,19 @@ int sm_count() {
   return n;
 }
 
+// OZK_GEMM_PAIR=1 in the environment selects the CTA-pair (cta_group::2) kernel where the shape allows it.
+// It is off by default: it moves 25 % fewer bytes from L2 and reads a third less shared memory per
+// MMA, but from K = 12288 on its L2 hit rate collapses (60 % against 85 % at 16384^3, 350 GB against
+// 70 GB of DRAM reads per launch) and it ends up slower under the power cap.
+bool pair_kernel_enabled() {
+  static int v = -1;
+  if (v < 0) {
+    const char* e = getenv("OZK_GEMM_PAIR");
+    v = (e && e[0] == '1') ? 1 : 0;
+  }
+  return v == 1;
+}
+
 template <int NP, int NQ, int W, int STAGES, class Epi>
 ozk_status launch_limb_gemm(const CUtensorMap& map_p, const CUtensorMap& map_q, const GemmCore& core,
                             const typename Epi::Params& ep, cudaStream_t st) {
@@ -609,9 +850,10 @@ ozk_status gemm_residues(const Geometry& g, const ModulusTable& mt, uint8_t* ws,
   core.group = 16;
   core.skip_top_first = (mt.m[0] == 169) ? 1 : 0;  // 13^2 a1 b1 vanishes mod 169 (Section 5.1)
   core.q_groups = 0;
+  core.fast_combine = g.K <= 17476 ? 1 : 0;  // 128 K + 13 * 64 K = 960 K < 2^24
   core.status = reinterpret_cast<StatusBlock*>(ws + g.off_status);
   core.scale_word = 0x80808080u;  // UE8M0 byte 0x80 = 2: both operands doubled, accumulators hold integers
-  ResidueEpilogue::Params ep;
+  ResidueParams ep;
   for (int l = 0; l < kMaxModuli; ++l) {
     ep.m[l] = mt.m[l];
     ep.recip[l] = mt.recip[l];
@@ -620,7 +862,28 @@ ozk_status gemm_residues(const Geometry& g, const ModulusTable& mt, uint8_t* ws,
   ep.res = ws + g.off_res;
   ep.res_ld = g.Mp;
   ep.res_stride = (size_t)g.Mp * (size_t)g.Np;
-  return launch_limb_gemm<2, 2, 128, 3, ResidueEpilogue>(map_p, map_q, core, ep, st);
+  if (g.Np % 256 == 0 && pair_kernel_enabled()) {
+    core.tiles_p = (int)(g.Np / 256);
+    core.group = 8;  // 8 column tiles of 256 = the same 2048-column band as before
+    core.skip_top_first = 0;
+    const size_t smem = (size_t)kPairStages * kPairStageBytes + sizeof(GemmShared) + 1024;
+    static int max_pairs = -1;
+    if (max_pairs < 0) {
+      if (cudaFuncSetAttribute(residue_gemm_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+          cudaFuncSetAttribute(residue_gemm_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return OZK_ERR_CUDA;
+      max_pairs = sm_count() / 2;
+    }
+    const long long items = (long long)core.L * core.tiles_p * core.tiles_q;
+    const int pairs = (int)(items < max_pairs ? items : max_pairs);
+    if (core.fast_combine)
+      residue_gemm_pair_kernel<true><<<2 * pairs, kPairThreads, smem, st>>>(map_p, map_q, core, ep);
+    else
+      residue_gemm_pair_kernel<false><<<2 * pairs, kPairThreads, smem, st>>>(map_p, map_q, core, ep);
+    return cudaGetLastError() == cudaSuccess ? OZK_OK : OZK_ERR_CUDA;
+  }
+  if (core.fast_combine) return launch_limb_gemm<2, 2, 128, 3, ResidueEpilogue<true>>(map_p, map_q, core, ep, st);
+  return launch_limb_gemm<2, 2, 128, 3, ResidueEpilogue<false>>(map_p, map_q, core, ep, st);
 }
 
 // INT8 path: C (int32, column-major) from three limb planes per operand.
@@ -638,6 +901,7 @@ ozk_status gemm_int8(const uint8_t* planes_a, const uint8_t* planes_b, int64_t M
   core.group = 16;
   core.skip_top_first = 0;
   core.q_groups = 0;
+  core.fast_combine = 0;
   core.status = status;
   core.scale_word = 0x80808080u;
   Int32Epilogue::Params ep;
@@ -664,6 +928,7 @@ ozk_status gemm_oz1_passes(const uint8_t* planes_a, const uint8_t* planes_b, int
   core.group = 16;
   core.skip_top_first = 0;
   core.q_groups = 5;
+  core.fast_combine = 0;
   core.status = status;
   core.scale_word = 0x80808080u;
   Int64BlockEpilogue::Params ep;

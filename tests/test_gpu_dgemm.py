@@ -77,3 +77,24 @@ def test_invalid_arguments():
     assert ozk.ozk_dgemm(8, 8, 8, None, 8, None, 8, None, 8, 19, 0) == ozk.OZK_ERR_INVALID_ARG      # null pointers
     assert ozk.ozk_dgemm(4096, 4096, 4096, None, 4096, None, 4096, None, 4096, 19, 0) == ozk.OZK_ERR_WORKSPACE
     assert ozk.ozk_dgemm(0, 8, 8, None, 1, None, 8, None, 1, 19, 0) == ozk.OZK_OK                   # empty result
+
+
+def test_cta_pair_kernel_bit_exact_in_a_subprocess():
+    """The opt-in cta_group::2 variant of the limb GEMM (OZK_GEMM_PAIR=1, column count a multiple of 256)
+    gives the same bits as the oracle."""
+    import os
+    import subprocess
+    import sys
+    code = (
+        "import numpy as np\n"
+        "from oracle import ozaki2\n"
+        "from paper_2608_06812_b200 import inputs\n"
+        "from tests import gpu_util as gu\n"
+        "for (M, N, K, L) in [(256, 256, 256, 14), (384, 512, 1280, 19), (130, 768, 4096, 20), (200, 256, 20000, 19)]:\n"
+        "    A = inputs.lognormal_matrix(M, K, 1.0, seed=0); B = inputs.lognormal_matrix(K, N, 1.0, seed=1)\n"
+        "    assert gu.bits_equal(gu.dgemm(A, B, L), ozaki2.dgemm(A, B, L).C), (M, N, K, L)\n"
+        "print('pair ok')\n")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    out = subprocess.run([sys.executable, "-c", code], cwd=root, env=dict(os.environ, OZK_GEMM_PAIR="1"),
+                         capture_output=True, text=True, timeout=600)
+    assert out.returncode == 0 and "pair ok" in out.stdout, out.stdout + out.stderr
