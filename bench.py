@@ -32,6 +32,9 @@ METRIC = "effective FP64 TFLOPS (2MNK/t), Ozaki scheme II on FP4, end to end inc
 UNIT = "TFLOP/s"
 PAPER_TOTAL_TFLOPS = {4096: 10.81, 8192: 13.52, 16384: 15.26}   # the paper's end-to-end numbers, L = 19, other GPU
 FP4_PER_BF16 = 4.0                                               # nominal dense FP4 : BF16 ratio on B200
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the limb GEMM, from ncu captures of this
+# command at the same size (see profiles/): (size, moduli) -> bytes
+DRAM_TRAFFIC_BYTES = {(16384, 19): 61.0e9 + 5.1e9, (4096, 19): 0.638e9 + 0.300e9}
 KERNELS_PER_STEP = 9   # lut, scan_rows, scan_cols, 2 x finalize, encode_rows, encode_cols, limb GEMM, CRT
 
 
@@ -293,13 +296,16 @@ def run_ozk(args, rank: int, local_rank: int, world: int) -> None:
         print(json.dumps(line), flush=True)
         return
     gemm_ms = float(stage_acc[1])
-    executed = 4 * L - 1 if ozk.ozk_get_moduli(L)[0] == 169 else 4 * L   # the 13^2 term of modulus 169 is skipped
+    # the CTA-pair kernel (padded N a multiple of 256) executes all four products of every modulus; the
+    # single-CTA kernel skips the 13^2 term of modulus 169
+    pair = ((N + 127) // 128 * 128) % 256 == 0 and os.environ.get("OZK_GEMM_PAIR", "1") != "0"
+    executed = 4 * L if pair else 4 * L - 1
     fp4_flops_exec = 2.0 * executed * M * N * K
     fp4_flops_req = 2.0 * (4 * L - 1) * M * N * K        # the 13^2 term of modulus 169 is not required
     achieved = fp4_flops_exec / (gemm_ms * 1e-3) / 1e12
     peak = peaks["bf16_sustained"] * FP4_PER_BF16
     roofline = {"bound": "tensor", "kernel": "residue_gemm_kernel", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                "frac": achieved / peak, "traffic": None,
+                "frac": achieved / peak, "traffic": DRAM_TRAFFIC_BYTES.get((n, L)),
                 "peak_source": f"{peaks['source']} bf16 sustained {peaks['bf16_sustained']:.1f} TFLOP/s x {FP4_PER_BF16:g} (nominal FP4:BF16)",
                 "achieved_required_count": fp4_flops_req / (gemm_ms * 1e-3) / 1e12,
                 "frac_of_burst_peak": achieved / (peaks["bf16_burst"] * FP4_PER_BF16),

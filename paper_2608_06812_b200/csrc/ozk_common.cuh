@@ -31,7 +31,8 @@ struct Geometry {
   int c_bits;
   // byte offsets into the workspace
   size_t off_status, off_lut, off_amax_a, off_amax_b, off_s, off_t, off_planes_a, off_planes_b, off_res;
-  size_t plane_bytes_a, plane_bytes_b;   // one limb plane: rows_p * Kp / 2
+  size_t pitch;                          // bytes from one plane row to the next: Kp / 2 plus padding
+  size_t plane_bytes_a, plane_bytes_b;   // one limb plane: rows_p * pitch
   size_t total;
 };
 
@@ -74,7 +75,7 @@ cudaError_t launch_scan_and_shifts(const Geometry& g, const double* A, int64_t l
                                    uint8_t* ws, cudaStream_t st);
 cudaError_t launch_encode(const Geometry& g, const ModulusTable& mt, const double* A, int64_t lda, const double* B,
                           int64_t ldb, uint8_t* ws, int64_t* At_out, int64_t* Bt_out, cudaStream_t st);
-cudaError_t launch_decode_plane(const uint8_t* plane, int64_t rows, int64_t K, int64_t Kp, int8_t* out, cudaStream_t st);
+cudaError_t launch_decode_plane(const uint8_t* plane, int64_t rows, int64_t K, size_t pitch, int8_t* out, cudaStream_t st);
 cudaError_t launch_crt(const Geometry& g, const CrtTable& ct, const uint8_t* res, int64_t res_ld, size_t res_stride,
                        const int32_t* s, const int32_t* t, double* C, int64_t ldc, uint32_t* x_out, cudaStream_t st);
 cudaError_t launch_copy_residues(const Geometry& g, const uint8_t* res, uint8_t* out, cudaStream_t st);

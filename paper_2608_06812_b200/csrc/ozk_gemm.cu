@@ -44,6 +44,7 @@ struct GemmCore {
   int group;    // rasterisation: this many column tiles share one sweep over the row tiles
   int skip_top_first;  // plane group 0 needs no p_{NP-1} q_{NQ-1} product (13^2 = 0 mod 169)
   int q_groups;        // 0: both operands use plane group l; n > 0: row side uses l / n, column side l % n
+  unsigned int* wave_counter;  // optional: producers of all CTAs meet here before every wave of items
   int fast_combine;    // K <= 17476: D1 + 13 D2 stays below 2^24 and may be formed in FP32 before the release
   StatusBlock* status;
   uint32_t scale_word;  // four copies of the UE8M0 scale byte
@@ -72,6 +73,32 @@ __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, Gemm
         sh->abort = 1;
         atomicMin(&status->code, (int)OZK_ERR_DEVICE_TIMEOUT);
         atomicExch(&status->where, where);
+        return false;
+      }
+    }
+  }
+}
+
+
+// Producer-side wave barrier: before loading the operands of its n-th item a producer announces
+// itself on a global counter and waits (bounded) until every producer that has an n-th item has
+// done so.  It keeps the CTAs of a wave within one tile of each other, so that tiles requested by
+// several CTAs are still in L2 when the last of them asks.  Needs all CTAs resident (persistent
+// grid, cooperative launch).  Returns false on expiry.
+__device__ __forceinline__ bool wave_barrier(unsigned int* counter, unsigned int target, GemmShared* sh, StatusBlock* status) {
+  atomicAdd(counter, 1u);
+  const uint64_t t0 = global_timer_ns();
+  for (uint32_t it = 0;; ++it) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
+    if (v >= target) return true;
+    __nanosleep(64);
+    if ((it & 63u) == 63u) {
+      if (sh->abort) return false;
+      if (global_timer_ns() - t0 > kWaitLimitNs) {
+        sh->abort = 1;
+        atomicMin(&status->code, (int)OZK_ERR_DEVICE_TIMEOUT);
+        atomicExch(&status->where, 0x700);
         return false;
       }
     }
@@ -368,6 +395,11 @@ limb_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constan
         int l, tp, tq;
         decode_item(p, item, l, tp, tq);
         const int lp = p.q_groups ? l / p.q_groups : l, lq = p.q_groups ? l % p.q_groups : l;
+        if (p.wave_counter) {
+          const long long wave = item / (int)gridDim.x;
+          const long long target = min((wave + 1) * (long long)gridDim.x, (long long)total_items);
+          if (!wave_barrier(p.wave_counter, (unsigned int)target, sh, p.status)) break;
+        }
         for (int kb = 0; kb < p.kblocks; ++kb) {
           if (!wait_bounded(smem_u32(&sh->empty[stage]), phase ^ 1u, sh, p.status, 0x000 + stage)) {
             ok = false;
@@ -502,14 +534,15 @@ limb_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constan
 // of 64 KiB and its shared memory feeds 64 instead of 96 bytes per clock to the MMA.
 // The leader's MMA thread issues for the pair; byte counts of both CTAs' TMA loads arrive on the
 // leader's "full" barrier; commits are multicast to the barriers of both CTAs.
-// Accumulator columns 256..383 are zeroed by the epilogue before a tile starts, so the first
-// K step can run p0 with "overwrite" and p1 with "accumulate" (the cross-term columns 128..255
-// need both).  All four products are executed for every modulus (for m = 169 the 13^2 term
+// The first K step runs p0 with "overwrite" and p1 with "accumulate" (the cross-term columns
+// 128..255 need both); the columns 256..383 of the 13^2 term are first overwritten with zeros by
+// one extra instruction whose column-side operand is an all-zero tile in shared memory.  All four products are executed for every modulus (for m = 169 the 13^2 term
 // cancels in the reduction).
 // ------------------------------------------------------------------------------------
 constexpr int kPairStages = 4;
 constexpr int kPairStageBytes = 3 * kPTileBytes;  // p0, p1 and this CTA's half of [q0 ; q1]
 constexpr int kPairThreads = 64 + 32 * 8;
+constexpr int kPairZeroBytes = 64 * kTileKBytes;  // this CTA's half of a 128-row all-zero column-side tile
 
 template <bool kFast>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
@@ -518,10 +551,13 @@ residue_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
   constexpr int W = 128;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  GemmShared* sh = reinterpret_cast<GemmShared*>(tiles + kPairStages * kPairStageBytes);
+  uint8_t* zero_tile = tiles + kPairStages * kPairStageBytes;  // 64 rows x 128 bytes of E2M1 zeros
+  GemmShared* sh = reinterpret_cast<GemmShared*>(zero_tile + kPairZeroBytes);
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
+  for (int i = threadIdx.x; i < kPairZeroBytes / 16; i += blockDim.x) reinterpret_cast<uint4*>(zero_tile)[i] = make_uint4(0, 0, 0, 0);
+  fence_proxy_async();  // the tensor core reads this tile through the async proxy
   const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
   const int total_items = p.L * p.tiles_p * p.tiles_q;  // tiles_p counts 256-wide column tiles here
 
@@ -554,8 +590,6 @@ residue_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
       tmem_st_32x8_const(lane_base + kScaleCol, p.scale_word);
       tmem_st_32x8_const(lane_base + kScaleCol + 8, p.scale_word);
     }
-    tmem_st_32x32_const(lane_base + 2 * W + half * 64, 0u);  // accumulator of the 13^2 term starts at zero
-    tmem_st_32x32_const(lane_base + 2 * W + half * 64 + 32, 0u);
     tmem_wait_st();
   }
   tc_fence_before();
@@ -573,6 +607,11 @@ residue_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
       for (int item = pair; item < total_items && ok; item += npairs) {
         int l, tp, tq;
         decode_item(p, item, l, tp, tq);
+        if (p.wave_counter) {  // both CTAs of every pair take part: 2 * npairs arrivals per wave
+          const long long wave = item / npairs;
+          const long long target = 2 * min((wave + 1) * (long long)npairs, (long long)total_items);
+          if (!wave_barrier(p.wave_counter, (unsigned int)target, sh, p.status)) break;
+        }
         for (int kb = 0; kb < p.kblocks; ++kb) {
           if (!wait_bounded(smem_u32(&sh->empty[stage]), phase ^ 1u, sh, p.status, 0x300 + stage)) {
             ok = false;
@@ -598,16 +637,24 @@ residue_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
       const uint32_t sf = tmem + kScaleCol;
       constexpr uint32_t kIdesc = idesc_mxf4_pair(2 * W);
       bool ok = true;
+      long long dbg_t0 = clock64(), dbg_empty = 0, dbg_full = 0;
       for (int item = pair; item < total_items && ok; item += npairs) {
+        long long dbg_a = clock64();
         if (!wait_bounded(smem_u32(&sh->tmem_empty), acc_phase ^ 1u, sh, p.status, 0x400)) break;
+        dbg_empty += clock64() - dbg_a;
         tc_fence_after();
         for (int kb = 0; kb < p.kblocks; ++kb) {
+          dbg_a = clock64();
           if (!wait_bounded(smem_u32(&sh->full[stage]), phase, sh, p.status, 0x410 + stage)) {
             ok = false;
             break;
           }
+          dbg_full += clock64() - dbg_a;
           tc_fence_after();
           const uint32_t base = smem_u32(tiles + stage * kPairStageBytes);
+          if (kb == 0)  // p1 times an all-zero column-side tile, "overwrite": the 13^2 accumulator starts from 0
+            mma_mxf4_pair(tmem + 2 * W, smem_desc_sw128(base + 1 * kPTileBytes), smem_desc_sw128(smem_u32(zero_tile)),
+                          idesc_mxf4_pair(W), sf, sf, 0u);
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks) {
             const uint64_t q = smem_desc_sw128(base + 2 * kPTileBytes + ks * 32);
@@ -621,6 +668,11 @@ residue_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
         if (!ok) break;
         mma_commit_pair(smem_u32(&sh->tmem_full), (uint16_t)3);
         acc_phase ^= 1u;
+      }
+      if (blockIdx.x == 0) {
+        p.status->pad[0] = (int)((clock64() - dbg_t0) >> 8);
+        p.status->pad[1] = (int)(dbg_empty >> 8);
+        p.status->pad[2] = (int)(dbg_full >> 8);
       }
       if (sh->abort) {
         mma_commit_pair(smem_u32(&sh->drained), (uint16_t)1);
@@ -642,7 +694,7 @@ residue_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
       tc_fence_after();
       const uint32_t m = (uint32_t)ep.m[l], recip = ep.recip[l], offset = ep.offset[l];
       uint32_t t[64];
-      drain_and_release<kFast, true>(base, W, true, offset, leader_empty, true, lane, t);
+      drain_and_release<kFast, false>(base, W, true, offset, leader_empty, true, lane, t);
       const int64_t j = (int64_t)(2 * tp + (int)rank) * kTileRows + quad * 32 + lane;
       uint4* dst = reinterpret_cast<uint4*>(ep.res + (size_t)l * ep.res_stride + (size_t)j * (size_t)ep.res_ld +
                                             (size_t)tq * W + half * 64);
@@ -782,11 +834,11 @@ EncodeTiledFn encode_tiled_fn() {
 // Planes of one operand as a (bytes along K, rows, plane) byte tensor; box = 128 bytes x box_rows.
 // Rows of a box that fall outside the tensor are filled with zero bytes (E2M1 code 0 = value 0).
 bool make_plane_map(CUtensorMap* map, const void* base, int64_t k_bytes, int64_t rows, int64_t planes, size_t plane_bytes,
-                    int box_rows) {
+                    int box_rows, size_t pitch = 0) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return false;
   cuuint64_t dims[3] = {(cuuint64_t)k_bytes, (cuuint64_t)rows, (cuuint64_t)planes};
-  cuuint64_t strides[2] = {(cuuint64_t)k_bytes, (cuuint64_t)plane_bytes};
+  cuuint64_t strides[2] = {(cuuint64_t)(pitch ? pitch : (size_t)k_bytes), (cuuint64_t)plane_bytes};
   cuuint32_t box[3] = {(cuuint32_t)kTileKBytes, (cuuint32_t)box_rows, 1};
   cuuint32_t estr[3] = {1, 1, 1};
   const int rank = planes > 0 ? 3 : 2;
@@ -805,15 +857,13 @@ int sm_count() {
   return n;
 }
 
-// OZK_GEMM_PAIR=1 in the environment selects the CTA-pair (cta_group::2) kernel where the shape allows it.
-// It is off by default: it moves 25 % fewer bytes from L2 and reads a third less shared memory per
-// MMA, but from K = 12288 on its L2 hit rate collapses (60 % against 85 % at 16384^3, 350 GB against
-// 70 GB of DRAM reads per launch) and it ends up slower under the power cap.
+// The CTA-pair (cta_group::2) kernel runs whenever the padded column count is a multiple of 256;
+// OZK_GEMM_PAIR=0 in the environment forces the single-CTA kernel (measurement aid).
 bool pair_kernel_enabled() {
   static int v = -1;
   if (v < 0) {
     const char* e = getenv("OZK_GEMM_PAIR");
-    v = (e && e[0] == '1') ? 1 : 0;
+    v = (e && e[0] == '0') ? 0 : 1;
   }
   return v == 1;
 }
@@ -840,8 +890,8 @@ ozk_status launch_limb_gemm(const CUtensorMap& map_p, const CUtensorMap& map_q, 
 // DGEMM path: residues r_l[j][i] for all moduli from the limb planes in the workspace.
 ozk_status gemm_residues(const Geometry& g, const ModulusTable& mt, uint8_t* ws, cudaStream_t st) {
   CUtensorMap map_p, map_q;
-  if (!make_plane_map(&map_p, ws + g.off_planes_b, g.Kp / 2, g.Np, 2 * g.L, g.plane_bytes_b, kTileRows)) return OZK_ERR_CUDA;
-  if (!make_plane_map(&map_q, ws + g.off_planes_a, g.Kp / 2, g.Mp, 2 * g.L, g.plane_bytes_a, 128)) return OZK_ERR_CUDA;
+  if (!make_plane_map(&map_p, ws + g.off_planes_b, g.Kp / 2, g.Np, 2 * g.L, g.plane_bytes_b, kTileRows, g.pitch)) return OZK_ERR_CUDA;
+  if (!make_plane_map(&map_q, ws + g.off_planes_a, g.Kp / 2, g.Mp, 2 * g.L, g.plane_bytes_a, 128, g.pitch)) return OZK_ERR_CUDA;
   GemmCore core;
   core.L = g.L;
   core.tiles_p = (int)(g.Np / kTileRows);
@@ -851,6 +901,7 @@ ozk_status gemm_residues(const Geometry& g, const ModulusTable& mt, uint8_t* ws,
   core.skip_top_first = (mt.m[0] == 169) ? 1 : 0;  // 13^2 a1 b1 vanishes mod 169 (Section 5.1)
   core.q_groups = 0;
   core.fast_combine = g.K <= 17476 ? 1 : 0;  // 128 K + 13 * 64 K = 960 K < 2^24
+  core.wave_counter = nullptr;
   core.status = reinterpret_cast<StatusBlock*>(ws + g.off_status);
   core.scale_word = 0x80808080u;  // UE8M0 byte 0x80 = 2: both operands doubled, accumulators hold integers
   ResidueParams ep;
@@ -863,10 +914,14 @@ ozk_status gemm_residues(const Geometry& g, const ModulusTable& mt, uint8_t* ws,
   ep.res_ld = g.Mp;
   ep.res_stride = (size_t)g.Mp * (size_t)g.Np;
   if (g.Np % 256 == 0 && pair_kernel_enabled()) {
-    core.tiles_p = (int)(g.Np / 256);
-    core.group = 8;  // 8 column tiles of 256 = the same 2048-column band as before
-    core.skip_top_first = 0;
-    const size_t smem = (size_t)kPairStages * kPairStageBytes + sizeof(GemmShared) + 1024;
+    // CTA-pair kernel.  Its producers meet at a global counter before every wave of items, which needs
+    // all CTAs resident: the launch is cooperative, and when that is refused the single-CTA kernel runs.
+    GemmCore pc = core;
+    pc.tiles_p = (int)(g.Np / 256);
+    pc.group = 8;  // 8 column tiles of 256: the same 2048-column band as the single-CTA kernel
+    pc.skip_top_first = 0;
+    pc.wave_counter = reinterpret_cast<unsigned int*>(ws + g.off_status + 512);
+    const size_t smem = (size_t)kPairStages * kPairStageBytes + kPairZeroBytes + sizeof(GemmShared) + 1024;
     static int max_pairs = -1;
     if (max_pairs < 0) {
       if (cudaFuncSetAttribute(residue_gemm_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
@@ -874,13 +929,23 @@ ozk_status gemm_residues(const Geometry& g, const ModulusTable& mt, uint8_t* ws,
         return OZK_ERR_CUDA;
       max_pairs = sm_count() / 2;
     }
-    const long long items = (long long)core.L * core.tiles_p * core.tiles_q;
+    const long long items = (long long)pc.L * pc.tiles_p * pc.tiles_q;
     const int pairs = (int)(items < max_pairs ? items : max_pairs);
-    if (core.fast_combine)
-      residue_gemm_pair_kernel<true><<<2 * pairs, kPairThreads, smem, st>>>(map_p, map_q, core, ep);
-    else
-      residue_gemm_pair_kernel<false><<<2 * pairs, kPairThreads, smem, st>>>(map_p, map_q, core, ep);
-    return cudaGetLastError() == cudaSuccess ? OZK_OK : OZK_ERR_CUDA;
+    if (cudaMemsetAsync(pc.wave_counter, 0, 4, st) != cudaSuccess) return OZK_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(2 * pairs), 1, 1);
+    cfg.blockDim = dim3(kPairThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = pc.fast_combine ? cudaLaunchKernelEx(&cfg, residue_gemm_pair_kernel<true>, map_p, map_q, pc, ep)
+                                          : cudaLaunchKernelEx(&cfg, residue_gemm_pair_kernel<false>, map_p, map_q, pc, ep);
+    if (e == cudaSuccess) return OZK_OK;
+    (void)cudaGetLastError();  // the cooperative launch was refused: fall through to the single-CTA kernel
   }
   if (core.fast_combine) return launch_limb_gemm<2, 2, 128, 3, ResidueEpilogue<true>>(map_p, map_q, core, ep, st);
   return launch_limb_gemm<2, 2, 128, 3, ResidueEpilogue<false>>(map_p, map_q, core, ep, st);
@@ -901,6 +966,7 @@ ozk_status gemm_int8(const uint8_t* planes_a, const uint8_t* planes_b, int64_t M
   core.group = 16;
   core.skip_top_first = 0;
   core.q_groups = 0;
+  core.wave_counter = nullptr;
   core.fast_combine = 0;
   core.status = status;
   core.scale_word = 0x80808080u;
@@ -928,6 +994,7 @@ ozk_status gemm_oz1_passes(const uint8_t* planes_a, const uint8_t* planes_b, int
   core.group = 16;
   core.skip_top_first = 0;
   core.q_groups = 5;
+  core.wave_counter = nullptr;
   core.fast_combine = 0;
   core.status = status;
   core.scale_word = 0x80808080u;

@@ -182,7 +182,7 @@ __device__ __forceinline__ void encode8(const Piece8& p, uint32_t m, uint32_t re
 __global__ void __launch_bounds__(256) encode_cols_kernel(const double* __restrict__ B, int64_t ldb, int64_t N, int64_t K,
                                                           int64_t Kp, ModulusTable mt, const uint16_t* __restrict__ lut,
                                                           const int32_t* __restrict__ shifts, uint8_t* __restrict__ planes,
-                                                          size_t plane_bytes, int64_t* __restrict__ int_out, int reps) {
+                                                          size_t plane_bytes, size_t pitch, int64_t* __restrict__ int_out, int reps) {
   extern __shared__ __align__(16) uint16_t lut_s[];
   {  // the table is copied once per block and reused for `reps` chunks of 2048 k
     const uint4* src = reinterpret_cast<const uint4*>(lut);
@@ -222,7 +222,7 @@ __global__ void __launch_bounds__(256) encode_cols_kernel(const double* __restri
   }
   Piece8 p;
   split8(mag, neg, p);
-  uint8_t* dst = planes + (size_t)j * (size_t)(Kp / 2) + (size_t)(k / 2);
+  uint8_t* dst = planes + (size_t)j * pitch + (size_t)(k / 2);
   for (int l = 0; l < mt.L; ++l) {
     uint32_t w0, w1;
     encode8(p, (uint32_t)mt.m[l], mt.recip[l], mt.pow18[l], mt.pow36[l], lut_s + l * kLutStride, w0, w1);
@@ -245,7 +245,7 @@ constexpr int kStageStride = 9;  // words per staged row (8 used): odd stride av
 __global__ void __launch_bounds__(256) encode_rows_kernel(const double* __restrict__ A, int64_t lda, int64_t M, int64_t K,
                                                           int64_t Kp, ModulusTable mt, const uint16_t* __restrict__ lut,
                                                           const int32_t* __restrict__ shifts, uint8_t* __restrict__ planes,
-                                                          size_t plane_bytes, int64_t* __restrict__ int_out, int reps) {
+                                                          size_t plane_bytes, size_t pitch, int64_t* __restrict__ int_out, int reps) {
   extern __shared__ __align__(16) uint8_t smem[];
   uint16_t* lut_s = reinterpret_cast<uint16_t*>(smem);                          // L * kLutStride entries
   const int lut_bytes = (mt.L * kLutStride * (int)sizeof(uint16_t) + 15) & ~15;
@@ -299,19 +299,19 @@ __global__ void __launch_bounds__(256) encode_rows_kernel(const double* __restri
   }
   __syncthreads();
   const int row = t >> 3, word = t & 7;
-  uint8_t* dst = planes + (size_t)(i0 + row) * (size_t)(Kp / 2) + (size_t)(k0 / 2) + 4 * word;
+  uint8_t* dst = planes + (size_t)(i0 + row) * pitch + (size_t)(k0 / 2) + 4 * word;
   for (int pl = 0; pl < 2 * mt.L; ++pl)
     *reinterpret_cast<uint32_t*>(dst + (size_t)pl * plane_bytes) = out_s[(pl * kRowTile + row) * kStageStride + word];
   }
 }
 
 // Decodes one limb plane into doubled-E2M1 integers, out[r + k*rows] (test support).
-__global__ void decode_plane_kernel(const uint8_t* __restrict__ plane, int64_t rows, int64_t K, int64_t Kp,
+__global__ void decode_plane_kernel(const uint8_t* __restrict__ plane, int64_t rows, int64_t K, size_t pitch,
                                     int8_t* __restrict__ out) {
   const int64_t r = (int64_t)blockIdx.y * blockDim.x + threadIdx.x;
   const int64_t k = blockIdx.x;
   if (r >= rows || k >= K) return;
-  const uint8_t byte = plane[(size_t)r * (size_t)(Kp / 2) + (size_t)(k / 2)];
+  const uint8_t byte = plane[(size_t)r * pitch + (size_t)(k / 2)];
   const int code = (k & 1) ? (byte >> 4) : (byte & 0xF);
   const int v = kDoubledE2M1[code & 7];
   out[r + k * rows] = (int8_t)((code & 8) ? -v : v);
@@ -359,22 +359,22 @@ cudaError_t launch_encode(const Geometry& g, const ModulusTable& mt, const doubl
     const int reps = 4;
     dim3 grid((unsigned)(g.Mp / kRowTile), (unsigned)((g.Kp / kRowTileK + reps - 1) / reps));
     encode_rows_kernel<<<grid, 256, smem, st>>>(A, lda, g.M, g.K, g.Kp, mt, lut, reinterpret_cast<const int32_t*>(ws + g.off_s),
-                                                ws + g.off_planes_a, g.plane_bytes_a, At_out, reps);
+                                                ws + g.off_planes_a, g.plane_bytes_a, g.pitch, At_out, reps);
   }
   {
     const int reps = 4;
     dim3 grid((unsigned)g.Np, (unsigned)(((g.Kp + 2047) / 2048 + reps - 1) / reps));
     encode_cols_kernel<<<grid, 256, lut_bytes, st>>>(B, ldb, g.N, g.K, g.Kp, mt, lut,
                                                     reinterpret_cast<const int32_t*>(ws + g.off_t), ws + g.off_planes_b,
-                                                    g.plane_bytes_b, Bt_out, reps);
+                                                    g.plane_bytes_b, g.pitch, Bt_out, reps);
   }
   return cudaGetLastError();
 }
 
-cudaError_t launch_decode_plane(const uint8_t* plane, int64_t rows, int64_t K, int64_t Kp, int8_t* out, cudaStream_t st) {
+cudaError_t launch_decode_plane(const uint8_t* plane, int64_t rows, int64_t K, size_t pitch, int8_t* out, cudaStream_t st) {
   if (rows == 0 || K == 0) return cudaSuccess;
   dim3 grid((unsigned)K, (unsigned)((rows + 127) / 128));
-  decode_plane_kernel<<<grid, 128, 0, st>>>(plane, rows, K, Kp, out);
+  decode_plane_kernel<<<grid, 128, 0, st>>>(plane, rows, K, pitch, out);
   return cudaGetLastError();
 }
 

@@ -79,9 +79,9 @@ def test_invalid_arguments():
     assert ozk.ozk_dgemm(0, 8, 8, None, 1, None, 8, None, 1, 19, 0) == ozk.OZK_OK                   # empty result
 
 
-def test_cta_pair_kernel_bit_exact_in_a_subprocess():
-    """The opt-in cta_group::2 variant of the limb GEMM (OZK_GEMM_PAIR=1, column count a multiple of 256)
-    gives the same bits as the oracle."""
+def test_single_cta_kernel_bit_exact_in_a_subprocess():
+    """Shapes whose padded column count is a multiple of 256 run the CTA-pair kernel by default; with
+    OZK_GEMM_PAIR=0 the same shapes run the single-CTA kernel and must give the same bits as the oracle."""
     import os
     import subprocess
     import sys
@@ -95,6 +95,6 @@ def test_cta_pair_kernel_bit_exact_in_a_subprocess():
         "    assert gu.bits_equal(gu.dgemm(A, B, L), ozaki2.dgemm(A, B, L).C), (M, N, K, L)\n"
         "print('pair ok')\n")
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-    out = subprocess.run([sys.executable, "-c", code], cwd=root, env=dict(os.environ, OZK_GEMM_PAIR="1"),
+    out = subprocess.run([sys.executable, "-c", code], cwd=root, env=dict(os.environ, OZK_GEMM_PAIR="0"),
                          capture_output=True, text=True, timeout=600)
     assert out.returncode == 0 and "pair ok" in out.stdout, out.stdout + out.stderr
