@@ -14,7 +14,8 @@ constexpr int kTileKNibbles = 256;   // k extent of one pipeline stage: 256 E2M1
 constexpr int kTileKBytes = 128;
 constexpr int kMaxModuli = OZK_MAX_MODULI;
 constexpr int kCrtWords = 6;         // 192-bit integers cover sum r_l w_l for all 27 moduli
-constexpr int kLutStride = 352;      // 16-bit entries per modulus in the limb-pair table: residues 0 .. 2m-1, m <= 169
+constexpr int kLutStride = 192;      // 16-bit entries per modulus in the limb-pair table: centred residues -96 .. 95
+constexpr int kLutOffset = 96;
 
 // ---- status word (first bytes of the workspace) -------------------------------------
 struct StatusBlock {
@@ -43,8 +44,10 @@ struct ModulusTable {
   int L;
   int m[kMaxModuli];
   uint32_t recip[kMaxModuli];      // floor(2^32 / m)
-  uint32_t pow18[kMaxModuli];      // 2^18 mod m
-  uint32_t pow36[kMaxModuli];      // 2^36 mod m
+  // encoder constants (FP32 arithmetic on exact small integers): centred residues of 2^14, 2^28, 2^42
+  float c14[kMaxModuli], c28[kMaxModuli], c42[kMaxModuli];
+  float inv_m[kMaxModuli];         // 1 / m rounded to FP32
+  float m_f[kMaxModuli];           // m
 };
 
 struct CrtTable {

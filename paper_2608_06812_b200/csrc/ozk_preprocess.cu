@@ -1,7 +1,7 @@
 // Preprocessing kernels (Section 4.2 shared-exponent conversion; Section 5.1 residues and
 // two-limb encoding; Section 6.2 fused decomposition with K-contiguous write-out).
 //
-//   build_lut         per modulus, for every x in [0, 2m) one limb pair (c0, c1) as two E2M1 codes
+//   build_lut         per modulus, for every centred residue one limb pair (c0, c1) as two E2M1 codes
 //   scan_rows/cols    max |.| over the rows of A / the columns of B (exponent scan)
 //   finalize_shifts   s_i = c - 1 - e_i, t_j likewise; flags NaN/Inf
 //   encode_cols       B-side planes: source is already K-contiguous
@@ -18,30 +18,29 @@ namespace {
 __device__ __constant__ int8_t kDoubledE2M1[8] = {0, 1, 2, 3, 4, 6, 8, 12};
 
 // ------------------------------------------------------------------------------------
-// Limb-pair table: for modulus m and every x in [0, 2m) one 16-bit entry holding the E2M1 codes of a
-// limb pair (c0, c1) with c0 + 13 c1 = x (mod m): code(c0) in bits 0..3, code(c1) in bits 8..11.
-// Both limbs are in S and the pair minimises max(|c0|,|c1|), then |c0|+|c1|.  The range 2m lets the
-// encoder skip the last conditional subtraction of its modular reduction.
+// Limb-pair table: for modulus m and every centred residue r in [-96, 96) one 16-bit entry (index
+// r + 96) holding the E2M1 codes of a limb pair (c0, c1) with c0 + 13 c1 = r (mod m): code(c0) in bits
+// 0..3, code(c1) in bits 8..11.  Both limbs are in S and the pair minimises max(|c0|,|c1|), then
+// |c0|+|c1|.  The encoder's residue is centred (|r| <= m/2 + 2 <= 87), so the sign of the converted
+// integer needs no separate handling.
 // ------------------------------------------------------------------------------------
 __global__ void build_lut_kernel(ModulusTable mt, uint16_t* __restrict__ lut) {
   const int l = blockIdx.x;
   const int m = mt.m[l];
   for (int x = threadIdx.x; x < kLutStride; x += blockDim.x) {
+    const int rho = ((x - kLutOffset) % m + m) % m;
     int best_key = 1 << 30, best = 0;
-    if (x < 2 * m) {
-      const int rho = x % m;
-      for (int i1 = 0; i1 < 16; ++i1) {
-        for (int i0 = 0; i0 < 16; ++i0) {
-          if ((i0 == 8) || (i1 == 8)) continue;  // skip the negative-zero codes
-          const int c0 = kDoubledE2M1[i0 & 7] * ((i0 & 8) ? -1 : 1);
-          const int c1 = kDoubledE2M1[i1 & 7] * ((i1 & 8) ? -1 : 1);
-          if ((c0 + 13 * c1 - rho) % m != 0) continue;
-          const int a0 = abs(c0), a1 = abs(c1);
-          const int key = max(a0, a1) * 64 + (a0 + a1);
-          if (key < best_key) {
-            best_key = key;
-            best = (i1 << 8) | i0;
-          }
+    for (int i1 = 0; i1 < 16; ++i1) {
+      for (int i0 = 0; i0 < 16; ++i0) {
+        if ((i0 == 8) || (i1 == 8)) continue;  // skip the negative-zero codes
+        const int c0 = kDoubledE2M1[i0 & 7] * ((i0 & 8) ? -1 : 1);
+        const int c1 = kDoubledE2M1[i1 & 7] * ((i1 & 8) ? -1 : 1);
+        if ((c0 + 13 * c1 - rho) % m != 0) continue;
+        const int a0 = abs(c0), a1 = abs(c1);
+        const int key = max(a0, a1) * 64 + (a0 + a1);
+        if (key < best_key) {
+          best_key = key;
+          best = (i1 << 8) | i0;
         }
       }
     }
@@ -134,29 +133,34 @@ __device__ __forceinline__ unsigned long long to_integer_magnitude(double x, int
   return q + ((rem > half) || (rem == half && (q & 1ull)) ? 1ull : 0ull);
 }
 
-// Eight consecutive-k integers of one plane row, split into 18-bit pieces, with sign masks.
+// Eight consecutive-k integers of one plane row as four signed 14-bit pieces each, held in FP32
+// (a = x3 2^42 + x2 2^28 + x1 2^14 + x0, every piece carrying the sign of a).
 struct Piece8 {
-  uint32_t x0[8], x1[8], x2[8];
-  uint32_t sgn[8];  // 0x0808 for negative values: flips the sign bit of both E2M1 codes of a table entry
+  float x0[8], x1[8], x2[8], x3[8];
 };
 
 __device__ __forceinline__ void split8(const unsigned long long (&mag)[8], const bool (&neg)[8], Piece8& p) {
 #pragma unroll
   for (int e = 0; e < 8; ++e) {
-    p.x0[e] = (uint32_t)(mag[e] & 0x3FFFFull);
-    p.x1[e] = (uint32_t)((mag[e] >> 18) & 0x3FFFFull);
-    p.x2[e] = (uint32_t)(mag[e] >> 36);
-    p.sgn[e] = neg[e] ? 0x0808u : 0u;
+    const float sgn = neg[e] ? -1.0f : 1.0f;
+    p.x0[e] = sgn * (float)(uint32_t)(mag[e] & 0x3FFFull);
+    p.x1[e] = sgn * (float)(uint32_t)((mag[e] >> 14) & 0x3FFFull);
+    p.x2[e] = sgn * (float)(uint32_t)((mag[e] >> 28) & 0x3FFFull);
+    p.x3[e] = sgn * (float)(uint32_t)(mag[e] >> 42);  // <= 2^11
   }
 }
 
-// Residues of the eight values mod m_l and their limb codes packed as 8 nibbles per limb.
-// |a| = x2 2^36 + x1 2^18 + x0  =>  t = x2 (2^36 mod m) + x1 (2^18 mod m) + x0 < 2^27; one multiply-high
-// gives x = t - floor'(t/m) m in [0, 2m), which indexes the table directly; limbs(-rho) = -limbs(rho)
-// because S is symmetric.  Two neighbouring k share a byte: entry(even k) | entry(odd k) << 4 has the
-// byte of limb 0 in bits 0..7 and the byte of limb 1 in bits 8..15.
-__device__ __forceinline__ void encode8(const Piece8& p, uint32_t m, uint32_t recip, uint32_t pow18, uint32_t pow36,
+// Residues of the eight values mod m_l and their limb codes packed as 8 nibbles per limb, on the FP32
+// pipe (the integer pipes of this GPU run at half its rate).  All quantities are small exact integers:
+//   t = x0 + x1 c14 + x2 c28 + x3 c42       |t| < 2^22   (c = centred residues of 2^14, 2^28, 2^42)
+//   q = round(t / m) by the add-2^23 trick,  r = t - q m   centred residue, |r| <= m/2 + 2
+//   byte offset of the table entry = 2 (r + 96), read from the low bits of 2 r + 192 + 1.5 * 2^23
+// Two neighbouring k share a byte: entry(even k) | entry(odd k) << 4 has the byte of limb 0 in bits
+// 0..7 and the byte of limb 1 in bits 8..15.
+__device__ __forceinline__ void encode8(const Piece8& p, float c14, float c28, float c42, float inv_m, float m_f,
                                         const uint16_t* __restrict__ lut_l, uint32_t& w0, uint32_t& w1) {
+  constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23: adding it rounds to an integer in the low mantissa bits
+  const char* lut_bytes = reinterpret_cast<const char*>(lut_l);
   uint32_t pair[4];
 #pragma unroll
   for (int h = 0; h < 4; ++h) {
@@ -164,9 +168,11 @@ __device__ __forceinline__ void encode8(const Piece8& p, uint32_t m, uint32_t re
 #pragma unroll
     for (int o = 0; o < 2; ++o) {
       const int e = 2 * h + o;
-      const uint32_t t = p.x2[e] * pow36 + p.x1[e] * pow18 + p.x0[e];
-      const uint32_t x = t - __umulhi(t, recip) * m;
-      v[o] = (uint32_t)lut_l[x] ^ p.sgn[e];
+      const float t = fmaf(p.x3[e], c42, fmaf(p.x2[e], c28, fmaf(p.x1[e], c14, p.x0[e])));
+      const float q = fmaf(t, inv_m, kMagic) - kMagic;
+      const float r = fmaf(-q, m_f, t);
+      const uint32_t off = __float_as_uint(fmaf(r, 2.0f, kMagic + 2.0f * kLutOffset)) & 0x1FFu;
+      v[o] = *reinterpret_cast<const uint16_t*>(lut_bytes + off);
     }
     pair[h] = v[0] | (v[1] << 4);
   }
@@ -225,7 +231,7 @@ __global__ void __launch_bounds__(256) encode_cols_kernel(const double* __restri
   uint8_t* dst = planes + (size_t)j * pitch + (size_t)(k / 2);
   for (int l = 0; l < mt.L; ++l) {
     uint32_t w0, w1;
-    encode8(p, (uint32_t)mt.m[l], mt.recip[l], mt.pow18[l], mt.pow36[l], lut_s + l * kLutStride, w0, w1);
+    encode8(p, mt.c14[l], mt.c28[l], mt.c42[l], mt.inv_m[l], mt.m_f[l], lut_s + l * kLutStride, w0, w1);
     *reinterpret_cast<uint32_t*>(dst + (size_t)(2 * l) * plane_bytes) = w0;
     *reinterpret_cast<uint32_t*>(dst + (size_t)(2 * l + 1) * plane_bytes) = w1;
   }
@@ -293,7 +299,7 @@ __global__ void __launch_bounds__(256) encode_rows_kernel(const double* __restri
   split8(mag, neg, p);
   for (int l = 0; l < mt.L; ++l) {
     uint32_t w0, w1;
-    encode8(p, (uint32_t)mt.m[l], mt.recip[l], mt.pow18[l], mt.pow36[l], lut_s + l * kLutStride, w0, w1);
+    encode8(p, mt.c14[l], mt.c28[l], mt.c42[l], mt.inv_m[l], mt.m_f[l], lut_s + l * kLutStride, w0, w1);
     out_s[((2 * l) * kRowTile + r) * kStageStride + g] = w0;
     out_s[((2 * l + 1) * kRowTile + r) * kStageStride + g] = w1;
   }
@@ -320,7 +326,7 @@ __global__ void decode_plane_kernel(const uint8_t* __restrict__ plane, int64_t r
 }  // namespace
 
 cudaError_t launch_build_lut(const ModulusTable& mt, uint8_t* lut, cudaStream_t st) {
-  build_lut_kernel<<<mt.L, 384, 0, st>>>(mt, reinterpret_cast<uint16_t*>(lut));
+  build_lut_kernel<<<mt.L, 192, 0, st>>>(mt, reinterpret_cast<uint16_t*>(lut));
   return cudaGetLastError();
 }
 

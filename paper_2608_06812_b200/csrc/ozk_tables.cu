@@ -147,10 +147,18 @@ bool host_build_modulus_table(int L, ModulusTable* t) {
   for (int i = 0; i < L; ++i) {
     uint32_t m = (uint32_t)t->m[i];
     t->recip[i] = (uint32_t)(0x100000000ull / m);
-    t->pow18[i] = (uint32_t)((1ull << 18) % m);
-    t->pow36[i] = (uint32_t)((1ull << 36) % m);
+    auto centred = [m](unsigned long long v) {
+      const long long r = (long long)(v % m);
+      return (float)(r > (long long)(m / 2) ? r - (long long)m : r);
+    };
+    t->c14[i] = centred(1ull << 14);
+    t->c28[i] = centred(1ull << 28);
+    t->c42[i] = centred(1ull << 42);
+    t->inv_m[i] = 1.0f / (float)m;
+    t->m_f[i] = (float)m;
   }
-  for (int i = L; i < kMaxModuli; ++i) t->m[i] = 1, t->recip[i] = 0, t->pow18[i] = 0, t->pow36[i] = 0;
+  for (int i = L; i < kMaxModuli; ++i)
+    t->m[i] = 1, t->recip[i] = 0, t->c14[i] = t->c28[i] = t->c42[i] = 0.0f, t->inv_m[i] = 1.0f, t->m_f[i] = 1.0f;
   return true;
 }
 
