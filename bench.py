@@ -34,7 +34,7 @@ PAPER_TOTAL_TFLOPS = {4096: 10.81, 8192: 13.52, 16384: 15.26}   # the paper's en
 FP4_PER_BF16 = 4.0                                               # nominal dense FP4 : BF16 ratio on B200
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the limb GEMM, from ncu captures of this
 # command at the same size (see profiles/): (size, moduli) -> bytes
-DRAM_TRAFFIC_BYTES = {(16384, 19): 61.0e9 + 5.1e9, (4096, 19): 0.638e9 + 0.300e9}
+DRAM_TRAFFIC_BYTES = {(16384, 19): 61.0e9 + 5.1e9, (4096, 19): 0.638e9 + 0.301e9}
 KERNELS_PER_STEP = 9   # lut, scan_rows, scan_cols, 2 x finalize, encode_rows, encode_cols, limb GEMM, CRT
 
 
@@ -304,7 +304,7 @@ def run_ozk(args, rank: int, local_rank: int, world: int) -> None:
     fp4_flops_req = 2.0 * (4 * L - 1) * M * N * K        # the 13^2 term of modulus 169 is not required
     achieved = fp4_flops_exec / (gemm_ms * 1e-3) / 1e12
     peak = peaks["bf16_sustained"] * FP4_PER_BF16
-    roofline = {"bound": "tensor", "kernel": "residue_gemm_kernel", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+    roofline = {"bound": "tensor", "kernel": "residue_gemm_pair_kernel" if pair else "limb_gemm_kernel", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                 "frac": achieved / peak, "traffic": DRAM_TRAFFIC_BYTES.get((n, L)),
                 "peak_source": f"{peaks['source']} bf16 sustained {peaks['bf16_sustained']:.1f} TFLOP/s x {FP4_PER_BF16:g} (nominal FP4:BF16)",
                 "achieved_required_count": fp4_flops_req / (gemm_ms * 1e-3) / 1e12,
