@@ -43,6 +43,18 @@ def test_every_modulus_count_bit_exact(L):
     assert gu.bits_equal(gu.dgemm(A, B, L), ozaki2.dgemm(A, B, L).C)
 
 
+@pytest.mark.parametrize("shape,L", [((64, 128, 20000), 19), ((40, 256, 65536), 19), ((128, 128, 131072), 20)])
+def test_long_inner_products_bit_exact(shape, L):
+    """K beyond 17476 takes the integer recombination before the TMEM release; K up to 131072 keeps every
+    FP32 partial sum an exact integer (128 K <= 2^24 with limbs |c| <= 8)."""
+    M, N, K = shape
+    A = inputs.lognormal_matrix(M, K, 0.5, seed=20)
+    B = inputs.lognormal_matrix(K, N, 0.5, seed=21)
+    A[0, :] = np.abs(A[0, :])                         # a row of one sign against a column of one sign: no cancellation
+    B[:, 0] = np.abs(B[:, 0])
+    assert gu.bits_equal(gu.dgemm(A, B, L), ozaki2.dgemm(A, B, L).C)
+
+
 def test_small_integers_give_the_exact_integer_product():
     A = inputs.small_integer_matrix(200, 333, 1000, seed=1)
     B = inputs.small_integer_matrix(333, 150, 1000, seed=2)
