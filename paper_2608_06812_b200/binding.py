@@ -37,6 +37,8 @@ SIGNATURES = {
     "ozk_get_async_status": (c_int, [c_void_p]),
     "ozk_dgemm": (c_int, [c_int64, c_int64, c_int64, c_void_p, c_int64, c_void_p, c_int64, c_void_p, c_int64, c_int, c_void_p]),
     "ozk_igemm_i8": (c_int, [c_int64, c_int64, c_int64, c_void_p, c_int64, c_void_p, c_int64, c_void_p, c_int64, c_void_p]),
+    "ozk_dgemm_host_workspace_bytes": (c_size_t, [c_int64, c_int64, c_int64, c_int]),
+    "ozk_dgemm_host": (c_int, [c_int64, c_int64, c_int64, c_void_p, c_int64, c_void_p, c_int64, c_void_p, c_int64, c_int, c_void_p]),
     "ozk_dgemm_oz1_workspace_bytes": (c_size_t, [c_int64, c_int64, c_int64]),
     "ozk_dgemm_oz1": (c_int, [c_int64, c_int64, c_int64, c_void_p, c_int64, c_void_p, c_int64, c_void_p, c_int64, c_void_p]),
     "ozk_stage_preprocess": (c_int, [c_int64, c_int64, c_int64, c_void_p, c_int64, c_void_p, c_int64, c_int,
@@ -174,3 +176,12 @@ def ozk_dgemm_oz1_workspace_bytes(M: int, N: int, K: int) -> int:
 
 def ozk_dgemm_oz1(M, N, K, A, lda, B, ldb, C, ldc, stream=0) -> int:
     return lib().ozk_dgemm_oz1(M, N, K, A, lda, B, ldb, C, ldc, stream)
+
+
+def ozk_dgemm_host_workspace_bytes(M: int, N: int, K: int, num_moduli: int) -> int:
+    return lib().ozk_dgemm_host_workspace_bytes(M, N, K, num_moduli)
+
+
+def ozk_dgemm_host(M, N, K, A, lda, B, ldb, C, ldc, num_moduli, stream=0) -> int:
+    """A, B, C are HOST addresses (pinned memory for full speed)."""
+    return lib().ozk_dgemm_host(M, N, K, A, lda, B, ldb, C, ldc, num_moduli, stream)

@@ -40,7 +40,7 @@ size_t plane_row_padding(int64_t Kp) {
 }
 
 // Workspace layout for an (M, N, K, L) problem.  Returns false on invalid sizes.
-bool make_geometry(int64_t M, int64_t N, int64_t K, int L, Geometry* g) {
+bool make_geometry_impl(int64_t M, int64_t N, int64_t K, int L, Geometry* g) {
   if (M < 0 || N < 0 || K < 0 || L < OZK_MIN_MODULI || L > OZK_MAX_MODULI) return false;
   memset(g, 0, sizeof *g);
   g->M = M;
@@ -109,6 +109,7 @@ ozk_status run_preprocess(const Geometry& g, const ModulusTable& mt, const doubl
 
 }  // namespace
 
+bool make_geometry(int64_t M, int64_t N, int64_t K, int L, Geometry* g) { return make_geometry_impl(M, N, K, L, g); }
 uint8_t* workspace_ptr() { return g_ws.ptr; }
 size_t workspace_bytes() { return g_ws.bytes; }
 

@@ -62,9 +62,10 @@ struct CrtTable {
   int p_bits;                              // bit length of P
 };
 
-// registered workspace (ozk_api.cu)
+// registered workspace and layout (ozk_api.cu)
 uint8_t* workspace_ptr();
 size_t workspace_bytes();
+bool make_geometry(int64_t M, int64_t N, int64_t K, int L, Geometry* g);
 
 // host-side constant builders (ozk_tables.cu)
 int host_select_moduli(int count, int* out);
@@ -74,6 +75,9 @@ bool host_build_crt_table(int L, CrtTable* t);
 
 // kernels' launchers (each returns cudaError_t of the launch)
 cudaError_t launch_build_lut(const ModulusTable& mt, uint8_t* lut, cudaStream_t st);
+cudaError_t launch_scan_operand(const Geometry& g, int which, const double* X, int64_t ldx, uint8_t* ws, cudaStream_t st);
+cudaError_t launch_encode_operand(const Geometry& g, const ModulusTable& mt, int which, const double* X, int64_t ldx,
+                                  uint8_t* ws, int64_t* int_out, cudaStream_t st);
 cudaError_t launch_scan_and_shifts(const Geometry& g, const double* A, int64_t lda, const double* B, int64_t ldb,
                                    uint8_t* ws, cudaStream_t st);
 cudaError_t launch_encode(const Geometry& g, const ModulusTable& mt, const double* A, int64_t lda, const double* B,

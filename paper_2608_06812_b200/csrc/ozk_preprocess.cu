@@ -330,51 +330,71 @@ cudaError_t launch_build_lut(const ModulusTable& mt, uint8_t* lut, cudaStream_t 
   return cudaGetLastError();
 }
 
-cudaError_t launch_scan_and_shifts(const Geometry& g, const double* A, int64_t lda, const double* B, int64_t ldb,
-                                   uint8_t* ws, cudaStream_t st) {
-  auto* amax_a = reinterpret_cast<unsigned long long*>(ws + g.off_amax_a);
-  auto* amax_b = reinterpret_cast<unsigned long long*>(ws + g.off_amax_b);
+// Row shifts s_i of A (which = 0) or column shifts t_j of B (which = 1): maxima, then c - 1 - e.
+cudaError_t launch_scan_operand(const Geometry& g, int which, const double* X, int64_t ldx, uint8_t* ws, cudaStream_t st) {
   auto* status = reinterpret_cast<StatusBlock*>(ws + g.off_status);
-  cudaError_t e = cudaMemsetAsync(amax_a, 0, (size_t)(g.Mp + g.Np) * sizeof(unsigned long long), st);
-  if (e != cudaSuccess) return e;
-  if (g.K > 0) {
-    const int kslab_a = 64;
-    dim3 ga((unsigned)((g.M + 255) / 256), (unsigned)((g.K + kslab_a - 1) / kslab_a));
-    scan_rows_kernel<<<ga, 256, 0, st>>>(A, lda, g.M, g.K, kslab_a, amax_a);
-    const int kslab_b = 2048;
-    dim3 gb((unsigned)g.N, (unsigned)((g.K + kslab_b - 1) / kslab_b));
-    scan_cols_kernel<<<gb, 256, 0, st>>>(B, ldb, g.K, kslab_b, amax_b);
+  if (which == 0) {
+    auto* amax = reinterpret_cast<unsigned long long*>(ws + g.off_amax_a);
+    cudaError_t e = cudaMemsetAsync(amax, 0, (size_t)g.Mp * sizeof(unsigned long long), st);
+    if (e != cudaSuccess) return e;
+    if (g.K > 0) {
+      const int kslab = 64;
+      dim3 grid((unsigned)((g.M + 255) / 256), (unsigned)((g.K + kslab - 1) / kslab));
+      scan_rows_kernel<<<grid, 256, 0, st>>>(X, ldx, g.M, g.K, kslab, amax);
+    }
+    finalize_shifts_kernel<<<(unsigned)((g.Mp + 255) / 256), 256, 0, st>>>(amax, g.M, g.Mp, g.c_bits,
+                                                                          reinterpret_cast<int32_t*>(ws + g.off_s), status);
+  } else {
+    auto* amax = reinterpret_cast<unsigned long long*>(ws + g.off_amax_b);
+    cudaError_t e = cudaMemsetAsync(amax, 0, (size_t)g.Np * sizeof(unsigned long long), st);
+    if (e != cudaSuccess) return e;
+    if (g.K > 0) {
+      const int kslab = 2048;
+      dim3 grid((unsigned)g.N, (unsigned)((g.K + kslab - 1) / kslab));
+      scan_cols_kernel<<<grid, 256, 0, st>>>(X, ldx, g.K, kslab, amax);
+    }
+    finalize_shifts_kernel<<<(unsigned)((g.Np + 255) / 256), 256, 0, st>>>(amax, g.N, g.Np, g.c_bits,
+                                                                          reinterpret_cast<int32_t*>(ws + g.off_t), status);
   }
-  finalize_shifts_kernel<<<(unsigned)((g.Mp + 255) / 256), 256, 0, st>>>(amax_a, g.M, g.Mp, g.c_bits,
-                                                                        reinterpret_cast<int32_t*>(ws + g.off_s), status);
-  finalize_shifts_kernel<<<(unsigned)((g.Np + 255) / 256), 256, 0, st>>>(amax_b, g.N, g.Np, g.c_bits,
-                                                                        reinterpret_cast<int32_t*>(ws + g.off_t), status);
   return cudaGetLastError();
 }
 
-cudaError_t launch_encode(const Geometry& g, const ModulusTable& mt, const double* A, int64_t lda, const double* B,
-                          int64_t ldb, uint8_t* ws, int64_t* At_out, int64_t* Bt_out, cudaStream_t st) {
+cudaError_t launch_scan_and_shifts(const Geometry& g, const double* A, int64_t lda, const double* B, int64_t ldb,
+                                   uint8_t* ws, cudaStream_t st) {
+  cudaError_t e = launch_scan_operand(g, 0, A, lda, ws, st);
+  if (e != cudaSuccess) return e;
+  return launch_scan_operand(g, 1, B, ldb, ws, st);
+}
+
+// Limb planes of A (which = 0, rows of A) or of B (which = 1, columns of B).
+cudaError_t launch_encode_operand(const Geometry& g, const ModulusTable& mt, int which, const double* X, int64_t ldx,
+                                  uint8_t* ws, int64_t* int_out, cudaStream_t st) {
   const uint16_t* lut = reinterpret_cast<const uint16_t*>(ws + g.off_lut);
   const int lut_bytes = (mt.L * kLutStride * (int)sizeof(uint16_t) + 15) & ~15;
-  {
+  const int reps = 4;
+  if (which == 0) {
     const size_t stage = (size_t)2 * mt.L * kRowTile * kStageStride * sizeof(uint32_t);
     const size_t in_bytes = (size_t)kRowTileK * kRowTile * sizeof(double);
     const size_t smem = lut_bytes + (stage > in_bytes ? stage : in_bytes);
     cudaError_t e = cudaFuncSetAttribute(encode_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    const int reps = 4;
     dim3 grid((unsigned)(g.Mp / kRowTile), (unsigned)((g.Kp / kRowTileK + reps - 1) / reps));
-    encode_rows_kernel<<<grid, 256, smem, st>>>(A, lda, g.M, g.K, g.Kp, mt, lut, reinterpret_cast<const int32_t*>(ws + g.off_s),
-                                                ws + g.off_planes_a, g.plane_bytes_a, g.pitch, At_out, reps);
-  }
-  {
-    const int reps = 4;
+    encode_rows_kernel<<<grid, 256, smem, st>>>(X, ldx, g.M, g.K, g.Kp, mt, lut, reinterpret_cast<const int32_t*>(ws + g.off_s),
+                                                ws + g.off_planes_a, g.plane_bytes_a, g.pitch, int_out, reps);
+  } else {
     dim3 grid((unsigned)g.Np, (unsigned)(((g.Kp + 2047) / 2048 + reps - 1) / reps));
-    encode_cols_kernel<<<grid, 256, lut_bytes, st>>>(B, ldb, g.N, g.K, g.Kp, mt, lut,
+    encode_cols_kernel<<<grid, 256, lut_bytes, st>>>(X, ldx, g.N, g.K, g.Kp, mt, lut,
                                                     reinterpret_cast<const int32_t*>(ws + g.off_t), ws + g.off_planes_b,
-                                                    g.plane_bytes_b, g.pitch, Bt_out, reps);
+                                                    g.plane_bytes_b, g.pitch, int_out, reps);
   }
   return cudaGetLastError();
+}
+
+cudaError_t launch_encode(const Geometry& g, const ModulusTable& mt, const double* A, int64_t lda, const double* B,
+                          int64_t ldb, uint8_t* ws, int64_t* At_out, int64_t* Bt_out, cudaStream_t st) {
+  cudaError_t e = launch_encode_operand(g, mt, 0, A, lda, ws, At_out, st);
+  if (e != cudaSuccess) return e;
+  return launch_encode_operand(g, mt, 1, B, ldb, ws, Bt_out, st);
 }
 
 cudaError_t launch_decode_plane(const uint8_t* plane, int64_t rows, int64_t K, size_t pitch, int8_t* out, cudaStream_t st) {
