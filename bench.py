@@ -47,8 +47,9 @@ def parse_args():
     ap.add_argument("--moduli", type=int, default=19)
     ap.add_argument("--phi", type=float, default=1.0)
     ap.add_argument("--impl", default="ozk", choices=["ozk", "reference"])
-    ap.add_argument("--scheme", default="oz2", choices=["oz2", "oz1"],
-                    help="oz2 = Ozaki scheme II (the headline path); oz1 = Ozaki scheme I, 15 x 15 limbs")
+    ap.add_argument("--scheme", default="oz2", choices=["oz2", "oz1", "i8"],
+                    help="oz2 = Ozaki scheme II (the headline path); oz1 = Ozaki scheme I, 15 x 15 limbs; "
+                         "i8 = INT8 x INT8 -> INT32 GEMM on FP4 limbs (reports integer TOP/s)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-fp64-context", action="store_true")
@@ -188,6 +189,46 @@ def reduce_over_ranks(ms_per_step: float, flops_per_step: float, dist=None, devi
 # ---------------------------------------------------------------------------------------------
 # the GPU arm
 # ---------------------------------------------------------------------------------------------
+def run_int8(args) -> None:
+    """INT8 GEMM emulated on FP4 (9 limb products): device-resident timing, one JSON line."""
+    import torch
+    from paper_2608_06812_b200 import binding as ozk
+    from paper_2608_06812_b200 import inputs
+    n = args.size
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    stream = torch.cuda.current_stream().cuda_stream
+    dA = torch.from_numpy(np.ascontiguousarray(inputs.int8_matrix(n, n, seed=0).T)).to(dev)
+    dB = torch.from_numpy(np.ascontiguousarray(inputs.int8_matrix(n, n, seed=1).T)).to(dev)
+    dC = torch.empty((n, n), dtype=torch.int32, device=dev)
+    ws = torch.empty(ozk.ozk_igemm_i8_workspace_bytes(n, n, n), dtype=torch.uint8, device=dev)
+    ozk.check(ozk.ozk_set_workspace(ws.data_ptr(), ws.numel()), "ozk_set_workspace")
+
+    def step():
+        ozk.check(ozk.ozk_igemm_i8(n, n, n, dA.data_ptr(), n, dB.data_ptr(), n, dC.data_ptr(), n, stream), "ozk_igemm_i8")
+    for _ in range(max(args.warmup, 3)):
+        step()
+    ozk.check(ozk.ozk_get_async_status(stream), "status")
+    sampler = ClockSampler(0)
+    sampler.start()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    t0.record()
+    for _ in range(args.steps):
+        step()
+    t1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = t0.elapsed_time(t1) / args.steps
+    ops = 2.0 * n ** 3
+    print(json.dumps({"metric": "INT8 x INT8 -> INT32 GEMM emulated on FP4 limbs, 2MNK/t", "value": ops / (ms * 1e-3) / 1e12,
+                      "unit": "TOP/s", "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms,
+                      "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "fp4_e2m1 (fp32 accumulate, int32 out)",
+                      "data": "synthetic", "config": {"workload": f"M=N=K={n} int8 uniform on [-128,127], seeds 0/1"},
+                      "clocks": clocks, "gpu_launches": 3 * args.steps,
+                      "fp4_tflops_executed_9_products": 9 * ops / (ms * 1e-3) / 1e12}), flush=True)
+
+
 def run_ozk(args, rank: int, local_rank: int, world: int) -> None:
     import torch
     import torch.distributed as dist
@@ -356,6 +397,10 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     if args.impl == "reference":
         run_reference(args, rank, world)
+        return
+    if args.scheme == "i8":
+        if rank == 0:
+            run_int8(args)
         return
     run_ozk(args, rank, local_rank, world)
     if world > 1:

@@ -27,18 +27,6 @@ void mark(int i, cudaStream_t st) {
   if (g_timing.enabled) cudaEventRecord(g_timing.ev[i], st);
 }
 
-// Padding bytes appended to every plane row (a multiple of 16 for TMA).
-size_t plane_row_padding(int64_t Kp) {
-  static long pad = -1;
-  if (pad < 0) {
-    const char* e = getenv("OZK_PLANE_PAD");
-    pad = e ? atol(e) : 0;
-    pad = pad / 16 * 16;
-  }
-  (void)Kp;
-  return (size_t)pad;
-}
-
 // Workspace layout for an (M, N, K, L) problem.  Returns false on invalid sizes.
 bool make_geometry_impl(int64_t M, int64_t N, int64_t K, int L, Geometry* g) {
   if (M < 0 || N < 0 || K < 0 || L < OZK_MIN_MODULI || L > OZK_MAX_MODULI) return false;
@@ -65,7 +53,7 @@ bool make_geometry_impl(int64_t M, int64_t N, int64_t K, int L, Geometry* g) {
   off += align_up((size_t)g->Mp * 4, 1024);
   g->off_t = off;
   off += align_up((size_t)g->Np * 4, 1024);
-  g->pitch = (size_t)(g->Kp / 2) + plane_row_padding(g->Kp);
+  g->pitch = (size_t)(g->Kp / 2);
   g->plane_bytes_a = (size_t)g->Mp * g->pitch;
   g->plane_bytes_b = (size_t)g->Np * g->pitch;
   g->off_planes_a = off;

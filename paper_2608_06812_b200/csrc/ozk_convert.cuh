@@ -1,0 +1,29 @@
+// Shared-exponent integer conversion (Section 4.2): round-to-nearest-even of x * 2^s, done on the integer
+// significand so that the scaling is an exact exponent shift for every finite input, subnormals and
+// shifts beyond the FP64 exponent range included.
+#pragma once
+
+#include <cuda_runtime.h>
+
+namespace ozk {
+
+// Returns the magnitude of round(x * 2^s) (at most 2^53 when |x| is at most its row or column maximum);
+// *neg receives the sign of x.
+__device__ __forceinline__ unsigned long long to_integer_magnitude(double x, int s, bool* neg) {
+  const unsigned long long bits = (unsigned long long)__double_as_longlong(x);
+  *neg = (bits >> 63) != 0;
+  const int E = (int)((bits >> 52) & 0x7FF);
+  unsigned long long mant = bits & 0x000FFFFFFFFFFFFFull;
+  if (E) mant |= 1ull << 52;
+  if (mant == 0) return 0;
+  const int sh = (E ? E : 1) - 1075 + s;  // x * 2^s = mant * 2^sh
+  if (sh >= 0) return sh > 52 ? 0 : mant << sh;  // sh > 0 only for subnormal x; |x 2^s| < 2^53 bounds it by 52
+  const int d = -sh;
+  if (d > 54) return 0;
+  const unsigned long long q = mant >> d;
+  const unsigned long long rem = mant & ((1ull << d) - 1);
+  const unsigned long long half = 1ull << (d - 1);
+  return q + ((rem > half) || (rem == half && (q & 1ull)) ? 1ull : 0ull);
+}
+
+}  // namespace ozk

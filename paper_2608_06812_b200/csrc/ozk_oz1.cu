@@ -14,6 +14,7 @@
 #include <string.h>
 
 #include "ozk_common.cuh"
+#include "ozk_convert.cuh"
 #include "ozk_round.cuh"
 
 namespace ozk {
@@ -56,23 +57,6 @@ __device__ __forceinline__ void decompose15(unsigned long long mag, uint32_t fli
   for (int d = 0; d < kLimbs; ++d) codes[d] ^= (codes[d] & 7u) ? flip : 0u;  // no negative zeros
 }
 
-__device__ __forceinline__ unsigned long long to_integer_magnitude53(double x, int s, bool* neg) {
-  const unsigned long long bits = (unsigned long long)__double_as_longlong(x);
-  *neg = (bits >> 63) != 0;
-  const int E = (int)((bits >> 52) & 0x7FF);
-  unsigned long long mant = bits & 0x000FFFFFFFFFFFFFull;
-  if (E) mant |= 1ull << 52;
-  if (mant == 0) return 0;
-  const int sh = (E ? E : 1) - 1075 + s;  // x * 2^s = mant * 2^sh
-  if (sh >= 0) return sh > 52 ? 0 : mant << sh;
-  const int d = -sh;
-  if (d > 54) return 0;
-  const unsigned long long q = mant >> d;
-  const unsigned long long rem = mant & ((1ull << d) - 1);
-  const unsigned long long half = 1ull << (d - 1);
-  return q + ((rem > half) || (rem == half && (q & 1ull)) ? 1ull : 0ull);
-}
-
 // B side: plane row = column j of B (K contiguous).  Thread = 8 consecutive k, 16 planes written
 // (plane 15 is the all-zero pad that completes the fourth row-side group).
 __global__ void __launch_bounds__(256) oz1_encode_cols_kernel(const double* __restrict__ B, int64_t ldb, int64_t N, int64_t K,
@@ -90,7 +74,7 @@ __global__ void __launch_bounds__(256) oz1_encode_cols_kernel(const double* __re
     for (int e = 0; e < 8; ++e) {
       if (k + e < K) {
         bool neg;
-        const unsigned long long mag = to_integer_magnitude53(__ldg(B + j * ldb + k + e), s, &neg);
+        const unsigned long long mag = to_integer_magnitude(__ldg(B + j * ldb + k + e), s, &neg);
         uint32_t codes[kLimbs];
         decompose15(mag, neg ? 8u : 0u, codes);
 #pragma unroll
@@ -130,7 +114,7 @@ __global__ void __launch_bounds__(256) oz1_encode_rows_kernel(const double* __re
 #pragma unroll
   for (int e = 0; e < 8; ++e) {
     bool neg;
-    const unsigned long long mag = to_integer_magnitude53(in_s[(8 * g + e) * 32 + r], s, &neg);
+    const unsigned long long mag = to_integer_magnitude(in_s[(8 * g + e) * 32 + r], s, &neg);
     uint32_t codes[kLimbs];
     decompose15(mag, neg ? 8u : 0u, codes);
 #pragma unroll

@@ -10,6 +10,7 @@
 // A limb plane is rows_p x Kp nibbles, K-contiguous, two nibbles per byte, the lower-k element
 // in the low nibble.  Plane (l, limb) of an operand starts at (2*l + limb) * plane_bytes.
 #include "ozk_common.cuh"
+#include "ozk_convert.cuh"
 
 namespace ozk {
 namespace {
@@ -110,27 +111,6 @@ __global__ void finalize_shifts_kernel(const unsigned long long* __restrict__ am
     }
   }
   shifts[i] = s;
-}
-
-// ------------------------------------------------------------------------------------
-// Integer conversion: round-to-nearest-even of x * 2^s on the significand (exact shift).
-// Returns the magnitude (<= 2^53); *neg receives the sign.
-// ------------------------------------------------------------------------------------
-__device__ __forceinline__ unsigned long long to_integer_magnitude(double x, int s, bool* neg) {
-  const unsigned long long bits = (unsigned long long)__double_as_longlong(x);
-  *neg = (bits >> 63) != 0;
-  const int E = (int)((bits >> 52) & 0x7FF);
-  unsigned long long mant = bits & 0x000FFFFFFFFFFFFFull;
-  if (E) mant |= 1ull << 52;
-  if (mant == 0) return 0;
-  const int sh = (E ? E : 1) - 1075 + s;  // x * 2^s = mant * 2^sh
-  if (sh >= 0) return sh > 52 ? 0 : mant << sh;  // sh > 0 only for subnormal x; |x 2^s| < 2^53 bounds it by 52
-  const int d = -sh;
-  if (d > 54) return 0;
-  const unsigned long long q = mant >> d;
-  const unsigned long long rem = mant & ((1ull << d) - 1);
-  const unsigned long long half = 1ull << (d - 1);
-  return q + ((rem > half) || (rem == half && (q & 1ull)) ? 1ull : 0ull);
 }
 
 // Eight consecutive-k integers of one plane row as four signed 14-bit pieces each, held in FP32

@@ -9,11 +9,6 @@
 namespace ozk {
 
 template <int NW>
-struct Words {
-  uint32_t w[NW];
-};
-
-template <int NW>
 __device__ __forceinline__ bool ge(const uint32_t (&a)[NW], const uint32_t* b) {  // a >= b
 #pragma unroll
   for (int i = NW - 1; i >= 0; --i) {
