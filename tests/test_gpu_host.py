@@ -48,6 +48,24 @@ def test_back_to_back_calls_and_device_path_agree():
     assert gu.bits_equal(C1, gu.dgemm(A, B1, 19)) and gu.bits_equal(C2, gu.dgemm(A, B2, 19))
 
 
+def test_row_and_column_blocks_agree_with_the_device_path():
+    """More than one block in both directions (4096-row blocks of A, 4096-column blocks of B), with ragged
+    last blocks: the device-resident path, itself checked against the oracle, must give the same bits."""
+    for (M, N, K, L) in [(4100, 4200, 96, 19), (8200, 300, 160, 14), (9000, 8500, 64, 19)]:
+        A = inputs.lognormal_matrix(M, K, 2.0, seed=40)
+        B = inputs.lognormal_matrix(K, N, 2.0, seed=41)
+        A[4097 % M, :] = 0.0
+        C = dgemm_host(A, B, L, lda=M + 2, ldb=K + 3, ldc=M + 1)
+        assert gu.bits_equal(C, gu.dgemm(A, B, L)), (M, N, K, L)
+    # and one ragged multi-block case straight against the oracle on sampled rows / columns
+    M, N, K, L = 4100, 4200, 96, 19
+    A = inputs.lognormal_matrix(M, K, 2.0, seed=40)
+    B = inputs.lognormal_matrix(K, N, 2.0, seed=41)
+    C = dgemm_host(A, B, L)
+    rows = np.array([0, 1, 4095, 4096, 4099]); cols = np.array([0, 255, 4095, 4096, 4199])
+    assert gu.bits_equal(C[np.ix_(rows, cols)], ozaki2.dgemm(A[rows], B[:, cols], L).C)
+
+
 def test_argument_errors():
     gu.register_small_workspace(8 << 20)
     assert ozk.ozk_dgemm_host(4096, 4096, 4096, None, 4096, None, 4096, None, 4096, 19, 0) == ozk.OZK_ERR_WORKSPACE
