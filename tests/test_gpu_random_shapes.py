@@ -1,0 +1,49 @@
+"""Randomised shapes, modulus counts and leading dimensions: ozk_dgemm against the CPU oracle bit for bit, and
+many calls enqueued back to back on one stream before any synchronisation."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ozaki2
+from paper_2608_06812_b200 import binding as ozk
+from paper_2608_06812_b200 import inputs
+from tests import gpu_util as gu
+
+pytestmark = pytest.mark.gpu
+
+
+def test_random_shapes_bit_exact():
+    rng = np.random.default_rng(2024)
+    for trial in range(24):
+        M = int(rng.integers(1, 300))
+        N = int(rng.integers(1, 600))
+        K = int(rng.integers(0, 700))
+        L = int(rng.integers(2, 28))
+        phi = float(rng.choice([0.5, 1.0, 4.0]))
+        A = inputs.lognormal_matrix(M, K, phi, seed=1000 + trial)
+        B = inputs.lognormal_matrix(K, N, phi, seed=2000 + trial)
+        C = gu.dgemm(A, B, L, lda=M + int(rng.integers(0, 5)), ldb=max(K, 1) + int(rng.integers(0, 5)), ldc=M + int(rng.integers(0, 5)))
+        assert gu.bits_equal(C, ozaki2.dgemm(A, B, L).C), (M, N, K, L, phi)
+
+
+def test_back_to_back_calls_without_synchronisation():
+    """Calls that share the workspace are ordered by the stream alone: results of a mixed sequence (both limb-GEMM
+    kernels, different modulus counts) must not depend on host synchronisation between them."""
+    cases = [(256, 256, 512, 19), (130, 70, 300, 14), (384, 512, 256, 20), (64, 768, 1024, 12), (200, 130, 64, 27)]
+    gu.ensure_workspace(max(ozk.ozk_dgemm_workspace_bytes(M, N, K, L) for M, N, K, L in cases))
+    work = []
+    for rep in range(3):
+        for (M, N, K, L) in cases:
+            A = inputs.lognormal_matrix(M, K, 1.0, seed=rep * 10 + L)
+            B = inputs.lognormal_matrix(K, N, 1.0, seed=rep * 10 + L + 1)
+            dA, dB = gu.to_dev_colmajor(A), gu.to_dev_colmajor(B)
+            dC = torch.empty((N, M), dtype=torch.float64, device="cuda")
+            work.append((A, B, L, dA, dB, dC))
+    for (A, B, L, dA, dB, dC) in work:                       # enqueue everything, synchronise once
+        M, K = A.shape
+        N = B.shape[1]
+        ozk.check(ozk.ozk_dgemm(M, N, K, dA.data_ptr(), M, dB.data_ptr(), K, dC.data_ptr(), M, L, gu.stream()), "ozk_dgemm")
+    ozk.check(ozk.ozk_get_async_status(gu.stream()), "status")
+    for (A, B, L, dA, dB, dC) in work:
+        M, N = A.shape[0], B.shape[1]
+        assert gu.bits_equal(gu.from_dev_colmajor(dC, M, N), ozaki2.dgemm(A, B, L).C)
