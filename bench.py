@@ -347,10 +347,9 @@ def run_ozk(args, rank: int, local_rank: int, world: int) -> None:
         print(json.dumps(line), flush=True)
         return
     gemm_ms = float(stage_acc[1])
-    # the CTA-pair kernel (padded N a multiple of 256) executes all four products of every modulus; the
-    # single-CTA kernel skips the 13^2 term of modulus 169
+    # both limb-GEMM kernels skip the 13^2 term of modulus 169: executed = required = 4L - 1 products
     pair = ((N + 127) // 128 * 128) % 256 == 0 and os.environ.get("OZK_GEMM_PAIR", "1") != "0"
-    executed = 4 * L if pair else 4 * L - 1
+    executed = 4 * L - 1 if ozk.ozk_get_moduli(L)[0] == 169 else 4 * L
     fp4_flops_exec = 2.0 * executed * M * N * K
     fp4_flops_req = 2.0 * (4 * L - 1) * M * N * K        # the 13^2 term of modulus 169 is not required
     achieved = fp4_flops_exec / (gemm_ms * 1e-3) / 1e12

@@ -536,8 +536,9 @@ limb_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constan
 // leader's "full" barrier; commits are multicast to the barriers of both CTAs.
 // The first K step runs p0 with "overwrite" and p1 with "accumulate" (the cross-term columns
 // 128..255 need both); the columns 256..383 of the 13^2 term are first overwritten with zeros by
-// one extra instruction whose column-side operand is an all-zero tile in shared memory.  All four products are executed for every modulus (for m = 169 the 13^2 term
-// cancels in the reduction).
+// one extra instruction whose column-side operand is an all-zero tile in shared memory.
+// For m = 169 (13^2 = 0) the p1 q1 product is not needed: those items run three 256 x 128 x 64
+// instructions per K step instead, with each CTA supplying half the rows of q0 and of q1.
 // ------------------------------------------------------------------------------------
 constexpr int kPairStages = 4;
 constexpr int kPairStageBytes = 3 * kPTileBytes;  // p0, p1 and this CTA's half of [q0 ; q1]
@@ -547,7 +548,8 @@ constexpr int kPairZeroBytes = 64 * kTileKBytes;  // this CTA's half of a 128-ro
 template <bool kFast>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
 residue_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_q,
-                         const __grid_constant__ GemmCore p, const __grid_constant__ ResidueParams ep) {
+                         const __grid_constant__ CUtensorMap map_qh, const __grid_constant__ GemmCore p,
+                         const __grid_constant__ ResidueParams ep) {
   constexpr int W = 128;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -624,7 +626,14 @@ residue_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
           const int prow = (2 * tp + (int)rank) * kTileRows;
           tma_load_3d_pair(dst + 0 * kPTileBytes, &map_p, leader_full, x, prow, 2 * l + 0);
           tma_load_3d_pair(dst + 1 * kPTileBytes, &map_p, leader_full, x, prow, 2 * l + 1);
-          tma_load_3d_pair(dst + 2 * kPTileBytes, &map_q, leader_full, x, tq * W, 2 * l + (int)rank);
+          if (p.skip_top_first && l == 0) {
+            // m = 169 needs p0 q0, p0 q1, p1 q0 only: three 128-column instructions, for which this CTA
+            // supplies rows [64 rank, 64 rank + 64) of q0 and of q1 instead of all of one of them
+            tma_load_3d_pair(dst + 2 * kPTileBytes, &map_qh, leader_full, x, tq * W + 64 * (int)rank, 0);
+            tma_load_3d_pair(dst + 2 * kPTileBytes + kPTileBytes / 2, &map_qh, leader_full, x, tq * W + 64 * (int)rank, 1);
+          } else {
+            tma_load_3d_pair(dst + 2 * kPTileBytes, &map_q, leader_full, x, tq * W, 2 * l + (int)rank);
+          }
           if (++stage == kPairStages) stage = 0, phase ^= 1u;
         }
       }
@@ -639,6 +648,9 @@ residue_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
       bool ok = true;
       long long dbg_t0 = clock64(), dbg_empty = 0, dbg_full = 0;
       for (int item = pair; item < total_items && ok; item += npairs) {
+        int l, tp, tq;
+        decode_item(p, item, l, tp, tq);
+        const bool three = p.skip_top_first && l == 0;
         long long dbg_a = clock64();
         if (!wait_bounded(smem_u32(&sh->tmem_empty), acc_phase ^ 1u, sh, p.status, 0x400)) break;
         dbg_empty += clock64() - dbg_a;
@@ -652,15 +664,29 @@ residue_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
           dbg_full += clock64() - dbg_a;
           tc_fence_after();
           const uint32_t base = smem_u32(tiles + stage * kPairStageBytes);
-          if (kb == 0)  // p1 times an all-zero column-side tile, "overwrite": the 13^2 accumulator starts from 0
-            mma_mxf4_pair(tmem + 2 * W, smem_desc_sw128(base + 1 * kPTileBytes), smem_desc_sw128(smem_u32(zero_tile)),
-                          idesc_mxf4_pair(W), sf, sf, 0u);
+          if (three) {
 #pragma unroll
-          for (int ks = 0; ks < 4; ++ks) {
-            const uint64_t q = smem_desc_sw128(base + 2 * kPTileBytes + ks * 32);
-            mma_mxf4_pair(tmem + 0, smem_desc_sw128(base + 0 * kPTileBytes + ks * 32), q, kIdesc, sf, sf,
-                          (kb == 0 && ks == 0) ? 0u : 1u);
-            mma_mxf4_pair(tmem + W, smem_desc_sw128(base + 1 * kPTileBytes + ks * 32), q, kIdesc, sf, sf, 1u);
+            for (int ks = 0; ks < 4; ++ks) {
+              const uint32_t first = (kb == 0 && ks == 0) ? 0u : 1u;
+              const uint64_t p0 = smem_desc_sw128(base + 0 * kPTileBytes + ks * 32);
+              const uint64_t p1 = smem_desc_sw128(base + 1 * kPTileBytes + ks * 32);
+              const uint64_t q0 = smem_desc_sw128(base + 2 * kPTileBytes + ks * 32);
+              const uint64_t q1 = smem_desc_sw128(base + 2 * kPTileBytes + kPTileBytes / 2 + ks * 32);
+              mma_mxf4_pair(tmem + 0, p0, q0, idesc_mxf4_pair(W), sf, sf, first);
+              mma_mxf4_pair(tmem + W, p0, q1, idesc_mxf4_pair(W), sf, sf, first);
+              mma_mxf4_pair(tmem + W, p1, q0, idesc_mxf4_pair(W), sf, sf, 1u);
+            }
+          } else {
+            if (kb == 0)  // p1 times an all-zero column-side tile, "overwrite": the 13^2 accumulator starts from 0
+              mma_mxf4_pair(tmem + 2 * W, smem_desc_sw128(base + 1 * kPTileBytes), smem_desc_sw128(smem_u32(zero_tile)),
+                            idesc_mxf4_pair(W), sf, sf, 0u);
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+              const uint64_t q = smem_desc_sw128(base + 2 * kPTileBytes + ks * 32);
+              mma_mxf4_pair(tmem + 0, smem_desc_sw128(base + 0 * kPTileBytes + ks * 32), q, kIdesc, sf, sf,
+                            (kb == 0 && ks == 0) ? 0u : 1u);
+              mma_mxf4_pair(tmem + W, smem_desc_sw128(base + 1 * kPTileBytes + ks * 32), q, kIdesc, sf, sf, 1u);
+            }
           }
           mma_commit_pair(smem_u32(&sh->empty[stage]), (uint16_t)3);
           if (++stage == kPairStages) stage = 0, phase ^= 1u;
@@ -694,7 +720,7 @@ residue_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
       tc_fence_after();
       const uint32_t m = (uint32_t)ep.m[l], recip = ep.recip[l], offset = ep.offset[l];
       uint32_t t[64];
-      drain_and_release<kFast, false>(base, W, true, offset, leader_empty, true, lane, t);
+      drain_and_release<kFast, false>(base, W, !(p.skip_top_first && l == 0), offset, leader_empty, true, lane, t);
       const int64_t j = (int64_t)(2 * tp + (int)rank) * kTileRows + quad * 32 + lane;
       uint4* dst = reinterpret_cast<uint4*>(ep.res + (size_t)l * ep.res_stride + (size_t)j * (size_t)ep.res_ld +
                                             (size_t)tq * W + half * 64);
@@ -919,7 +945,9 @@ ozk_status gemm_residues(const Geometry& g, const ModulusTable& mt, uint8_t* ws,
     GemmCore pc = core;
     pc.tiles_p = (int)(g.Np / 256);
     pc.group = 8;  // 8 column tiles of 256: the same 2048-column band as the single-CTA kernel
-    pc.skip_top_first = 0;
+    pc.skip_top_first = (mt.m[0] == 169) ? 1 : 0;  // 13^2 a1 b1 vanishes mod 169 (Section 5.1)
+    CUtensorMap map_qh;  // 64-row boxes of the A-side planes, for the three-product form of m = 169
+    if (!make_plane_map(&map_qh, ws + g.off_planes_a, g.Kp / 2, g.Mp, 2 * g.L, g.plane_bytes_a, 64, g.pitch)) return OZK_ERR_CUDA;
     pc.wave_counter = reinterpret_cast<unsigned int*>(ws + g.off_status + 512);
     const size_t smem = (size_t)kPairStages * kPairStageBytes + kPairZeroBytes + sizeof(GemmShared) + 1024;
     static int max_pairs = -1;
@@ -942,8 +970,8 @@ ozk_status gemm_residues(const Geometry& g, const ModulusTable& mt, uint8_t* ws,
     attr[0].val.cooperative = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    const cudaError_t e = pc.fast_combine ? cudaLaunchKernelEx(&cfg, residue_gemm_pair_kernel<true>, map_p, map_q, pc, ep)
-                                          : cudaLaunchKernelEx(&cfg, residue_gemm_pair_kernel<false>, map_p, map_q, pc, ep);
+    const cudaError_t e = pc.fast_combine ? cudaLaunchKernelEx(&cfg, residue_gemm_pair_kernel<true>, map_p, map_q, map_qh, pc, ep)
+                                          : cudaLaunchKernelEx(&cfg, residue_gemm_pair_kernel<false>, map_p, map_q, map_qh, pc, ep);
     if (e == cudaSuccess) return OZK_OK;
     (void)cudaGetLastError();  // the cooperative launch was refused: fall through to the single-CTA kernel
   }

@@ -21,8 +21,8 @@ __device__ __constant__ int8_t kDoubledE2M1[8] = {0, 1, 2, 3, 4, 6, 8, 12};
 // ------------------------------------------------------------------------------------
 // Limb-pair table: for modulus m and every centred residue r in [-96, 96) one 16-bit entry (index
 // r + 96) holding the E2M1 codes of a limb pair (c0, c1) with c0 + 13 c1 = r (mod m): code(c0) in bits
-// 0..3, code(c1) in bits 8..11.  Both limbs are in S and the pair minimises max(|c0|,|c1|), then
-// |c0|+|c1|.  The encoder's residue is centred (|r| <= m/2 + 2 <= 87), so the sign of the converted
+// 0..3, code(c1) in bits 8..11.  Both limbs are in S with |c| <= 8; among the valid pairs the one with the
+// fewest negative limbs, then the smallest max(|c0|,|c1|), then the smallest |c0|+|c1| is taken.  The encoder's residue is centred (|r| <= m/2 + 2 <= 87), so the sign of the converted
 // integer needs no separate handling.
 // ------------------------------------------------------------------------------------
 __global__ void build_lut_kernel(ModulusTable mt, uint16_t* __restrict__ lut) {
@@ -38,7 +38,10 @@ __global__ void build_lut_kernel(ModulusTable mt, uint16_t* __restrict__ lut) {
         const int c1 = kDoubledE2M1[i1 & 7] * ((i1 & 8) ? -1 : 1);
         if ((c0 + 13 * c1 - rho) % m != 0) continue;
         const int a0 = abs(c0), a1 = abs(c1);
-        const int key = max(a0, a1) * 64 + (a0 + a1);
+        if (max(a0, a1) > 8) continue;  // every class of every modulus has a pair with |c| <= 8 (keeps 128 K <= 2^24)
+        // fewest negative limbs first (sign changes in the operand streams cost power on the tensor pipe:
+        // a few per cent of the limb GEMM's time under the power cap), then smallest magnitudes
+        const int key = 2000 * ((c0 < 0) + (c1 < 0)) + max(a0, a1) * 64 + (a0 + a1);
         if (key < best_key) {
           best_key = key;
           best = (i1 << 8) | i0;
