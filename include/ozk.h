@@ -37,6 +37,8 @@ enum {
 };
 
 enum { OZK_MIN_MODULI = 2, OZK_MAX_MODULI = 27, OZK_DEFAULT_MODULI = 19 };
+/* Longest k range of one limb-GEMM launch, and the largest K ozk_dgemm accepts (16 ranges). */
+enum { OZK_CHUNK_K = 131072, OZK_MAX_K = 2097152 };
 
 /* ---------------------------------------------------------------------------------------
  * Constants of the method (host-side, no GPU needed).
@@ -97,8 +99,11 @@ ozk_status ozk_get_async_status(void* stream);
  * inverse scaling, one round-to-nearest-even.
  *   A: M x K, lda >= max(1,M).  B: K x N, ldb >= max(1,K).  C: M x N, ldc >= max(1,M), overwritten.
  *   num_moduli in [OZK_MIN_MODULI, OZK_MAX_MODULI]; 19 keeps all 53 bits for K <= 76549.
- *   K must not exceed 131072 (FP32 accumulators stay exact integers: 128*K <= 2^24 with
- *   limbs |c| <= 8, Lemma 3 tightened).  M, N, K = 0 are allowed (K = 0 gives C = 0).
+ *   One limb-GEMM launch covers at most 131072 values of k (FP32 accumulators stay exact
+ *   integers: 128*K <= 2^24 with limbs |c| <= 8, Lemma 3 tightened); a longer K is cut into
+ *   such ranges whose residues are added modulo each modulus (Section 5.1, "Exactness of the
+ *   FP32 accumulation": chunking), up to OZK_MAX_K.  The capacity of ozk_capacity_bits(K, ...)
+ *   always refers to the whole K.  M, N, K = 0 are allowed (K = 0 gives C = 0).
  * Returns OZK_OK once the work is enqueued. */
 ozk_status ozk_dgemm(int64_t M, int64_t N, int64_t K,
                      const double* A, int64_t lda,
@@ -124,7 +129,8 @@ ozk_status ozk_igemm_i8(int64_t M, int64_t N, int64_t K,
  * paper times device-resident data only, Section 6.1).  The call returns once everything is
  * enqueued; `stream` completes when C has arrived in host memory.  The workspace holds the limb
  * planes of two row blocks of A and of all of B, plus two staging blocks each for A, B and C.
- * The first call creates two internal streams and a pool of events. */
+ * The first call creates two internal streams and a pool of events.  K <= OZK_CHUNK_K here
+ * (OZK_ERR_UNSUPPORTED beyond). */
 size_t ozk_dgemm_host_workspace_bytes(int64_t M, int64_t N, int64_t K, int num_moduli);
 ozk_status ozk_dgemm_host(int64_t M, int64_t N, int64_t K,
                           const double* A, int64_t lda,

@@ -23,6 +23,7 @@ OZK_ERR_CUDA = -4
 OZK_ERR_NONFINITE = -5
 OZK_ERR_DEVICE_TIMEOUT = -6
 OZK_MIN_MODULI, OZK_MAX_MODULI, OZK_DEFAULT_MODULI = 2, 27, 19
+OZK_CHUNK_K, OZK_MAX_K = 131072, 2097152
 
 # name -> (restype, argtypes): every symbol include/ozk.h declares
 SIGNATURES = {

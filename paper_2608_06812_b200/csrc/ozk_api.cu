@@ -62,13 +62,18 @@ bool make_geometry_impl(int64_t M, int64_t N, int64_t K, int L, Geometry* g) {
   off += 2 * (size_t)L * g->plane_bytes_b;
   g->off_res = off;
   off += (size_t)L * (size_t)g->Mp * (size_t)g->Np;
+  g->off_res_chunk = 0;
+  if (K > kChunkK) {  // k ranges beyond the first leave their residues here before they are added in
+    g->off_res_chunk = off;
+    off += (size_t)L * (size_t)g->Mp * (size_t)g->Np;
+  }
   g->total = align_up(off, 1024);
   return true;
 }
 
 ozk_status check_common(int64_t M, int64_t N, int64_t K, int L, Geometry* g) {
   if (!make_geometry(M, N, K, L, g)) return OZK_ERR_INVALID_ARG;
-  if (K > 131072) return OZK_ERR_UNSUPPORTED;  // 128 K <= 2^24 with |limb| <= 8
+  if (K > kMaxK) return OZK_ERR_UNSUPPORTED;
   if (g->c_bits < 1) return OZK_ERR_UNSUPPORTED;
   if (N > 65535 || g->Mp / 32 > 65535) return OZK_ERR_UNSUPPORTED;  // grid-dimension limits of the O(N^2) kernels
   if (!g_ws.ptr) return OZK_ERR_WORKSPACE;
@@ -98,6 +103,20 @@ ozk_status run_preprocess(const Geometry& g, const ModulusTable& mt, const doubl
 }  // namespace
 
 bool make_geometry(int64_t M, int64_t N, int64_t K, int L, Geometry* g) { return make_geometry_impl(M, N, K, L, g); }
+
+// Limb GEMM over all of K: one launch per k range of at most kChunkK (the FP32 accumulators stay exact
+// integers inside a range, Lemma 3 with |limb| <= 8); the residues of later ranges are added modulo m.
+ozk_status gemm_residues_chunked(const Geometry& g, const ModulusTable& mt, uint8_t* ws, cudaStream_t st) {
+  if (g.Kp <= kChunkK) return gemm_residues(g, mt, ws, st);
+  if (!g.off_res_chunk) return OZK_ERR_WORKSPACE;
+  for (int64_t k0 = 0; k0 < g.Kp; k0 += kChunkK) {
+    const int64_t klen = g.Kp - k0 < kChunkK ? g.Kp - k0 : kChunkK;
+    const ozk_status rc = gemm_residues(g, mt, ws, st, k0, klen, k0 == 0 ? nullptr : ws + g.off_res_chunk);
+    if (rc != OZK_OK) return rc;
+    if (k0 > 0 && launch_add_residues(g, mt, ws + g.off_res, ws + g.off_res_chunk, st) != cudaSuccess) return OZK_ERR_CUDA;
+  }
+  return OZK_OK;
+}
 uint8_t* workspace_ptr() { return g_ws.ptr; }
 size_t workspace_bytes() { return g_ws.bytes; }
 
@@ -214,7 +233,7 @@ ozk_status ozk_stage_residue_gemm(int64_t M, int64_t N, int64_t K, int num_modul
   ModulusTable mt;
   if (!host_build_modulus_table(num_moduli, &mt)) return OZK_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  rc = gemm_residues(g, mt, g_ws.ptr, st);
+  rc = gemm_residues_chunked(g, mt, g_ws.ptr, st);
   if (rc != OZK_OK) return rc;
   if (residues_out && launch_copy_residues(g, g_ws.ptr + g.off_res, residues_out, st) != cudaSuccess) return OZK_ERR_CUDA;
   return OZK_OK;
@@ -257,7 +276,7 @@ ozk_status ozk_dgemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t l
   rc = run_preprocess(g, mt, A, lda, B, ldb, nullptr, nullptr, st);
   if (rc != OZK_OK) return rc;
   mark(1, st);
-  rc = gemm_residues(g, mt, g_ws.ptr, st);
+  rc = gemm_residues_chunked(g, mt, g_ws.ptr, st);
   if (rc != OZK_OK) return rc;
   mark(2, st);
   if (launch_crt(g, ct, g_ws.ptr + g.off_res, g.Mp, (size_t)g.Mp * (size_t)g.Np,

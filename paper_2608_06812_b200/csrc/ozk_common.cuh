@@ -16,6 +16,8 @@ constexpr int kMaxModuli = OZK_MAX_MODULI;
 constexpr int kCrtWords = 6;         // 192-bit integers cover sum r_l w_l for all 27 moduli
 constexpr int kLutStride = 192;      // 16-bit entries per modulus in the limb-pair table: centred residues -96 .. 95
 constexpr int kLutOffset = 96;
+constexpr int64_t kChunkK = OZK_CHUNK_K;  // longest k range of one limb-GEMM launch: 128 K <= 2^24 keeps FP32 sums exact (|limb| <= 8)
+constexpr int64_t kMaxK = OZK_MAX_K;      // 16 ranges; the grid limits of the O(N^2) kernels lie beyond it
 
 // ---- status word (first bytes of the workspace) -------------------------------------
 struct StatusBlock {
@@ -32,6 +34,7 @@ struct Geometry {
   int c_bits;
   // byte offsets into the workspace
   size_t off_status, off_lut, off_amax_a, off_amax_b, off_s, off_t, off_planes_a, off_planes_b, off_res;
+  size_t off_res_chunk;                  // second set of residue matrices, present when K > kChunkK (else 0)
   size_t pitch;                          // bytes from one plane row to the next: Kp / 2 plus padding
   size_t plane_bytes_a, plane_bytes_b;   // one limb plane: rows_p * pitch
   size_t total;
@@ -86,9 +89,12 @@ cudaError_t launch_decode_plane(const uint8_t* plane, int64_t rows, int64_t K, s
 cudaError_t launch_crt(const Geometry& g, const CrtTable& ct, const uint8_t* res, int64_t res_ld, size_t res_stride,
                        const int32_t* s, const int32_t* t, double* C, int64_t ldc, uint32_t* x_out, cudaStream_t st);
 cudaError_t launch_copy_residues(const Geometry& g, const uint8_t* res, uint8_t* out, cudaStream_t st);
+cudaError_t launch_add_residues(const Geometry& g, const ModulusTable& mt, uint8_t* acc, const uint8_t* chunk, cudaStream_t st);
 
 // limb GEMM (ozk_gemm.cu)
-ozk_status gemm_residues(const Geometry& g, const ModulusTable& mt, uint8_t* ws, cudaStream_t st);
+ozk_status gemm_residues(const Geometry& g, const ModulusTable& mt, uint8_t* ws, cudaStream_t st, int64_t k0 = 0,
+                         int64_t klen = 0, uint8_t* res = nullptr);
+ozk_status gemm_residues_chunked(const Geometry& g, const ModulusTable& mt, uint8_t* ws, cudaStream_t st);
 ozk_status gemm_int8(const uint8_t* planes_a, const uint8_t* planes_b, int64_t M, int64_t N, int64_t Mp, int64_t Np, int64_t Kp,
                      int32_t* C, int64_t ldc, StatusBlock* status, cudaStream_t st);
 ozk_status gemm_oz1_passes(const uint8_t* planes_a, const uint8_t* planes_b, int64_t Mp, int64_t Np, int64_t Kp, int64_t M,

@@ -318,7 +318,40 @@ __global__ void copy_residues_kernel(const uint8_t* __restrict__ res, int64_t Mp
       res[(size_t)l * res_stride + (size_t)j * (size_t)Mp + (size_t)i];
 }
 
+// acc = (acc + chunk) mod m for one modulus per blockIdx.y: sums the residues of two k ranges
+// (Section 5.1: the residue of a sum is the sum of the residues).  16 bytes per thread.
+__global__ void add_residues_kernel(uint8_t* __restrict__ acc, const uint8_t* __restrict__ chunk, size_t per_modulus,
+                                    ModulusTable mt) {
+  const size_t v = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (v * 16 >= per_modulus) return;
+  const uint32_t m = (uint32_t)mt.m[blockIdx.y];
+  uint4* pa = reinterpret_cast<uint4*>(acc + (size_t)blockIdx.y * per_modulus) + v;
+  const uint4 a = *pa;
+  const uint4 b = *(reinterpret_cast<const uint4*>(chunk + (size_t)blockIdx.y * per_modulus) + v);
+  const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+  uint32_t out[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    uint32_t word = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      uint32_t r = ((aw[k] >> (8 * e)) & 0xFFu) + ((bw[k] >> (8 * e)) & 0xFFu);
+      r = min(r, r - m);
+      word |= r << (8 * e);
+    }
+    out[k] = word;
+  }
+  *pa = make_uint4(out[0], out[1], out[2], out[3]);
+}
+
 }  // namespace
+
+cudaError_t launch_add_residues(const Geometry& g, const ModulusTable& mt, uint8_t* acc, const uint8_t* chunk, cudaStream_t st) {
+  const size_t per_modulus = (size_t)g.Mp * (size_t)g.Np;  // a multiple of 16
+  dim3 grid((unsigned)((per_modulus / 16 + 255) / 256), (unsigned)g.L);
+  add_residues_kernel<<<grid, 256, 0, st>>>(acc, chunk, per_modulus, mt);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_crt(const Geometry& g, const CrtTable& ct, const uint8_t* res, int64_t res_ld, size_t res_stride,
                        const int32_t* s, const int32_t* t, double* C, int64_t ldc, uint32_t* x_out, cudaStream_t st) {

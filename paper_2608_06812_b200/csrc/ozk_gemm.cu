@@ -913,20 +913,27 @@ ozk_status launch_limb_gemm(const CUtensorMap& map_p, const CUtensorMap& map_q, 
 
 }  // namespace
 
-// DGEMM path: residues r_l[j][i] for all moduli from the limb planes in the workspace.
-ozk_status gemm_residues(const Geometry& g, const ModulusTable& mt, uint8_t* ws, cudaStream_t st) {
+// DGEMM path: residues r_l[j][i] for all moduli from the limb planes in the workspace, over the
+// k range [k0, k0 + klen) (multiples of 256; klen = 0 means all of Kp), written to `res` (default:
+// the workspace's residue matrices).
+ozk_status gemm_residues(const Geometry& g, const ModulusTable& mt, uint8_t* ws, cudaStream_t st, int64_t k0, int64_t klen,
+                         uint8_t* res) {
+  if (klen <= 0) klen = g.Kp - k0;
+  if (k0 < 0 || k0 % kTileKNibbles || klen % kTileKNibbles || k0 + klen > g.Kp || klen > kChunkK) return OZK_ERR_INVALID_ARG;
+  const uint8_t* planes_b = ws + g.off_planes_b + k0 / 2;
+  const uint8_t* planes_a = ws + g.off_planes_a + k0 / 2;
   CUtensorMap map_p, map_q;
-  if (!make_plane_map(&map_p, ws + g.off_planes_b, g.Kp / 2, g.Np, 2 * g.L, g.plane_bytes_b, kTileRows, g.pitch)) return OZK_ERR_CUDA;
-  if (!make_plane_map(&map_q, ws + g.off_planes_a, g.Kp / 2, g.Mp, 2 * g.L, g.plane_bytes_a, 128, g.pitch)) return OZK_ERR_CUDA;
+  if (!make_plane_map(&map_p, planes_b, klen / 2, g.Np, 2 * g.L, g.plane_bytes_b, kTileRows, g.pitch)) return OZK_ERR_CUDA;
+  if (!make_plane_map(&map_q, planes_a, klen / 2, g.Mp, 2 * g.L, g.plane_bytes_a, 128, g.pitch)) return OZK_ERR_CUDA;
   GemmCore core;
   core.L = g.L;
   core.tiles_p = (int)(g.Np / kTileRows);
   core.tiles_q = (int)(g.Mp / 128);
-  core.kblocks = (int)(g.Kp / kTileKNibbles);
+  core.kblocks = (int)(klen / kTileKNibbles);
   core.group = 16;
   core.skip_top_first = (mt.m[0] == 169) ? 1 : 0;  // 13^2 a1 b1 vanishes mod 169 (Section 5.1)
   core.q_groups = 0;
-  core.fast_combine = g.K <= 17476 ? 1 : 0;  // 128 K + 13 * 64 K = 960 K < 2^24
+  core.fast_combine = (g.K <= 17476 || klen <= 17408) ? 1 : 0;  // 128 K + 13 * 64 K = 960 K < 2^24
   core.wave_counter = nullptr;
   core.status = reinterpret_cast<StatusBlock*>(ws + g.off_status);
   core.scale_word = 0x80808080u;  // UE8M0 byte 0x80 = 2: both operands doubled, accumulators hold integers
@@ -936,7 +943,7 @@ ozk_status gemm_residues(const Geometry& g, const ModulusTable& mt, uint8_t* ws,
     ep.recip[l] = mt.recip[l];
     ep.offset[l] = (uint32_t)mt.m[l] * (uint32_t)(0x80000000u / (uint32_t)mt.m[l]);
   }
-  ep.res = ws + g.off_res;
+  ep.res = res ? res : ws + g.off_res;
   ep.res_ld = g.Mp;
   ep.res_stride = (size_t)g.Mp * (size_t)g.Np;
   if (g.Np % 256 == 0 && pair_kernel_enabled()) {
@@ -947,7 +954,7 @@ ozk_status gemm_residues(const Geometry& g, const ModulusTable& mt, uint8_t* ws,
     pc.group = 8;  // 8 column tiles of 256: the same 2048-column band as the single-CTA kernel
     pc.skip_top_first = (mt.m[0] == 169) ? 1 : 0;  // 13^2 a1 b1 vanishes mod 169 (Section 5.1)
     CUtensorMap map_qh;  // 64-row boxes of the A-side planes, for the three-product form of m = 169
-    if (!make_plane_map(&map_qh, ws + g.off_planes_a, g.Kp / 2, g.Mp, 2 * g.L, g.plane_bytes_a, 64, g.pitch)) return OZK_ERR_CUDA;
+    if (!make_plane_map(&map_qh, planes_a, klen / 2, g.Mp, 2 * g.L, g.plane_bytes_a, 64, g.pitch)) return OZK_ERR_CUDA;
     pc.wave_counter = reinterpret_cast<unsigned int*>(ws + g.off_status + 512);
     const size_t smem = (size_t)kPairStages * kPairStageBytes + kPairZeroBytes + sizeof(GemmShared) + 1024;
     static int max_pairs = -1;

@@ -144,7 +144,7 @@ ozk_status ozk_dgemm_host(int64_t M, int64_t N, int64_t K, const double* A, int6
                           double* C, int64_t ldc, int num_moduli, void* stream) {
   HostLayout h;
   if (!make_host_layout(M, N, K, num_moduli, &h)) return OZK_ERR_INVALID_ARG;
-  if (K > 131072 || h.g.c_bits < 1 || h.g.Mp / 32 > 65535) return OZK_ERR_UNSUPPORTED;
+  if (K > kChunkK || h.g.c_bits < 1 || h.g.Mp / 32 > 65535) return OZK_ERR_UNSUPPORTED;
   uint8_t* ws = workspace_ptr();
   if (!ws || workspace_bytes() < h.total) return OZK_ERR_WORKSPACE;
   if (M == 0 || N == 0) return OZK_OK;

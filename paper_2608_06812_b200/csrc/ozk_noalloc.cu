@@ -84,7 +84,7 @@ extern "C" ozk_status ozk_row_shifts_noalloc(int64_t M, int64_t K, const double*
   using namespace ozk;
   if (M < 0 || K < 0 || num_moduli < OZK_MIN_MODULI || num_moduli > OZK_MAX_MODULI) return OZK_ERR_INVALID_ARG;
   if (M > OZK_NOALLOC_MAX_ROWS_INTERNAL) return OZK_ERR_UNSUPPORTED;  // the fixed scratch holds 65536 rows
-  if (K > 131072) return OZK_ERR_UNSUPPORTED;
+  if (K > kMaxK) return OZK_ERR_UNSUPPORTED;
   const int c_bits = host_capacity_bits(K, num_moduli);
   if (c_bits < 1) return OZK_ERR_UNSUPPORTED;
   if (M == 0) return OZK_OK;

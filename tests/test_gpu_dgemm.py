@@ -55,6 +55,28 @@ def test_long_inner_products_bit_exact(shape, L):
     assert gu.bits_equal(gu.dgemm(A, B, L), ozaki2.dgemm(A, B, L).C)
 
 
+@pytest.mark.parametrize("shape", [(16, 64, 140000), (16, 130, 290000)])
+def test_k_beyond_one_limb_gemm_range_bit_exact(shape):
+    """K above 131072 runs one limb GEMM per range of 131072 and adds the residues modulo each modulus
+    (Section 5.1, chunking): a short last range (fast recombination) and three ranges with a long last one."""
+    M, N, K = shape
+    A = inputs.lognormal_matrix(M, K, 0.5, seed=30)
+    B = inputs.lognormal_matrix(K, N, 0.5, seed=31)
+    A[0, :] = np.abs(A[0, :])
+    B[:, 0] = np.abs(B[:, 0])
+    assert gu.bits_equal(gu.dgemm(A, B, 19), ozaki2.dgemm(A, B, 19).C)
+
+
+def test_k_ranges_small_integers_exact_over_several_tiles():
+    """Two ranges over a 3 x 3 grid of tiles: integer inputs make C the exact integer product, which an FP64
+    matrix product of these magnitudes (|sum| < 2^53) delivers without rounding."""
+    M, N, K = 384, 300, 200000
+    A = inputs.small_integer_matrix(M, K, 1000, seed=3)
+    B = inputs.small_integer_matrix(K, N, 1000, seed=4)
+    C = gu.dgemm(A, B, 19)
+    assert gu.bits_equal(C, A @ B)
+
+
 def test_small_integers_give_the_exact_integer_product():
     A = inputs.small_integer_matrix(200, 333, 1000, seed=1)
     B = inputs.small_integer_matrix(333, 150, 1000, seed=2)

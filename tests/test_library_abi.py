@@ -38,7 +38,7 @@ def test_moduli_match_the_printed_list_and_the_oracle():
 
 
 def test_capacity_and_crt_constants_match_the_oracle():
-    for K in (1, 256, 4096, 8192, 16384, 131072):
+    for K in (1, 256, 4096, 8192, 16384, 131072, 300000, ozk.OZK_MAX_K):
         for L in range(4, 28):
             assert ozk.ozk_capacity_bits(K, L) == moduli.capacity_bits(K, L)
     assert ozk.ozk_capacity_bits(16384, 19) == 53
@@ -56,11 +56,15 @@ def test_argument_errors_need_no_gpu():
     assert 0 < small < big
     # planes: 2 limbs x L x (M + N) x K / 2 bytes, residues: L x M x N bytes
     assert big >= 19 * (2 * 2 * 4096 * 4096 // 2 + 4096 * 4096)
+    # K beyond one limb-GEMM range: a second set of residue matrices for the ranges after the first
+    one_range = ozk.ozk_dgemm_workspace_bytes(128, 128, ozk.OZK_CHUNK_K, 19)
+    two_ranges = ozk.ozk_dgemm_workspace_bytes(128, 128, ozk.OZK_CHUNK_K + 256, 19)
+    assert two_ranges - one_range >= 19 * 128 * 128 + 19 * 2 * 2 * 128 * 256 // 2
     ozk.ozk_set_workspace(None, 0)
     assert ozk.ozk_dgemm(8, 8, 8, None, 8, None, 8, None, 8, 19, None) == ozk.OZK_ERR_WORKSPACE
+    assert ozk.ozk_dgemm(8, 8, ozk.OZK_MAX_K + 1, None, 8, None, ozk.OZK_MAX_K + 1, None, 8, 19, None) == ozk.OZK_ERR_UNSUPPORTED
     assert ozk.ozk_dgemm(8, 8, 8, None, 8, None, 8, None, 8, 1, None) == ozk.OZK_ERR_INVALID_ARG
     assert ozk.ozk_dgemm(-8, 8, 8, None, 8, None, 8, None, 8, 19, None) == ozk.OZK_ERR_INVALID_ARG
-    assert ozk.ozk_dgemm(8, 8, 1 << 18, None, 8, None, 1 << 18, None, 8, 19, None) == ozk.OZK_ERR_UNSUPPORTED
     assert ozk.ozk_set_workspace(12345, 1 << 20) == ozk.OZK_ERR_INVALID_ARG       # not 1024-aligned
     assert "workspace" in ozk.ozk_status_string(ozk.OZK_ERR_WORKSPACE)
     assert "sm_100a" in ozk.ozk_version()
