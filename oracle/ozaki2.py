@@ -66,8 +66,10 @@ def round_half_even_scaled(x: float, s: int) -> int:
 def to_integers(A: np.ndarray, shifts: np.ndarray, axis: int) -> np.ndarray:
     """Section 4.2: A~ = round(A * 2^s) with one shift per row (axis=1) or per
     column (axis=0), as int64.  np.ldexp is an exact exponent shift here
-    (|A * 2^s| < 2^53, and a result too small to be normal rounds to 0 either
-    way); np.rint rounds half to even."""
+    (|A * 2^s| <= 2^53, or < 2^62 in the extended-capacity mode of dgemm, both
+    far inside the FP64 range; a result too small to be normal rounds to 0
+    either way); np.rint rounds half to even and leaves values of 2^52 and
+    above, which are integers already, unchanged."""
     sh = shifts.astype(np.int64)
     sh = sh[:, None] if axis == 1 else sh[None, :]
     scaled = np.ldexp(A, sh.astype(np.int32) if np.all(np.abs(sh) < 2 ** 31) else sh)
@@ -176,15 +178,27 @@ class Ozaki2Result:
     x: np.ndarray = field(repr=False, default=None)
 
 
-def dgemm(A: np.ndarray, B: np.ndarray, num_moduli: int = 19) -> Ozaki2Result:
-    """Emulated C = fl(AB) by Ozaki scheme II on base-13 limbs."""
+MAX_EXTENDED_BITS = 62
+
+
+def dgemm(A: np.ndarray, B: np.ndarray, num_moduli: int = 19, max_bits: int = 53) -> Ozaki2Result:
+    """Emulated C = fl(AB) by Ozaki scheme II on base-13 limbs.
+
+    max_bits = 53 is the paper's method (Section 4.2 caps the integer width at
+    53 bits).  A larger max_bits (up to 62) is an EXTENSION the paper does not
+    have: the same steps with the cap of the width c lifted, so that with more
+    than 19 moduli Eq. 3 admits wider integers; the row or column maximum then
+    converts without rounding and smaller entries keep up to max_bits - 53 more
+    bits below it."""
+    if not 1 <= max_bits <= MAX_EXTENDED_BITS:
+        raise ValueError("max_bits must lie in 1..62 (converted integers are held in int64)")
     A = np.asarray(A, dtype=np.float64)
     B = np.asarray(B, dtype=np.float64)
     M, K = A.shape
     K2, N = B.shape
     assert K == K2
     moduli = select_moduli(num_moduli)
-    c = capacity_bits(max(K, 1), num_moduli)
+    c = capacity_bits(max(K, 1), num_moduli, cap=max_bits)
     s = shared_shifts(A, axis=1, c=c)
     t = shared_shifts(B, axis=0, c=c)
     At = to_integers(A, s, axis=1)

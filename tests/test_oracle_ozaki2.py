@@ -234,6 +234,53 @@ def test_config1_law_error_levels():
     assert errs[14] > errs[17] >= errs[19] * 0.999
 
 
+# ---- extended capacity (not in the paper: the 53-bit cap of Section 4.2 lifted) -------------------
+@pytest.mark.parametrize("L,max_bits", [(20, 56), (22, 62), (27, 62)])
+def test_extended_capacity_brute_force_tiny(L, max_bits):
+    """Same pins as the paper's mode: x is the exact integer product of the converted inputs, C its
+    single rounding; the width follows Eq. 3 with the new cap; entries within 2^(c-53) of their row
+    or column maximum convert without any rounding."""
+    rng = np.random.default_rng(7 * L + max_bits)
+    for (M, N, K) in [(1, 1, 1), (3, 2, 5), (8, 8, 8)]:
+        A = (rng.random((M, K)) - 0.5) * np.exp(2.0 * rng.standard_normal((M, K)))
+        B = (rng.random((K, N)) - 0.5) * np.exp(2.0 * rng.standard_normal((K, N)))
+        r = ozaki2.dgemm(A, B, L, max_bits=max_bits)
+        assert r.c_bits == moduli.capacity_bits(K, L, cap=max_bits) and 53 < r.c_bits <= max_bits
+        assert np.max(np.abs(r.At)) < 2 ** r.c_bits and np.max(np.abs(r.Bt)) < 2 ** r.c_bits
+        for i in range(M):
+            for k in range(K):
+                want = Fraction(float(A[i, k])) * Fraction(2) ** int(r.s[i])
+                if abs(A[i, k]) * 2.0 ** (r.c_bits - 53) >= np.max(np.abs(A[i])):
+                    assert Fraction(int(r.At[i, k])) == want          # no rounding near the maximum
+                else:
+                    assert abs(Fraction(int(r.At[i, k])) - want) <= Fraction(1, 2)
+            for j in range(N):
+                tot = sum(int(r.At[i, k]) * int(r.Bt[k, j]) for k in range(K))
+                assert int(r.x[i, j]) == tot
+                assert r.C[i, j] == float(Fraction(tot) / Fraction(2) ** int(r.s[i] + r.t[j]))
+
+
+def test_extended_capacity_default_is_the_papers_mode_and_range_is_checked():
+    A = inputs.lognormal_matrix(5, 40, 1.0, seed=3)
+    B = inputs.lognormal_matrix(40, 4, 1.0, seed=4)
+    assert np.array_equal(ozaki2.dgemm(A, B, 22).C, ozaki2.dgemm(A, B, 22, max_bits=53).C)
+    assert moduli.capacity_bits(16384, 19, cap=62) == 54 and moduli.capacity_bits(16384, 22, cap=62) == 62   # Eq. 3 still limits c
+    with pytest.raises(ValueError):
+        ozaki2.dgemm(A, B, 22, max_bits=63)
+
+
+def test_extended_capacity_recovers_bits_on_wide_exponent_ranges():
+    """At phi = 4 the paper's mode saturates at L = 19 (53-bit cap); each further modulus of the
+    extended mode keeps about three more bits of the small entries."""
+    A = inputs.lognormal_matrix(16, 512, 4.0, seed=0)
+    B = inputs.lognormal_matrix(512, 16, 4.0, seed=1)
+    err = {(L, mb): exact.normwise_error(ozaki2.dgemm(A, B, L, max_bits=mb).C, A, B, against_rounded=True)
+           for (L, mb) in [(19, 53), (22, 53), (20, 62), (21, 62), (22, 62)]}
+    assert err[(22, 53)] == err[(19, 53)]
+    assert err[(20, 62)] < err[(19, 53)] / 16 and err[(21, 62)] < err[(20, 62)] / 2   # c = 59, then 62
+    assert err[(22, 62)] == err[(21, 62)]                                             # the int64 cap
+
+
 # ---- scheme I (Section 4) ---------------------------------------------------------------------
 def test_scheme1_equals_integer_product_and_scheme2_bit_for_bit():
     """Section 7.1: both schemes compute the exact product of the same converted integers and round
