@@ -48,6 +48,8 @@ def parse_args():
                     "metric is quoted on the square default)")
     ap.add_argument("--moduli", type=int, default=19)
     ap.add_argument("--phi", type=float, default=1.0)
+    ap.add_argument("--max-bits", type=int, default=53, help="width cap of the converted integers; values above 53 time the "
+                    "extended-capacity entry point ozk_dgemm_ext (not the paper's method, not the headline)")
     ap.add_argument("--impl", default="ozk", choices=["ozk", "reference"])
     ap.add_argument("--scheme", default="oz2", choices=["oz2", "oz1", "i8"],
                     help="oz2 = Ozaki scheme II (the headline path); oz1 = Ozaki scheme I, 15 x 15 limbs; "
@@ -270,6 +272,9 @@ def run_ozk(args, rank: int, local_rank: int, world: int) -> None:
     def step():
         if oz1:
             ozk.check(ozk.ozk_dgemm_oz1(M, N, K, dA.data_ptr(), M, dB.data_ptr(), K, dC.data_ptr(), M, stream), "ozk_dgemm_oz1")
+        elif args.max_bits != 53:
+            ozk.check(ozk.ozk_dgemm_ext(M, N, K, dA.data_ptr(), M, dB.data_ptr(), K, dC.data_ptr(), M, L, args.max_bits, stream),
+                      "ozk_dgemm_ext")
         else:
             ozk.check(ozk.ozk_dgemm(M, N, K, dA.data_ptr(), M, dB.data_ptr(), K, dC.data_ptr(), M, L, stream), "ozk_dgemm")
 
@@ -309,7 +314,7 @@ def run_ozk(args, rank: int, local_rank: int, world: int) -> None:
 
     # ---- end to end with host buffers -----------------------------------------------------
     e2e = None
-    if not args.no_e2e and not (not oz1 and K > ozk.OZK_CHUNK_K):   # the host-buffer entry point takes one k range
+    if not args.no_e2e and not (not oz1 and (K > ozk.OZK_CHUNK_K or args.max_bits != 53)):   # the host-buffer entry point takes one k range
         # the library's host-buffer entry point: A and B start in pinned host memory, C ends there; the copies
         # are inside the timed region (and overlap the stages inside the library)
         host_ws = ozk.ozk_dgemm_host_workspace_bytes(M, N, K, L) if not oz1 else 0
@@ -376,10 +381,11 @@ def run_ozk(args, rank: int, local_rank: int, world: int) -> None:
               "hbm_peak_gbs": peaks["hbm_gbs"], "per_step_ms": per_step}
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": ms_max, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": (value / world / PAPER_TOTAL_TFLOPS[n]) if (n in PAPER_TOTAL_TFLOPS and L == 19) else None,
+            "vs_baseline": (value / world / PAPER_TOTAL_TFLOPS[n]) if (n in PAPER_TOTAL_TFLOPS and L == 19 and args.max_bits == 53) else None,
             "dtype": "fp4_e2m1 (fp32 accumulate, integer CRT)", "data": "synthetic",
             "config": {"workload": workload_name(n, L, args.phi, shape), "l2": "inputs (%.2f + %.2f GiB) %s" % (M * K * 8 / 2 ** 30, K * N * 8 / 2 ** 30, "larger than L2" if (M * K + K * N) * 8 > (126 << 20) else "fit L2: not a valid timing size"),
-                       "parallelism": "replicas" if world > 1 else "single GPU", "moduli": L},
+                       "parallelism": "replicas" if world > 1 else "single GPU", "moduli": L,
+                       "integer_bits": ozk.ozk_capacity_bits_ext(K, L, args.max_bits)},
             "clocks": clocks, "e2e": e2e, "gpu_launches": (KERNELS_PER_STEP + 2 * (k_ranges - 1)) * args.steps, "roofline": roofline, "stages": stages}
 
     if not args.no_fp64_context:

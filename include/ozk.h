@@ -111,6 +111,22 @@ ozk_status ozk_dgemm(int64_t M, int64_t N, int64_t K,
                      double* C, int64_t ldc,
                      int num_moduli, void* stream);
 
+/* EXTENSION, not in the paper: ozk_dgemm with the 53-bit cap on the converted integers
+ * (Section 4.2) lifted to max_bits, 1 <= max_bits <= OZK_MAX_EXTENDED_BITS.  Every step is the
+ * paper's; only the width is c = min(max_bits, largest c with 2 K 2^(2c) < P) (Eq. 3), so
+ * with more than 19 moduli the row / column maximum converts without rounding and smaller
+ * entries keep up to max_bits - 53 more bits below it (converted integers are held in 64-bit
+ * words).  max_bits = 53 is ozk_dgemm itself.  Same arguments, workspace
+ * (ozk_dgemm_workspace_bytes), layout, asynchrony and error behaviour as ozk_dgemm;
+ * max_bits out of range -> OZK_ERR_INVALID_ARG.  ozk_capacity_bits_ext returns the width used. */
+enum { OZK_MAX_EXTENDED_BITS = 62 };
+int ozk_capacity_bits_ext(int64_t K, int num_moduli, int max_bits);
+ozk_status ozk_dgemm_ext(int64_t M, int64_t N, int64_t K,
+                         const double* A, int64_t lda,
+                         const double* B, int64_t ldb,
+                         double* C, int64_t ldc,
+                         int num_moduli, int max_bits, void* stream);
+
 /* Bit-exact INT8 x INT8 -> INT32 GEMM on FP4 tensor cores (Section 3, last paragraph;
  * Eq. 1 with p = q = 3): every int8 becomes three greedy base-13 limbs, nine limb
  * products are accumulated in five groups i+j = g and combined as sum_g 13^g G_g.

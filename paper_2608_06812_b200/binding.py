@@ -24,6 +24,7 @@ OZK_ERR_NONFINITE = -5
 OZK_ERR_DEVICE_TIMEOUT = -6
 OZK_MIN_MODULI, OZK_MAX_MODULI, OZK_DEFAULT_MODULI = 2, 27, 19
 OZK_CHUNK_K, OZK_MAX_K = 131072, 2097152
+OZK_MAX_EXTENDED_BITS = 62
 
 # name -> (restype, argtypes): every symbol include/ozk.h declares
 SIGNATURES = {
@@ -37,6 +38,8 @@ SIGNATURES = {
     "ozk_set_workspace": (c_int, [c_void_p, c_size_t]),
     "ozk_get_async_status": (c_int, [c_void_p]),
     "ozk_dgemm": (c_int, [c_int64, c_int64, c_int64, c_void_p, c_int64, c_void_p, c_int64, c_void_p, c_int64, c_int, c_void_p]),
+    "ozk_capacity_bits_ext": (c_int, [c_int64, c_int, c_int]),
+    "ozk_dgemm_ext": (c_int, [c_int64, c_int64, c_int64, c_void_p, c_int64, c_void_p, c_int64, c_void_p, c_int64, c_int, c_int, c_void_p]),
     "ozk_igemm_i8": (c_int, [c_int64, c_int64, c_int64, c_void_p, c_int64, c_void_p, c_int64, c_void_p, c_int64, c_void_p]),
     "ozk_dgemm_host_workspace_bytes": (c_size_t, [c_int64, c_int64, c_int64, c_int]),
     "ozk_dgemm_host": (c_int, [c_int64, c_int64, c_int64, c_void_p, c_int64, c_void_p, c_int64, c_void_p, c_int64, c_int, c_void_p]),
@@ -102,6 +105,10 @@ def ozk_capacity_bits(K: int, num_moduli: int) -> int:
     return lib().ozk_capacity_bits(K, num_moduli)
 
 
+def ozk_capacity_bits_ext(K: int, num_moduli: int, max_bits: int) -> int:
+    return lib().ozk_capacity_bits_ext(K, num_moduli, max_bits)
+
+
 def ozk_get_crt_constants(num_moduli: int) -> tuple[int, list[int]]:
     """P and the weights w_l as Python integers."""
     P = (ctypes.c_uint32 * 6)()
@@ -129,6 +136,10 @@ def ozk_get_async_status(stream: int = 0) -> int:
 
 def ozk_dgemm(M, N, K, A, lda, B, ldb, C, ldc, num_moduli, stream=0) -> int:
     return lib().ozk_dgemm(M, N, K, A, lda, B, ldb, C, ldc, num_moduli, stream)
+
+
+def ozk_dgemm_ext(M, N, K, A, lda, B, ldb, C, ldc, num_moduli, max_bits, stream=0) -> int:
+    return lib().ozk_dgemm_ext(M, N, K, A, lda, B, ldb, C, ldc, num_moduli, max_bits, stream)
 
 
 def ozk_igemm_i8(M, N, K, A, lda, B, ldb, C, ldc, stream=0) -> int:

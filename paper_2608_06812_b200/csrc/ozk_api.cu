@@ -28,8 +28,9 @@ void mark(int i, cudaStream_t st) {
 }
 
 // Workspace layout for an (M, N, K, L) problem.  Returns false on invalid sizes.
-bool make_geometry_impl(int64_t M, int64_t N, int64_t K, int L, Geometry* g) {
+bool make_geometry_impl(int64_t M, int64_t N, int64_t K, int L, Geometry* g, int max_bits) {
   if (M < 0 || N < 0 || K < 0 || L < OZK_MIN_MODULI || L > OZK_MAX_MODULI) return false;
+  if (max_bits < 1 || max_bits > OZK_MAX_EXTENDED_BITS) return false;
   memset(g, 0, sizeof *g);
   g->M = M;
   g->N = N;
@@ -38,7 +39,7 @@ bool make_geometry_impl(int64_t M, int64_t N, int64_t K, int L, Geometry* g) {
   g->Mp = round_up(M > 0 ? M : 1, kTileRows);
   g->Np = round_up(N > 0 ? N : 1, kTileRows);
   g->Kp = round_up(K > 0 ? K : 1, kTileKNibbles);
-  g->c_bits = host_capacity_bits(K, L);
+  g->c_bits = host_capacity_bits(K, L, max_bits);
   size_t off = 0;
   g->off_status = off;
   off += align_up(sizeof(StatusBlock), 1024);
@@ -71,8 +72,8 @@ bool make_geometry_impl(int64_t M, int64_t N, int64_t K, int L, Geometry* g) {
   return true;
 }
 
-ozk_status check_common(int64_t M, int64_t N, int64_t K, int L, Geometry* g) {
-  if (!make_geometry(M, N, K, L, g)) return OZK_ERR_INVALID_ARG;
+ozk_status check_common(int64_t M, int64_t N, int64_t K, int L, Geometry* g, int max_bits = 53) {
+  if (!make_geometry(M, N, K, L, g, max_bits)) return OZK_ERR_INVALID_ARG;
   if (K > kMaxK) return OZK_ERR_UNSUPPORTED;
   if (g->c_bits < 1) return OZK_ERR_UNSUPPORTED;
   if (N > 65535 || g->Mp / 32 > 65535) return OZK_ERR_UNSUPPORTED;  // grid-dimension limits of the O(N^2) kernels
@@ -102,7 +103,9 @@ ozk_status run_preprocess(const Geometry& g, const ModulusTable& mt, const doubl
 
 }  // namespace
 
-bool make_geometry(int64_t M, int64_t N, int64_t K, int L, Geometry* g) { return make_geometry_impl(M, N, K, L, g); }
+bool make_geometry(int64_t M, int64_t N, int64_t K, int L, Geometry* g, int max_bits) {
+  return make_geometry_impl(M, N, K, L, g, max_bits);
+}
 
 // Limb GEMM over all of K: one launch per k range of at most kChunkK (the FP32 accumulators stay exact
 // integers inside a range, Lemma 3 with |limb| <= 8); the residues of later ranges are added modulo m.
@@ -131,11 +134,14 @@ int ozk_get_moduli(int num_moduli, int* out) {
   return host_select_moduli(num_moduli, out) == num_moduli ? num_moduli : OZK_ERR_INVALID_ARG;
 }
 
-int ozk_capacity_bits(int64_t K, int num_moduli) {
-  if (K < 0 || num_moduli < 1 || num_moduli > OZK_MAX_MODULI) return OZK_ERR_INVALID_ARG;
-  const int c = host_capacity_bits(K, num_moduli);
+int ozk_capacity_bits_ext(int64_t K, int num_moduli, int max_bits) {
+  if (K < 0 || num_moduli < 1 || num_moduli > OZK_MAX_MODULI || max_bits < 1 || max_bits > OZK_MAX_EXTENDED_BITS)
+    return OZK_ERR_INVALID_ARG;
+  const int c = host_capacity_bits(K, num_moduli, max_bits);
   return c >= 1 ? c : OZK_ERR_UNSUPPORTED;
 }
+
+int ozk_capacity_bits(int64_t K, int num_moduli) { return ozk_capacity_bits_ext(K, num_moduli, 53); }
 
 ozk_status ozk_get_crt_constants(int num_moduli, uint32_t* P_words, uint32_t* weights) {
   CrtTable ct;
@@ -262,8 +268,13 @@ ozk_status ozk_stage_crt(int64_t M, int64_t N, int64_t K, int num_moduli, const 
 
 ozk_status ozk_dgemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, const double* B, int64_t ldb, double* C,
                      int64_t ldc, int num_moduli, void* stream) {
+  return ozk_dgemm_ext(M, N, K, A, lda, B, ldb, C, ldc, num_moduli, 53, stream);
+}
+
+ozk_status ozk_dgemm_ext(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, const double* B, int64_t ldb,
+                         double* C, int64_t ldc, int num_moduli, int max_bits, void* stream) {
   Geometry g;
-  ozk_status rc = check_common(M, N, K, num_moduli, &g);
+  ozk_status rc = check_common(M, N, K, num_moduli, &g, max_bits);
   if (rc != OZK_OK) return rc;
   if (M == 0 || N == 0) return OZK_OK;
   if (!C || ldc < M || (K > 0 && (!A || !B)) || lda < (M > 1 ? M : 1) || ldb < (K > 1 ? K : 1)) return OZK_ERR_INVALID_ARG;

@@ -49,6 +49,7 @@ struct ModulusTable {
   uint32_t recip[kMaxModuli];      // floor(2^32 / m)
   // encoder constants (FP32 arithmetic on exact small integers): centred residues of 2^14, 2^28, 2^42
   float c14[kMaxModuli], c28[kMaxModuli], c42[kMaxModuli];
+  float c56[kMaxModuli];           // centred residue of 2^56: fifth piece of integers wider than 56 bits
   float inv_m[kMaxModuli];         // 1 / m rounded to FP32
   float m_f[kMaxModuli];           // m
 };
@@ -68,11 +69,11 @@ struct CrtTable {
 // registered workspace and layout (ozk_api.cu)
 uint8_t* workspace_ptr();
 size_t workspace_bytes();
-bool make_geometry(int64_t M, int64_t N, int64_t K, int L, Geometry* g);
+bool make_geometry(int64_t M, int64_t N, int64_t K, int L, Geometry* g, int max_bits = 53);
 
 // host-side constant builders (ozk_tables.cu)
 int host_select_moduli(int count, int* out);
-int host_capacity_bits(int64_t K, int L);
+int host_capacity_bits(int64_t K, int L, int max_bits = 53);
 bool host_build_modulus_table(int L, ModulusTable* t);
 bool host_build_crt_table(int L, CrtTable* t);
 

@@ -7,7 +7,8 @@
 
 namespace ozk {
 
-// Returns the magnitude of round(x * 2^s) (at most 2^53 when |x| is at most its row or column maximum);
+// Returns the magnitude of round(x * 2^s): at most 2^c when |x| is at most its row or column maximum and s the
+// shift for a width of c <= 62 bits (c > 53 only in the extended-capacity mode);
 // *neg receives the sign of x.
 __device__ __forceinline__ unsigned long long to_integer_magnitude(double x, int s, bool* neg) {
   const unsigned long long bits = (unsigned long long)__double_as_longlong(x);
@@ -17,7 +18,7 @@ __device__ __forceinline__ unsigned long long to_integer_magnitude(double x, int
   if (E) mant |= 1ull << 52;
   if (mant == 0) return 0;
   const int sh = (E ? E : 1) - 1075 + s;  // x * 2^s = mant * 2^sh
-  if (sh >= 0) return sh > 52 ? 0 : mant << sh;  // sh > 0 only for subnormal x; |x 2^s| < 2^53 bounds it by 52
+  if (sh >= 0) return sh > 62 ? 0 : mant << sh;  // |x 2^s| <= 2^62 keeps the shifted significand inside 64 bits
   const int d = -sh;
   if (d > 54) return 0;
   const unsigned long long q = mant >> d;

@@ -116,31 +116,41 @@ __global__ void finalize_shifts_kernel(const unsigned long long* __restrict__ am
   shifts[i] = s;
 }
 
-// Eight consecutive-k integers of one plane row as four signed 14-bit pieces each, held in FP32
-// (a = x3 2^42 + x2 2^28 + x1 2^14 + x0, every piece carrying the sign of a).
+// Eight consecutive-k integers of one plane row as signed 14-bit pieces, held in FP32
+// (a = x3 2^42 + x2 2^28 + x1 2^14 + x0, every piece carrying the sign of a).  Integers of up to 56 bits
+// need four pieces; kWide adds x4 2^56 for the extended-capacity mode (up to 62 bits).
+template <bool kWide>
 struct Piece8 {
-  float x0[8], x1[8], x2[8], x3[8];
+  float x0[8], x1[8], x2[8], x3[8], x4[kWide ? 8 : 1];
 };
 
-__device__ __forceinline__ void split8(const unsigned long long (&mag)[8], const bool (&neg)[8], Piece8& p) {
+template <bool kWide>
+__device__ __forceinline__ void split8(const unsigned long long (&mag)[8], const bool (&neg)[8], Piece8<kWide>& p) {
 #pragma unroll
   for (int e = 0; e < 8; ++e) {
     const float sgn = neg[e] ? -1.0f : 1.0f;
     p.x0[e] = sgn * (float)(uint32_t)(mag[e] & 0x3FFFull);
     p.x1[e] = sgn * (float)(uint32_t)((mag[e] >> 14) & 0x3FFFull);
     p.x2[e] = sgn * (float)(uint32_t)((mag[e] >> 28) & 0x3FFFull);
-    p.x3[e] = sgn * (float)(uint32_t)(mag[e] >> 42);  // <= 2^11
+    if (kWide) {
+      p.x3[e] = sgn * (float)(uint32_t)((mag[e] >> 42) & 0x3FFFull);
+      p.x4[e] = sgn * (float)(uint32_t)(mag[e] >> 56);  // <= 2^6
+    } else {
+      p.x3[e] = sgn * (float)(uint32_t)(mag[e] >> 42);  // < 2^14
+    }
   }
 }
 
 // Residues of the eight values mod m_l and their limb codes packed as 8 nibbles per limb, on the FP32
 // pipe (the integer pipes of this GPU run at half its rate).  All quantities are small exact integers:
-//   t = x0 + x1 c14 + x2 c28 + x3 c42       |t| < 2^22   (c = centred residues of 2^14, 2^28, 2^42)
+//   t = x0 + x1 c14 + x2 c28 + x3 c42 (+ x4 c56)   |t| < 2^22   (c = centred residues of 2^14, 2^28, ...;
+//                                                  |c| <= 84: 16383 (1 + 3 * 84) + 63 * 84 < 2^22)
 //   q = round(t / m) by the add-2^23 trick,  r = t - q m   centred residue, |r| <= m/2 + 2
 //   byte offset of the table entry = 2 (r + 96), read from the low bits of 2 r + 192 + 1.5 * 2^23
 // Two neighbouring k share a byte: entry(even k) | entry(odd k) << 4 has the byte of limb 0 in bits
 // 0..7 and the byte of limb 1 in bits 8..15.
-__device__ __forceinline__ void encode8(const Piece8& p, float c14, float c28, float c42, float inv_m, float m_f,
+template <bool kWide>
+__device__ __forceinline__ void encode8(const Piece8<kWide>& p, float c14, float c28, float c42, float c56, float inv_m, float m_f,
                                         const uint16_t* __restrict__ lut_l, uint32_t& w0, uint32_t& w1) {
   constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23: adding it rounds to an integer in the low mantissa bits
   const char* lut_bytes = reinterpret_cast<const char*>(lut_l);
@@ -151,7 +161,8 @@ __device__ __forceinline__ void encode8(const Piece8& p, float c14, float c28, f
 #pragma unroll
     for (int o = 0; o < 2; ++o) {
       const int e = 2 * h + o;
-      const float t = fmaf(p.x3[e], c42, fmaf(p.x2[e], c28, fmaf(p.x1[e], c14, p.x0[e])));
+      float t = fmaf(p.x3[e], c42, fmaf(p.x2[e], c28, fmaf(p.x1[e], c14, p.x0[e])));
+      if (kWide) t = fmaf(p.x4[e], c56, t);
       const float q = fmaf(t, inv_m, kMagic) - kMagic;
       const float r = fmaf(-q, m_f, t);
       const uint32_t off = __float_as_uint(fmaf(r, 2.0f, kMagic + 2.0f * kLutOffset)) & 0x1FFu;
@@ -168,6 +179,7 @@ __device__ __forceinline__ void encode8(const Piece8& p, float c14, float c28, f
 // B side: plane row = column j of B, source already K-contiguous.
 // Block = 256 threads = 2048 consecutive k of one column; thread = 8 consecutive k.
 // ------------------------------------------------------------------------------------
+template <bool kWide>
 __global__ void __launch_bounds__(256) encode_cols_kernel(const double* __restrict__ B, int64_t ldb, int64_t N, int64_t K,
                                                           int64_t Kp, ModulusTable mt, const uint16_t* __restrict__ lut,
                                                           const int32_t* __restrict__ shifts, uint8_t* __restrict__ planes,
@@ -209,12 +221,12 @@ __global__ void __launch_bounds__(256) encode_cols_kernel(const double* __restri
         if (k + e < K) int_out[j * K + k + e] = neg[e] ? -(long long)mag[e] : (long long)mag[e];
     }
   }
-  Piece8 p;
-  split8(mag, neg, p);
+  Piece8<kWide> p;
+  split8<kWide>(mag, neg, p);
   uint8_t* dst = planes + (size_t)j * pitch + (size_t)(k / 2);
   for (int l = 0; l < mt.L; ++l) {
     uint32_t w0, w1;
-    encode8(p, mt.c14[l], mt.c28[l], mt.c42[l], mt.inv_m[l], mt.m_f[l], lut_s + l * kLutStride, w0, w1);
+    encode8<kWide>(p, mt.c14[l], mt.c28[l], mt.c42[l], mt.c56[l], mt.inv_m[l], mt.m_f[l], lut_s + l * kLutStride, w0, w1);
     *reinterpret_cast<uint32_t*>(dst + (size_t)(2 * l) * plane_bytes) = w0;
     *reinterpret_cast<uint32_t*>(dst + (size_t)(2 * l + 1) * plane_bytes) = w1;
   }
@@ -231,6 +243,7 @@ constexpr int kRowTile = 32;
 constexpr int kRowTileK = 64;
 constexpr int kStageStride = 9;  // words per staged row (8 used): odd stride avoids bank conflicts
 
+template <bool kWide>
 __global__ void __launch_bounds__(256) encode_rows_kernel(const double* __restrict__ A, int64_t lda, int64_t M, int64_t K,
                                                           int64_t Kp, ModulusTable mt, const uint16_t* __restrict__ lut,
                                                           const int32_t* __restrict__ shifts, uint8_t* __restrict__ planes,
@@ -278,11 +291,11 @@ __global__ void __launch_bounds__(256) encode_rows_kernel(const double* __restri
     }
   }
   __syncthreads();  // in_s is dead from here on; out_s takes its place
-  Piece8 p;
-  split8(mag, neg, p);
+  Piece8<kWide> p;
+  split8<kWide>(mag, neg, p);
   for (int l = 0; l < mt.L; ++l) {
     uint32_t w0, w1;
-    encode8(p, mt.c14[l], mt.c28[l], mt.c42[l], mt.inv_m[l], mt.m_f[l], lut_s + l * kLutStride, w0, w1);
+    encode8<kWide>(p, mt.c14[l], mt.c28[l], mt.c42[l], mt.c56[l], mt.inv_m[l], mt.m_f[l], lut_s + l * kLutStride, w0, w1);
     out_s[((2 * l) * kRowTile + r) * kStageStride + g] = w0;
     out_s[((2 * l + 1) * kRowTile + r) * kStageStride + g] = w1;
   }
@@ -355,20 +368,22 @@ cudaError_t launch_encode_operand(const Geometry& g, const ModulusTable& mt, int
   const uint16_t* lut = reinterpret_cast<const uint16_t*>(ws + g.off_lut);
   const int lut_bytes = (mt.L * kLutStride * (int)sizeof(uint16_t) + 15) & ~15;
   const int reps = 4;
+  const bool wide = g.c_bits > 56;  // integers beyond 56 bits take a fifth 14-bit piece
   if (which == 0) {
     const size_t stage = (size_t)2 * mt.L * kRowTile * kStageStride * sizeof(uint32_t);
     const size_t in_bytes = (size_t)kRowTileK * kRowTile * sizeof(double);
     const size_t smem = lut_bytes + (stage > in_bytes ? stage : in_bytes);
-    cudaError_t e = cudaFuncSetAttribute(encode_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    auto* kernel = wide ? encode_rows_kernel<true> : encode_rows_kernel<false>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     dim3 grid((unsigned)(g.Mp / kRowTile), (unsigned)((g.Kp / kRowTileK + reps - 1) / reps));
-    encode_rows_kernel<<<grid, 256, smem, st>>>(X, ldx, g.M, g.K, g.Kp, mt, lut, reinterpret_cast<const int32_t*>(ws + g.off_s),
-                                                ws + g.off_planes_a, g.plane_bytes_a, g.pitch, int_out, reps);
+    kernel<<<grid, 256, smem, st>>>(X, ldx, g.M, g.K, g.Kp, mt, lut, reinterpret_cast<const int32_t*>(ws + g.off_s),
+                                    ws + g.off_planes_a, g.plane_bytes_a, g.pitch, int_out, reps);
   } else {
     dim3 grid((unsigned)g.Np, (unsigned)(((g.Kp + 2047) / 2048 + reps - 1) / reps));
-    encode_cols_kernel<<<grid, 256, lut_bytes, st>>>(X, ldx, g.N, g.K, g.Kp, mt, lut,
-                                                    reinterpret_cast<const int32_t*>(ws + g.off_t), ws + g.off_planes_b,
-                                                    g.plane_bytes_b, g.pitch, int_out, reps);
+    auto* kernel = wide ? encode_cols_kernel<true> : encode_cols_kernel<false>;
+    kernel<<<grid, 256, lut_bytes, st>>>(X, ldx, g.N, g.K, g.Kp, mt, lut, reinterpret_cast<const int32_t*>(ws + g.off_t),
+                                         ws + g.off_planes_b, g.plane_bytes_b, g.pitch, int_out, reps);
   }
   return cudaGetLastError();
 }

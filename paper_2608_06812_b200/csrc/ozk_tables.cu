@@ -126,14 +126,15 @@ int host_select_moduli(int count, int* out) {
   return n;
 }
 
-// Eq. 3 for a c-bit integer width: 2 K 2^(2c) < P, capped at 53 bits (Section 4.2).
-int host_capacity_bits(int64_t K, int L) {
+// Eq. 3 for a c-bit integer width: 2 K 2^(2c) < P, capped at max_bits (53 in Section 4.2; up to 62 in
+// the extended-capacity mode).
+int host_capacity_bits(int64_t K, int L, int max_bits) {
   int m[kMaxModuli];
   if (L < 1 || L > kMaxModuli || host_select_moduli(L, m) != L) return -1;
   Big P = product_of(m, L);
   Big twoK = big_from(2 * (uint64_t)(K < 1 ? 1 : K));
   int c = 0;
-  while (c < 53) {
+  while (c < max_bits) {
     if (big_bits(twoK) + 2 * (c + 1) >= 32 * kW) break;
     if (big_cmp(big_shl(twoK, 2 * (c + 1)), P) >= 0) break;
     ++c;
@@ -154,11 +155,12 @@ bool host_build_modulus_table(int L, ModulusTable* t) {
     t->c14[i] = centred(1ull << 14);
     t->c28[i] = centred(1ull << 28);
     t->c42[i] = centred(1ull << 42);
+    t->c56[i] = centred(1ull << 56);
     t->inv_m[i] = 1.0f / (float)m;
     t->m_f[i] = (float)m;
   }
   for (int i = L; i < kMaxModuli; ++i)
-    t->m[i] = 1, t->recip[i] = 0, t->c14[i] = t->c28[i] = t->c42[i] = 0.0f, t->inv_m[i] = 1.0f, t->m_f[i] = 1.0f;
+    t->m[i] = 1, t->recip[i] = 0, t->c14[i] = t->c28[i] = t->c42[i] = t->c56[i] = 0.0f, t->inv_m[i] = 1.0f, t->m_f[i] = 1.0f;
   return true;
 }
 

@@ -49,7 +49,8 @@ def from_dev_colmajor(T: torch.Tensor, rows: int, cols: int) -> np.ndarray:
     return T.cpu().numpy()[:cols, :rows].T.copy()
 
 
-def dgemm(A: np.ndarray, B: np.ndarray, L: int, lda=None, ldb=None, ldc=None) -> np.ndarray:
+def dgemm(A: np.ndarray, B: np.ndarray, L: int, lda=None, ldb=None, ldc=None, max_bits=None) -> np.ndarray:
+    """ozk_dgemm (or ozk_dgemm_ext when max_bits is given) on freshly uploaded column-major copies."""
     M, K = A.shape
     _, N = B.shape
     lda = max(M, 1) if lda is None else lda
@@ -58,7 +59,11 @@ def dgemm(A: np.ndarray, B: np.ndarray, L: int, lda=None, ldb=None, ldc=None) ->
     ensure_workspace(ozk.ozk_dgemm_workspace_bytes(M, N, K, L))
     dA, dB = to_dev_colmajor(A, lda), to_dev_colmajor(B, ldb)
     dC = torch.full((max(N, 1), ldc), float("nan"), dtype=torch.float64, device="cuda")
-    ozk.check(ozk.ozk_dgemm(M, N, K, dA.data_ptr(), lda, dB.data_ptr(), ldb, dC.data_ptr(), ldc, L, stream()), "ozk_dgemm")
+    if max_bits is None:
+        ozk.check(ozk.ozk_dgemm(M, N, K, dA.data_ptr(), lda, dB.data_ptr(), ldb, dC.data_ptr(), ldc, L, stream()), "ozk_dgemm")
+    else:
+        ozk.check(ozk.ozk_dgemm_ext(M, N, K, dA.data_ptr(), lda, dB.data_ptr(), ldb, dC.data_ptr(), ldc, L, max_bits, stream()),
+                  "ozk_dgemm_ext")
     ozk.check(ozk.ozk_get_async_status(stream()), "ozk_get_async_status")
     return from_dev_colmajor(dC, M, N)
 

@@ -41,6 +41,11 @@ def test_capacity_and_crt_constants_match_the_oracle():
     for K in (1, 256, 4096, 8192, 16384, 131072, 300000, ozk.OZK_MAX_K):
         for L in range(4, 28):
             assert ozk.ozk_capacity_bits(K, L) == moduli.capacity_bits(K, L)
+    for K in (40, 4096, 16384, 300000):
+        for L in (19, 20, 21, 22, 27):
+            for cap in (40, 53, 56, 57, 62):
+                assert ozk.ozk_capacity_bits_ext(K, L, cap) == moduli.capacity_bits(K, L, cap=cap)
+    assert ozk.ozk_capacity_bits_ext(16384, 22, 63) == ozk.OZK_ERR_INVALID_ARG
     assert ozk.ozk_capacity_bits(16384, 19) == 53
     assert ozk.ozk_capacity_bits(1 << 20, 2) == ozk.OZK_ERR_UNSUPPORTED
     for L in (2, 14, 19, 27):
