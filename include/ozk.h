@@ -139,14 +139,15 @@ ozk_status ozk_igemm_i8(int64_t M, int64_t N, int64_t K,
                         int32_t* C, int64_t ldc, void* stream);
 
 /* ozk_dgemm for matrices in HOST memory (pinned memory for full speed): same result, same
- * arguments, but A, B and C are host pointers.  C is produced in blocks of 4096 x 4096; the
- * host-to-device copies of the row blocks of A and the column blocks of B, the three stages, and
- * the device-to-host copies of the finished blocks of C run on three streams and overlap (the
- * paper times device-resident data only, Section 6.1).  The call returns once everything is
- * enqueued; `stream` completes when C has arrived in host memory.  The workspace holds the limb
- * planes of two row blocks of A and of all of B, plus two staging blocks each for A, B and C.
- * The first call creates two internal streams and a pool of events.  K <= OZK_CHUNK_K here
- * (OZK_ERR_UNSUPPORTED beyond). */
+ * arguments, but A, B and C are host pointers.  C is produced in blocks of 2048 x 2048 (larger
+ * when a dimension exceeds 131072); the host-to-device copies of the column blocks of B and the
+ * row blocks of A (sent alternately), the three stages, and the device-to-host copies of the
+ * finished blocks of C run on three streams and overlap: a block of C is computed as soon as
+ * its row block and its column block have arrived (the paper times device-resident data only,
+ * Section 6.1).  The call returns once everything is enqueued; `stream` completes when C has
+ * arrived in host memory.  The workspace holds the limb planes of A and B, one block of
+ * residues, and two staging blocks each for A, B and C.  The first call creates two internal
+ * streams and a pool of events.  K <= OZK_CHUNK_K here (OZK_ERR_UNSUPPORTED beyond). */
 size_t ozk_dgemm_host_workspace_bytes(int64_t M, int64_t N, int64_t K, int num_moduli);
 ozk_status ozk_dgemm_host(int64_t M, int64_t N, int64_t K,
                           const double* A, int64_t lda,
