@@ -47,7 +47,7 @@ bool make_geometry_impl(int64_t M, int64_t N, int64_t K, int L, Geometry* g, int
   off += align_up((size_t)kMaxModuli * kLutStride * sizeof(uint16_t), 1024);
   g->off_amax_a = off;
   off += (size_t)g->Mp * 8;
-  g->off_amax_b = off;  // must follow amax_a directly: both are cleared by one memset
+  g->off_amax_b = off;
   off += (size_t)g->Np * 8;
   off = align_up(off, 1024);
   g->off_s = off;

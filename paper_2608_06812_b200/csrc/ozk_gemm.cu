@@ -133,15 +133,12 @@ __device__ __forceinline__ void drain_and_release(uint32_t base, int W, bool top
     tmem_ld_32x32(base + 1 * W + c * 32, d1);
     if (top) tmem_ld_32x32(base + 2 * W + c * 32, d2);
     if constexpr (kFast) {
+      // D0 goes straight into t (raw FP32 bits until after the release): one wait covers all three loads
+      tmem_ld_32x32(base + 0 * W + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&t[c * 32]));
       tmem_wait_ld();
 #pragma unroll
       for (int e = 0; e < 32; ++e)
         u[c * 32 + e] = top ? __float_as_uint(fmaf(__uint_as_float(d2[e]), 13.0f, __uint_as_float(d1[e]))) : d1[e];
-      uint32_t d0[32];
-      tmem_ld_32x32(base + 0 * W + c * 32, d0);
-      tmem_wait_ld();
-#pragma unroll
-      for (int e = 0; e < 32; ++e) t[c * 32 + e] = d0[e];  // raw FP32 bits until after the release
     } else {
       uint32_t d0[32];
       tmem_ld_32x32(base + 0 * W + c * 32, d0);
