@@ -47,3 +47,25 @@ def test_back_to_back_calls_without_synchronisation():
     for (A, B, L, dA, dB, dC) in work:
         M, N = A.shape[0], B.shape[1]
         assert gu.bits_equal(gu.from_dev_colmajor(dC, M, N), ozaki2.dgemm(A, B, L).C)
+
+
+def test_operands_at_odd_addresses():
+    """A, B and C start 8 bytes past a 16-byte boundary and have odd leading dimensions: every vectorised load and
+    store in the O(N^2) kernels has to fall back to its scalar form and give the same bits."""
+    M, N, K, L = 203, 331, 517, 19
+    A = inputs.lognormal_matrix(M, K, 1.0, seed=77)
+    B = inputs.lognormal_matrix(K, N, 1.0, seed=78)
+    lda, ldb, ldc = M + 2, K + 4, M + 4                      # odd leading dimensions: columns alternate in alignment
+    bufA = torch.zeros(K * lda + 1, dtype=torch.float64, device="cuda")
+    bufB = torch.zeros(N * ldb + 1, dtype=torch.float64, device="cuda")
+    bufC = torch.full((N * ldc + 1,), float("nan"), dtype=torch.float64, device="cuda")
+    bufA[1:].view(K, lda)[:, :M] = torch.from_numpy(np.ascontiguousarray(A.T)).cuda()
+    bufB[1:].view(N, ldb)[:, :K] = torch.from_numpy(np.ascontiguousarray(B.T)).cuda()
+    assert bufA[1:].data_ptr() % 16 == 8
+    gu.ensure_workspace(ozk.ozk_dgemm_workspace_bytes(M, N, K, L))
+    ozk.check(ozk.ozk_dgemm(M, N, K, bufA[1:].data_ptr(), lda, bufB[1:].data_ptr(), ldb, bufC[1:].data_ptr(), ldc, L, gu.stream()),
+              "ozk_dgemm")
+    ozk.check(ozk.ozk_get_async_status(gu.stream()), "status")
+    C = bufC[1:].view(N, ldc).cpu().numpy()
+    assert gu.bits_equal(C[:, :M].T.copy(), ozaki2.dgemm(A, B, L).C)
+    assert np.isnan(C[:, M:]).all() and np.isnan(bufC[0].item())   # nothing outside C was written
