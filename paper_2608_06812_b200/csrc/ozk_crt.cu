@@ -202,7 +202,7 @@ __device__ __forceinline__ double reconstruct_lean(const unsigned long long (&ac
 }
 
 template <int WW, int NW, bool LEAN>
-__global__ void __launch_bounds__(256) crt4_kernel(const __grid_constant__ CrtTable ct, const uint8_t* __restrict__ res,
+__global__ void __launch_bounds__(256, LEAN ? 4 : 2) crt4_kernel(const __grid_constant__ CrtTable ct, const uint8_t* __restrict__ res,
                                                    int64_t res_ld, size_t res_stride, const int32_t* __restrict__ s,
                                                    const int32_t* __restrict__ t, int64_t M, int64_t N,
                                                    double* __restrict__ C, int64_t ldc) {
