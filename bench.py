@@ -287,6 +287,7 @@ def run_ozk(args, rank: int, local_rank: int, world: int) -> None:
     for _ in range(max(args.warmup, 3)):
         step()
     ozk.check(ozk.ozk_get_async_status(stream), "ozk_get_async_status")
+    ozk.check(ozk.ozk_stage_timing_enable(not oz1), "ozk_stage_timing_enable")   # forget the warm-up calls
 
     # ---- device-resident timing: exactly `steps` steps between two barriers -----------------
     sampler = ClockSampler(local_rank)
@@ -299,11 +300,11 @@ def run_ozk(args, rank: int, local_rank: int, world: int) -> None:
     for i in range(args.steps):
         step()
         ev[i + 1].record()
-        # per-stage CUDA events recorded by the library on this stream, read live inside the timed
-        # region (the read waits for this step's last event; a step is >100 ms, the wait adds microseconds)
-        if not oz1:
-            stage_acc += np.array(ozk.ozk_stage_timing_read())
     barrier()
+    # per-stage CUDA events the library recorded on this stream inside the timed steps (a ring of the
+    # last 64 calls), read after the region so that no step waits for the host
+    if not oz1:
+        stage_acc = np.array(ozk.ozk_stage_timing_read()) * args.steps
     total_ms = ev[0].elapsed_time(ev[args.steps])
     clocks = sampler.stop() if rank == 0 else None
     ozk.check(ozk.ozk_get_async_status(stream), "ozk_get_async_status")

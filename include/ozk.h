@@ -227,8 +227,10 @@ ozk_status ozk_row_shifts_noalloc(int64_t M, int64_t K, const double* A, int64_t
 /* Measurement aid (the paper times its stages with CUDA events, Section 6.1): when enabled,
  * ozk_dgemm records four CUDA events on its stream, before stage 1 and after each of the three
  * stages.  Enabling creates the events (a host-side allocation; do it outside timed regions).
- * ozk_stage_timing_read() synchronises on the last event and writes the milliseconds of
- * preprocessing, limb GEMM and reconstruction of the most recent ozk_dgemm to ms3[0..2] (host). */
+ * ozk_stage_timing_read() synchronises on those events and writes the milliseconds of
+ * preprocessing, limb GEMM and reconstruction to ms3[0..2] (host), averaged over the ozk_dgemm
+ * calls made since enabling or since the previous read (the most recent 64 of them), so that a
+ * timed loop need not synchronise between its calls.  No call since then -> OZK_ERR_INVALID_ARG. */
 ozk_status ozk_stage_timing_enable(int enable);
 ozk_status ozk_stage_timing_read(float* ms3);
 

@@ -16,15 +16,19 @@ Workspace g_ws;
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Stage events of the most recent calls, in a ring: the reader averages over the calls since the
+// last read without having synchronised between them.
+constexpr int kTimingRing = 64;
 struct StageTiming {
   bool enabled = false;
-  bool recorded = false;
-  cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
+  bool created = false;
+  int calls = 0;  // ozk_dgemm calls recorded since enable / the last read
+  cudaEvent_t ev[kTimingRing][4];
 };
 StageTiming g_timing;
 
 void mark(int i, cudaStream_t st) {
-  if (g_timing.enabled) cudaEventRecord(g_timing.ev[i], st);
+  if (g_timing.enabled) cudaEventRecord(g_timing.ev[g_timing.calls % kTimingRing][i], st);
 }
 
 // Workspace layout for an (M, N, K, L) problem.  Returns false on invalid sizes.
@@ -295,26 +299,38 @@ ozk_status ozk_dgemm_ext(int64_t M, int64_t N, int64_t K, const double* A, int64
                  nullptr, st) != cudaSuccess)
     return OZK_ERR_CUDA;
   mark(3, st);
-  g_timing.recorded = g_timing.enabled;
+  if (g_timing.enabled) ++g_timing.calls;
   return OZK_OK;
 }
 
 ozk_status ozk_stage_timing_enable(int enable) {
-  if (enable && !g_timing.ev[0]) {
-    for (int i = 0; i < 4; ++i)
-      if (cudaEventCreate(&g_timing.ev[i]) != cudaSuccess) return OZK_ERR_CUDA;
+  if (enable && !g_timing.created) {
+    for (int r = 0; r < kTimingRing; ++r)
+      for (int i = 0; i < 4; ++i)
+        if (cudaEventCreate(&g_timing.ev[r][i]) != cudaSuccess) return OZK_ERR_CUDA;
+    g_timing.created = true;
   }
   g_timing.enabled = enable != 0;
-  g_timing.recorded = false;
+  g_timing.calls = 0;
   return OZK_OK;
 }
 
 ozk_status ozk_stage_timing_read(float* ms3) {
   if (!ms3) return OZK_ERR_INVALID_ARG;
-  if (!g_timing.recorded) return OZK_ERR_INVALID_ARG;
-  if (cudaEventSynchronize(g_timing.ev[3]) != cudaSuccess) return OZK_ERR_CUDA;
-  for (int i = 0; i < 3; ++i)
-    if (cudaEventElapsedTime(&ms3[i], g_timing.ev[i], g_timing.ev[i + 1]) != cudaSuccess) return OZK_ERR_CUDA;
+  if (g_timing.calls < 1) return OZK_ERR_INVALID_ARG;
+  const int n = g_timing.calls < kTimingRing ? g_timing.calls : kTimingRing;
+  double sum[3] = {0.0, 0.0, 0.0};
+  for (int back = 0; back < n; ++back) {
+    cudaEvent_t* ev = g_timing.ev[(g_timing.calls - 1 - back) % kTimingRing];
+    if (cudaEventSynchronize(ev[3]) != cudaSuccess) return OZK_ERR_CUDA;
+    for (int i = 0; i < 3; ++i) {
+      float ms = 0.0f;
+      if (cudaEventElapsedTime(&ms, ev[i], ev[i + 1]) != cudaSuccess) return OZK_ERR_CUDA;
+      sum[i] += ms;
+    }
+  }
+  for (int i = 0; i < 3; ++i) ms3[i] = (float)(sum[i] / n);
+  g_timing.calls = 0;
   return OZK_OK;
 }
 

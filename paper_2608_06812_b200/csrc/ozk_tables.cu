@@ -4,6 +4,8 @@
 #include <math.h>
 #include <string.h>
 
+#include <mutex>
+
 #include "ozk_common.cuh"
 
 namespace ozk {
@@ -111,18 +113,34 @@ Big product_of(const int* m, int L) {
   return P;
 }
 
+// Section 5.1: 169 first, then descending, pairwise coprime, no other multiple of 13.  The search is
+// run once per process; later calls copy a prefix of its result.
+struct ModulusList {
+  int m[kMaxModuli];
+  int n;
+};
+const ModulusList& modulus_list() {
+  static const ModulusList list = [] {
+    ModulusList r;
+    r.n = 0;
+    for (int m = 169; m >= 2 && r.n < kMaxModuli; --m) {
+      if (m != 169 && m % 13 == 0) continue;
+      if (!two_limb_representable(m)) continue;
+      bool ok = true;
+      for (int i = 0; i < r.n; ++i) ok = ok && gcd_int(m, r.m[i]) == 1;
+      if (ok) r.m[r.n++] = m;
+    }
+    return r;
+  }();
+  return list;
+}
+
 }  // namespace
 
-// Section 5.1: 169 first, then descending, pairwise coprime, no other multiple of 13.
 int host_select_moduli(int count, int* out) {
-  int n = 0;
-  for (int m = 169; m >= 2 && n < count; --m) {
-    if (m != 169 && m % 13 == 0) continue;
-    if (!two_limb_representable(m)) continue;
-    bool ok = true;
-    for (int i = 0; i < n; ++i) ok = ok && gcd_int(m, out[i]) == 1;
-    if (ok) out[n++] = m;
-  }
+  const ModulusList& list = modulus_list();
+  const int n = count < list.n ? count : list.n;
+  for (int i = 0; i < n; ++i) out[i] = list.m[i];
   return n;
 }
 
@@ -142,7 +160,49 @@ int host_capacity_bits(int64_t K, int L, int max_bits) {
   return c;
 }
 
+namespace {
+bool build_modulus_table(int L, ModulusTable* t);
+bool build_crt_table(int L, CrtTable* t);
+}  // namespace
+
+// The per-L tables are built once per process and copied out afterwards.
 bool host_build_modulus_table(int L, ModulusTable* t) {
+  if (L < 1 || L > kMaxModuli) return false;
+  static std::mutex mu;
+  static bool have[kMaxModuli + 1];
+  static ModulusTable cache[kMaxModuli + 1];
+  std::lock_guard<std::mutex> lock(mu);
+  if (!have[L]) {
+    if (!build_modulus_table(L, &cache[L])) return false;
+    have[L] = true;
+  }
+  *t = cache[L];
+  return true;
+}
+
+bool host_build_crt_table(int L, CrtTable* t) {
+  if (L < 1 || L > kMaxModuli) {
+    memset(t, 0, sizeof *t);
+    return false;
+  }
+  static std::mutex mu;
+  static bool have[kMaxModuli + 1];
+  static CrtTable cache[kMaxModuli + 1];
+  std::lock_guard<std::mutex> lock(mu);
+  if (!have[L]) {
+    if (!build_crt_table(L, &cache[L])) {
+      *t = cache[L];
+      return false;
+    }
+    have[L] = true;
+  }
+  *t = cache[L];
+  return true;
+}
+
+namespace {
+
+bool build_modulus_table(int L, ModulusTable* t) {
   if (L < 1 || L > kMaxModuli || host_select_moduli(L, t->m) != L) return false;
   t->L = L;
   for (int i = 0; i < L; ++i) {
@@ -165,7 +225,7 @@ bool host_build_modulus_table(int L, ModulusTable* t) {
 }
 
 // Section 5.2: w_l = M_l (M_l^-1 mod m_l), M_l = P / m_l; S = sum r_l w_l <= sum (m_l - 1) w_l.
-bool host_build_crt_table(int L, CrtTable* t) {
+bool build_crt_table(int L, CrtTable* t) {
   memset(t, 0, sizeof *t);
   if (L < 1 || L > kMaxModuli || host_select_moduli(L, t->m) != L) return false;
   t->L = L;
@@ -198,5 +258,7 @@ bool host_build_crt_table(int L, CrtTable* t) {
   t->p_bits = big_bits(P);
   return true;
 }
+
+}  // namespace
 
 }  // namespace ozk

@@ -69,3 +69,13 @@ def test_extended_capacity_4096_phi4_samples_and_error():
     assert moduli.capacity_bits(n, L, cap=62) == 62
     err = {mb: exact.normwise_error(got[mb][:16, :16], A[rows[:16]], B[:, cols[:16]], against_rounded=True) for mb in (53, 62)}
     assert err[62] < err[53] / 100
+
+
+def test_extended_capacity_with_two_k_ranges():
+    """K beyond one limb-GEMM range in the extended mode: residues of the two ranges are added modulo m."""
+    M, N, K, L = 16, 64, 135000, 22
+    A = inputs.lognormal_matrix(M, K, 2.0, seed=11)
+    B = inputs.lognormal_matrix(K, N, 2.0, seed=12)
+    ref = ozaki2.dgemm(A, B, L, max_bits=62)
+    assert 53 < ref.c_bits < 62                                # Eq. 3 limits the width at this K
+    assert gu.bits_equal(gu.dgemm(A, B, L, max_bits=62), ref.C)

@@ -151,3 +151,23 @@ def test_crt_stage_matches_oracle_on_arbitrary_residues(L, fast):
                 assert words_to_int(X[j, i]) == int(xs[i, j]), (i, j)
             want = ozaki2.round_scaled_to_double(int(xs[i, j]), int(s[i]) + int(t[j]))
             assert np.float64(C[i, j]).view(np.uint64) == np.float64(want).view(np.uint64), (i, j, xs[i, j], s[i] + t[j])
+
+
+def test_stage_timing_averages_over_the_calls_since_the_last_read():
+    """Measurement aid: four events per ozk_dgemm call kept in a ring; one read after several calls returns
+    positive per-stage averages and empties the ring."""
+    A = inputs.lognormal_matrix(256, 512, 1.0, seed=1)
+    B = inputs.lognormal_matrix(512, 256, 1.0, seed=2)
+    ozk.check(ozk.ozk_stage_timing_enable(True), "enable")
+    try:
+        with pytest.raises(ozk.OzkError):
+            ozk.ozk_stage_timing_read()                      # nothing recorded yet
+        ref = gu.dgemm(A, B, 19)
+        for _ in range(3):
+            assert gu.bits_equal(gu.dgemm(A, B, 19), ref)
+        ms = ozk.ozk_stage_timing_read()
+        assert all(0.0 < v < 1000.0 for v in ms)
+        with pytest.raises(ozk.OzkError):
+            ozk.ozk_stage_timing_read()                      # the read emptied the ring
+    finally:
+        ozk.check(ozk.ozk_stage_timing_enable(False), "disable")
