@@ -104,7 +104,9 @@ ozk_status ozk_get_async_status(void* stream);
  *   such ranges whose residues are added modulo each modulus (Section 5.1, "Exactness of the
  *   FP32 accumulation": chunking), up to OZK_MAX_K.  The capacity of ozk_capacity_bits(K, ...)
  *   always refers to the whole K.  M, N, K = 0 are allowed (K = 0 gives C = 0).
- * Returns OZK_OK once the work is enqueued. */
+ * Returns OZK_OK once the work is enqueued.  The call only enqueues kernels and memsets on
+ * `stream` (no allocation, no synchronisation), so after one eager call, which sets the
+ * kernels' attributes, it may be captured into a CUDA graph and replayed. */
 ozk_status ozk_dgemm(int64_t M, int64_t N, int64_t K,
                      const double* A, int64_t lda,
                      const double* B, int64_t ldb,

@@ -69,3 +69,31 @@ def test_operands_at_odd_addresses():
     C = bufC[1:].view(N, ldc).cpu().numpy()
     assert gu.bits_equal(C[:, :M].T.copy(), ozaki2.dgemm(A, B, L).C)
     assert np.isnan(C[:, M:]).all() and np.isnan(bufC[0].item())   # nothing outside C was written
+
+
+def test_cuda_graph_capture_and_replay():
+    """ozk_dgemm only enqueues work on its stream (kernels, memsets, one cooperative launch), so a call can be
+    captured into a CUDA graph and replayed on new data in the same buffers."""
+    M, N, K, L = 384, 512, 640, 19
+    A1 = inputs.lognormal_matrix(M, K, 1.0, seed=5)
+    B1 = inputs.lognormal_matrix(K, N, 1.0, seed=6)
+    A2 = inputs.lognormal_matrix(M, K, 2.0, seed=7)
+    B2 = inputs.lognormal_matrix(K, N, 2.0, seed=8)
+    gu.ensure_workspace(ozk.ozk_dgemm_workspace_bytes(M, N, K, L))
+    dA, dB = gu.to_dev_colmajor(A1), gu.to_dev_colmajor(B1)
+    dC = torch.zeros((N, M), dtype=torch.float64, device="cuda")
+    ozk.check(ozk.ozk_dgemm(M, N, K, dA.data_ptr(), M, dB.data_ptr(), K, dC.data_ptr(), M, L, gu.stream()), "warm-up")
+    ozk.check(ozk.ozk_get_async_status(gu.stream()), "status")
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        ozk.check(ozk.ozk_dgemm(M, N, K, dA.data_ptr(), M, dB.data_ptr(), K, dC.data_ptr(), M, L, gu.stream()), "capture")
+    dC.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert gu.bits_equal(gu.from_dev_colmajor(dC, M, N), ozaki2.dgemm(A1, B1, L).C)
+    dA.copy_(gu.to_dev_colmajor(A2))
+    dB.copy_(gu.to_dev_colmajor(B2))
+    graph.replay()
+    torch.cuda.synchronize()
+    assert gu.bits_equal(gu.from_dev_colmajor(dC, M, N), ozaki2.dgemm(A2, B2, L).C)
+    ozk.check(ozk.ozk_get_async_status(gu.stream()), "status")
