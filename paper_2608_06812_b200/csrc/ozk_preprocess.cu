@@ -234,14 +234,17 @@ __global__ void __launch_bounds__(256) encode_cols_kernel(const double* __restri
 }
 
 // ------------------------------------------------------------------------------------
-// A side: plane row = row i of A, source is M-contiguous.  Block = tile of 32 rows x 64 k.
-//   load    coalesced along rows into shared memory (k-major)
-//   encode  thread = (row, group of 8 k), warp = 32 rows of one group (conflict-free reads)
-//   store   staged through shared memory so that each plane row receives 32 contiguous bytes
+// A side: plane row = row i of A, source is M-contiguous.  Block = tile of 16 rows x 128 k.
+//   load    coalesced along rows (16 rows = 128 contiguous bytes per k) into shared memory, stored
+//           [row][group of 8 k][k in group] with odd strides, so that both the row-major writes
+//           and the k-major reads below are free of bank conflicts
+//   encode  thread = (row, group of 8 k); half a warp = the 16 groups of one row
+//   store   straight to the planes: the 16 groups of a row are 64 contiguous bytes per plane
 // ------------------------------------------------------------------------------------
-constexpr int kRowTile = 32;
-constexpr int kRowTileK = 64;
-constexpr int kStageStride = 9;  // words per staged row (8 used): odd stride avoids bank conflicts
+constexpr int kRowTile = 16;
+constexpr int kRowTileK = 128;
+constexpr int kGroupStride = 9;                                         // doubles per group of 8 k (8 used)
+constexpr int kRowStride = (kRowTileK / 8) * kGroupStride + 1;          // doubles per row: 145, odd
 
 template <bool kWide>
 __global__ void __launch_bounds__(256) encode_rows_kernel(const double* __restrict__ A, int64_t lda, int64_t M, int64_t K,
@@ -251,8 +254,7 @@ __global__ void __launch_bounds__(256) encode_rows_kernel(const double* __restri
   extern __shared__ __align__(16) uint8_t smem[];
   uint16_t* lut_s = reinterpret_cast<uint16_t*>(smem);                          // L * kLutStride entries
   const int lut_bytes = (mt.L * kLutStride * (int)sizeof(uint16_t) + 15) & ~15;
-  double* in_s = reinterpret_cast<double*>(smem + lut_bytes);                    // [64][32] doubles
-  uint32_t* out_s = reinterpret_cast<uint32_t*>(smem + lut_bytes);               // [2L][32][9] words, reuses in_s
+  double* in_s = reinterpret_cast<double*>(smem + lut_bytes);                    // [16][145] doubles
   const int t = threadIdx.x;
   const int64_t i0 = (int64_t)blockIdx.x * kRowTile;
   {  // the table is copied once per block and reused for `reps` tiles along k
@@ -260,28 +262,28 @@ __global__ void __launch_bounds__(256) encode_rows_kernel(const double* __restri
     uint4* dst = reinterpret_cast<uint4*>(lut_s);
     for (int i = t; i < mt.L * kLutStride / 8; i += blockDim.x) dst[i] = src[i];
   }
+  const int r = t >> 4, g = t & 15;  // encode role: row r, k group g
+  const int64_t i = i0 + r;
+  const int s = shifts[i];           // shifts has Mp entries; padded rows hold 0
   for (int rep = 0; rep < reps; ++rep) {
-  const int64_t k0 = ((int64_t)blockIdx.y * reps + rep) * kRowTileK;
-  if (k0 >= Kp) break;  // uniform over the block
-  if (rep) __syncthreads();  // the previous tile's staged output has been written out
-  {
-    const int ti = t & 31, tk = t >> 5;
-    const int64_t i = i0 + ti;
+    const int64_t k0 = ((int64_t)blockIdx.y * reps + rep) * kRowTileK;
+    if (k0 >= Kp) break;        // uniform over the block
+    if (rep) __syncthreads();   // the previous tile has been read
+    {
+      const int ti = t & 15, tk = t >> 4;  // load role: row ti, k = tk, tk + 16, ...
+      const int64_t il = i0 + ti;
 #pragma unroll
-    for (int n = 0; n < 8; ++n) {
-      const int64_t k = k0 + tk + 8 * n;
-      in_s[(tk + 8 * n) * kRowTile + ti] = (i < M && k < K) ? __ldg(A + i + k * lda) : 0.0;
+      for (int n = 0; n < 8; ++n) {
+        const int kk = tk + 16 * n;
+        const int64_t k = k0 + kk;
+        in_s[ti * kRowStride + (kk >> 3) * kGroupStride + (kk & 7)] = (il < M && k < K) ? __ldg(A + il + k * lda) : 0.0;
+      }
     }
-  }
-  __syncthreads();
-  const int r = t & 31, g = t >> 5;
-  unsigned long long mag[8];
-  bool neg[8];
-  {
-    const int64_t i = i0 + r;
-    const int s = shifts[i];  // shifts has Mp entries; padded rows hold 0
+    __syncthreads();
+    unsigned long long mag[8];
+    bool neg[8];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) mag[e] = to_integer_magnitude(in_s[(8 * g + e) * kRowTile + r], s, &neg[e]);
+    for (int e = 0; e < 8; ++e) mag[e] = to_integer_magnitude(in_s[r * kRowStride + g * kGroupStride + e], s, &neg[e]);
     if (int_out && i < M) {
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
@@ -289,21 +291,15 @@ __global__ void __launch_bounds__(256) encode_rows_kernel(const double* __restri
         if (k < K) int_out[i + k * M] = neg[e] ? -(long long)mag[e] : (long long)mag[e];
       }
     }
-  }
-  __syncthreads();  // in_s is dead from here on; out_s takes its place
-  Piece8<kWide> p;
-  split8<kWide>(mag, neg, p);
-  for (int l = 0; l < mt.L; ++l) {
-    uint32_t w0, w1;
-    encode8<kWide>(p, mt.c14[l], mt.c28[l], mt.c42[l], mt.c56[l], mt.inv_m[l], mt.m_f[l], lut_s + l * kLutStride, w0, w1);
-    out_s[((2 * l) * kRowTile + r) * kStageStride + g] = w0;
-    out_s[((2 * l + 1) * kRowTile + r) * kStageStride + g] = w1;
-  }
-  __syncthreads();
-  const int row = t >> 3, word = t & 7;
-  uint8_t* dst = planes + (size_t)(i0 + row) * pitch + (size_t)(k0 / 2) + 4 * word;
-  for (int pl = 0; pl < 2 * mt.L; ++pl)
-    *reinterpret_cast<uint32_t*>(dst + (size_t)pl * plane_bytes) = out_s[(pl * kRowTile + row) * kStageStride + word];
+    Piece8<kWide> p;
+    split8<kWide>(mag, neg, p);
+    uint8_t* dst = planes + (size_t)i * pitch + (size_t)(k0 / 2) + 4 * g;
+    for (int l = 0; l < mt.L; ++l) {
+      uint32_t w0, w1;
+      encode8<kWide>(p, mt.c14[l], mt.c28[l], mt.c42[l], mt.c56[l], mt.inv_m[l], mt.m_f[l], lut_s + l * kLutStride, w0, w1);
+      *reinterpret_cast<uint32_t*>(dst + (size_t)(2 * l) * plane_bytes) = w0;
+      *reinterpret_cast<uint32_t*>(dst + (size_t)(2 * l + 1) * plane_bytes) = w1;
+    }
   }
 }
 
@@ -370,9 +366,7 @@ cudaError_t launch_encode_operand(const Geometry& g, const ModulusTable& mt, int
   const int reps = 4;
   const bool wide = g.c_bits > 56;  // integers beyond 56 bits take a fifth 14-bit piece
   if (which == 0) {
-    const size_t stage = (size_t)2 * mt.L * kRowTile * kStageStride * sizeof(uint32_t);
-    const size_t in_bytes = (size_t)kRowTileK * kRowTile * sizeof(double);
-    const size_t smem = lut_bytes + (stage > in_bytes ? stage : in_bytes);
+    const size_t smem = lut_bytes + (size_t)kRowTile * kRowStride * sizeof(double);
     auto* kernel = wide ? encode_rows_kernel<true> : encode_rows_kernel<false>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
