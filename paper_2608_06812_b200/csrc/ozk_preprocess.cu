@@ -152,8 +152,10 @@ __device__ __forceinline__ void split8(const unsigned long long (&mag)[8], const
 template <bool kWide>
 __device__ __forceinline__ void encode8(const Piece8<kWide>& p, float c14, float c28, float c42, float c56, float inv_m, float m_f,
                                         const uint16_t* __restrict__ lut_l, uint32_t& w0, uint32_t& w1) {
-  constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23: adding it rounds to an integer in the low mantissa bits
-  const char* lut_bytes = reinterpret_cast<const char*>(lut_l);
+  constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23 (bit pattern 0x4B400000): adding it rounds to an integer in the low mantissa bits
+  // shared-memory address of the table minus the bit pattern of the magic constant: one integer add turns the
+  // float below into the address of its entry
+  const uint32_t delta = (uint32_t)__cvta_generic_to_shared(lut_l) - 0x4B400000u;
   uint32_t pair[4];
 #pragma unroll
   for (int h = 0; h < 4; ++h) {
@@ -165,8 +167,8 @@ __device__ __forceinline__ void encode8(const Piece8<kWide>& p, float c14, float
       if (kWide) t = fmaf(p.x4[e], c56, t);
       const float q = fmaf(t, inv_m, kMagic) - kMagic;
       const float r = fmaf(-q, m_f, t);
-      const uint32_t off = __float_as_uint(fmaf(r, 2.0f, kMagic + 2.0f * kLutOffset)) & 0x1FFu;
-      v[o] = *reinterpret_cast<const uint16_t*>(lut_bytes + off);
+      const uint32_t addr = __float_as_uint(fmaf(r, 2.0f, kMagic + 2.0f * kLutOffset)) + delta;  // table + 2 (r + 96)
+      asm("ld.shared.u16 %0, [%1];" : "=r"(v[o]) : "r"(addr));
     }
     pair[h] = v[0] | (v[1] << 4);
   }
