@@ -170,9 +170,9 @@ __device__ __forceinline__ void encode8(const Piece8<kWide>& p, float c14, float
       const uint32_t addr = __float_as_uint(fmaf(r, 2.0f, kMagic + 2.0f * kLutOffset)) + delta;  // table + 2 (r + 96)
       asm("ld.shared.u16 %0, [%1];" : "=r"(v[o]) : "r"(addr));
     }
-    pair[h] = v[0] | (v[1] << 4);
+    pair[h] = v[1] * 16u + v[0];  // the nibbles do not overlap: one multiply-add instead of shift and or
   }
-  const uint32_t t0 = pair[0] | (pair[1] << 16), t1 = pair[2] | (pair[3] << 16);
+  const uint32_t t0 = __byte_perm(pair[0], pair[1], 0x5410), t1 = __byte_perm(pair[2], pair[3], 0x5410);
   w0 = __byte_perm(t0, t1, 0x6420);
   w1 = __byte_perm(t0, t1, 0x7531);
 }
