@@ -228,7 +228,7 @@ __global__ void __launch_bounds__(256, LEAN ? 4 : 2) crt4_kernel(const __grid_co
         for (int k = 0; k < WW; ++k) {
           const uint32_t w = ct.w[l][k];
 #pragma unroll
-          for (int e = 0; e < 4; ++e) acc[e][k] += (unsigned long long)((r4[l] >> (8 * e)) & 0xFFu) * w;
+          for (int e = 0; e < 4; ++e) acc[e][k] += (unsigned long long)__byte_perm(r4[l], 0u, 0x4440u + e) * w;
         }
       }
     }
