@@ -201,7 +201,9 @@ __device__ __forceinline__ double reconstruct_lean(const unsigned long long (&ac
   return over ? -r : r;
 }
 
-template <int WW, int NW, bool LEAN>
+// LMAX bounds the unrolled loops over the moduli (iterations beyond ct.L are predicated off but still
+// issue, so the common case of at most 19 moduli gets its own instantiation).
+template <int WW, int NW, bool LEAN, int LMAX>
 __global__ void __launch_bounds__(256, LEAN ? 4 : 2) crt4_kernel(const __grid_constant__ CrtTable ct, const uint8_t* __restrict__ res,
                                                    int64_t res_ld, size_t res_stride, const int32_t* __restrict__ s,
                                                    const int32_t* __restrict__ t, int64_t M, int64_t N,
@@ -217,12 +219,12 @@ __global__ void __launch_bounds__(256, LEAN ? 4 : 2) crt4_kernel(const __grid_co
       for (int k = 0; k < WW; ++k) acc[e][k] = 0ull;
     // all residue loads are issued before the first use: 19..27 independent 128-byte requests per
     // warp in flight instead of one (the streams of the moduli are 'res_stride' bytes apart)
-    uint32_t r4[kMaxModuli];
+    uint32_t r4[LMAX];
 #pragma unroll
-    for (int l = 0; l < kMaxModuli; ++l)
+    for (int l = 0; l < LMAX; ++l)
       r4[l] = (l < ct.L) ? __ldg(reinterpret_cast<const uint32_t*>(rp + (size_t)l * res_stride)) : 0u;
 #pragma unroll
-    for (int l = 0; l < kMaxModuli; ++l) {
+    for (int l = 0; l < LMAX; ++l) {
       if (l < ct.L) {
 #pragma unroll
         for (int k = 0; k < WW; ++k) {
@@ -365,9 +367,15 @@ cudaError_t launch_crt(const Geometry& g, const CrtTable& ct, const uint8_t* res
                     ((reinterpret_cast<uintptr_t>(s) & 15) == 0) && (g.M % 4 == 0 || s_padded);
   if (fast) {
     dim3 grid((unsigned)((g.M + 1023) / 1024), (unsigned)(g.N < 65535 ? g.N : 65535));
-#define OZK_CRT4(WW, NW) crt4_kernel<WW, NW, false><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc)
+#define OZK_CRT4(WW, NW)                                                                                             \
+  do {                                                                                                             \
+    if (ct.L <= 19)                                                                                                \
+      crt4_kernel<WW, NW, false, 19><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc);   \
+    else                                                                                                           \
+      crt4_kernel<WW, NW, false, kMaxModuli><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc); \
+  } while (0)
     if (ct.words <= 5 && ww <= 4 && ct.p_bits >= 101 && ct.p_bits <= 126)
-      crt4_kernel<4, 5, true><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc);
+      crt4_kernel<4, 5, true, 19><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc);
     else if (ct.words == 5 && ww <= 4) OZK_CRT4(4, 5);
     else if (ct.words <= 2) OZK_CRT4(2, 2);
     else if (ct.words == 3) OZK_CRT4(3, 3);
