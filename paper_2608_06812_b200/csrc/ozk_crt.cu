@@ -203,7 +203,8 @@ __device__ __forceinline__ double reconstruct_lean(const unsigned long long (&ac
 
 // LMAX bounds the unrolled loops over the moduli (iterations beyond ct.L are predicated off but still
 // issue, so the common case of at most 19 moduli gets its own instantiation).
-template <int WW, int NW, bool LEAN, int LMAX>
+// EXACT: ct.L equals LMAX, no per-modulus guard at all.
+template <int WW, int NW, bool LEAN, int LMAX, bool EXACT = false>
 __global__ void __launch_bounds__(256, LEAN ? 4 : 2) crt4_kernel(const __grid_constant__ CrtTable ct, const uint8_t* __restrict__ res,
                                                    int64_t res_ld, size_t res_stride, const int32_t* __restrict__ s,
                                                    const int32_t* __restrict__ t, int64_t M, int64_t N,
@@ -222,10 +223,10 @@ __global__ void __launch_bounds__(256, LEAN ? 4 : 2) crt4_kernel(const __grid_co
     uint32_t r4[LMAX];
 #pragma unroll
     for (int l = 0; l < LMAX; ++l)
-      r4[l] = (l < ct.L) ? __ldg(reinterpret_cast<const uint32_t*>(rp + (size_t)l * res_stride)) : 0u;
+      r4[l] = (EXACT || l < ct.L) ? __ldg(reinterpret_cast<const uint32_t*>(rp + (size_t)l * res_stride)) : 0u;
 #pragma unroll
     for (int l = 0; l < LMAX; ++l) {
-      if (l < ct.L) {
+      if (EXACT || l < ct.L) {
 #pragma unroll
         for (int k = 0; k < WW; ++k) {
           const uint32_t w = ct.w[l][k];
@@ -374,7 +375,9 @@ cudaError_t launch_crt(const Geometry& g, const CrtTable& ct, const uint8_t* res
     else                                                                                                           \
       crt4_kernel<WW, NW, false, kMaxModuli><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc); \
   } while (0)
-    if (ct.words <= 5 && ww <= 4 && ct.p_bits >= 101 && ct.p_bits <= 126)
+    if (ct.words <= 5 && ww <= 4 && ct.p_bits >= 101 && ct.p_bits <= 126 && ct.L == 19)
+      crt4_kernel<4, 5, true, 19, true><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc);
+    else if (ct.words <= 5 && ww <= 4 && ct.p_bits >= 101 && ct.p_bits <= 126)
       crt4_kernel<4, 5, true, 19><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc);
     else if (ct.words == 5 && ww <= 4) OZK_CRT4(4, 5);
     else if (ct.words <= 2) OZK_CRT4(2, 2);
