@@ -81,18 +81,38 @@ __global__ void __launch_bounds__(256) scan_rows_kernel(const double* __restrict
   if (best) atomicMax(amax + i, best);
 }
 
-// B is K x N column-major: block = (column, k slab); threads stride along k; warp-shuffle max.
+// B is K x N column-major: block = (column, k slab).  Each thread keeps four independent 16-byte loads in
+// flight; the maxima meet by warp shuffles and one shared-memory step, one atomicMax per block.
 __global__ void __launch_bounds__(256) scan_cols_kernel(const double* __restrict__ B, int64_t ldb, int64_t K, int kslab,
                                                         unsigned long long* __restrict__ amax) {
+  __shared__ unsigned long long warp_best[8];
   const int64_t j = blockIdx.x;
   const int64_t k0 = (int64_t)blockIdx.y * kslab;
   const int64_t k1 = min(K, k0 + (int64_t)kslab);
   const double* col = B + j * ldb;
   unsigned long long best = 0;
-  for (int64_t k = k0 + threadIdx.x; k < k1; k += blockDim.x) best = max(best, abs_bits(__ldg(col + k)));
+  int64_t k = k0;
+  if ((reinterpret_cast<uintptr_t>(col + k0) & 15) == 0) {  // kslab is even: every slab of an aligned column is aligned
+    const int64_t span = 8 * (int64_t)blockDim.x;           // doubles per step: four double2 per thread
+    for (; k + span <= k1; k += span) {
+      const double2* p = reinterpret_cast<const double2*>(col + k) + threadIdx.x;
+      double2 v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) v[u] = __ldg(p + u * blockDim.x);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) best = max(best, max(abs_bits(v[u].x), abs_bits(v[u].y)));
+    }
+  }
+  for (int64_t kk = k + threadIdx.x; kk < k1; kk += blockDim.x) best = max(best, abs_bits(__ldg(col + kk)));
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) best = max(best, __shfl_xor_sync(0xFFFFFFFFu, best, off));
-  if ((threadIdx.x & 31) == 0 && best) atomicMax(amax + j, best);
+  if ((threadIdx.x & 31) == 0) warp_best[threadIdx.x >> 5] = best;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+#pragma unroll
+    for (int w = 1; w < 8; ++w) best = max(best, warp_best[w]);
+    if (best) atomicMax(amax + j, best);
+  }
 }
 
 // e = floor(log2 |x|) from the bit pattern (subnormals included); shift = c - 1 - e; zero -> 0.
@@ -343,7 +363,7 @@ cudaError_t launch_scan_operand(const Geometry& g, int which, const double* X, i
     cudaError_t e = cudaMemsetAsync(amax, 0, (size_t)g.Np * sizeof(unsigned long long), st);
     if (e != cudaSuccess) return e;
     if (g.K > 0) {
-      const int kslab = 2048;
+      const int kslab = 8192;
       dim3 grid((unsigned)g.N, (unsigned)((g.K + kslab - 1) / kslab));
       scan_cols_kernel<<<grid, 256, 0, st>>>(X, ldx, g.K, kslab, amax);
     }
