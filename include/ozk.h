@@ -244,6 +244,14 @@ ozk_status ozk_stage_timing_read(float* ms3);
 ozk_status ozk_stage_mma_probe(const uint8_t* P, const uint8_t* Q, int64_t K, int scale_byte,
                                float* D, void* stream);
 
+/* Test aid for the bounded waits (every wait on a barrier or counter inside the kernels gives up after two
+ * seconds, records OZK_ERR_DEVICE_TIMEOUT in the status word and lets the kernel free its tensor memory
+ * and return): launches the probe kernel above on zero operands held in the workspace with a barrier
+ * that expects 16 bytes nobody sends, so that its wait runs out.  Afterwards ozk_get_async_status
+ * returns OZK_ERR_DEVICE_TIMEOUT once and the context and the library remain usable.  Needs a
+ * registered workspace of at least 192 KiB. */
+ozk_status ozk_stage_wait_probe(void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -51,6 +51,7 @@ SIGNATURES = {
     "ozk_stage_residue_gemm": (c_int, [c_int64, c_int64, c_int64, c_int, c_void_p, c_void_p]),
     "ozk_stage_crt": (c_int, [c_int64, c_int64, c_int64, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_int64,
                               c_void_p, c_void_p]),
+    "ozk_stage_wait_probe": (c_int, [c_void_p]),
     "ozk_row_shifts_noalloc": (c_int, [c_int64, c_int64, c_void_p, c_int64, c_int, c_void_p, c_void_p]),
     "ozk_stage_timing_enable": (c_int, [c_int]),
     "ozk_stage_timing_read": (c_int, [c_void_p]),
@@ -174,6 +175,10 @@ def ozk_stage_timing_read() -> tuple[float, float, float]:
     ms = (ctypes.c_float * 3)()
     check(lib().ozk_stage_timing_read(ms), "ozk_stage_timing_read")
     return float(ms[0]), float(ms[1]), float(ms[2])
+
+
+def ozk_stage_wait_probe(stream=0) -> int:
+    return lib().ozk_stage_wait_probe(stream)
 
 
 def ozk_row_shifts_noalloc(M, K, A, lda, num_moduli, s_out, stream=0) -> int:

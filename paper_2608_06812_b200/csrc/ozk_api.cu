@@ -342,4 +342,15 @@ ozk_status ozk_stage_mma_probe(const uint8_t* P, const uint8_t* Q, int64_t K, in
   return gemm_probe(P, Q, K, scale_byte, D, g_ws.ptr, static_cast<cudaStream_t>(stream));
 }
 
+ozk_status ozk_stage_wait_probe(void* stream) {
+  // operands and result of one 128 x 128 x 256 probe live in the workspace, past the status block and the tables
+  const size_t off_p = 64 << 10, off_q = 96 << 10, off_d = 128 << 10, need = (128 << 10) + 128 * 128 * sizeof(float);
+  if (!g_ws.ptr || g_ws.bytes < need) return OZK_ERR_WORKSPACE;
+  if (!device_is_sm100()) return OZK_ERR_UNSUPPORTED;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaMemsetAsync(g_ws.ptr + off_p, 0, 64 << 10, st) != cudaSuccess) return OZK_ERR_CUDA;
+  return gemm_probe(g_ws.ptr + off_p, g_ws.ptr + off_q, kTileKNibbles, 0x7F, reinterpret_cast<float*>(g_ws.ptr + off_d), g_ws.ptr, st,
+                    true);
+}
+
 }  // extern "C"

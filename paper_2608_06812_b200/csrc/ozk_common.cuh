@@ -100,6 +100,7 @@ ozk_status gemm_int8(const uint8_t* planes_a, const uint8_t* planes_b, int64_t M
                      int32_t* C, int64_t ldc, StatusBlock* status, cudaStream_t st);
 ozk_status gemm_oz1_passes(const uint8_t* planes_a, const uint8_t* planes_b, int64_t Mp, int64_t Np, int64_t Kp, int64_t M,
                            long long* out, int64_t out_ld, StatusBlock* status, cudaStream_t st);
-ozk_status gemm_probe(const uint8_t* P, const uint8_t* Q, int64_t K, int scale_byte, float* D, uint8_t* ws, cudaStream_t st);
+ozk_status gemm_probe(const uint8_t* P, const uint8_t* Q, int64_t K, int scale_byte, float* D, uint8_t* ws, cudaStream_t st,
+                      bool let_wait_expire = false);
 
 }  // namespace ozk

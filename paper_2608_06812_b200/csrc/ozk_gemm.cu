@@ -750,7 +750,7 @@ struct ProbeShared {
 
 __global__ void __launch_bounds__(192, 1)
 mma_probe_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_q, int kblocks,
-                 uint32_t scale_word, float* __restrict__ D, StatusBlock* status) {
+                 uint32_t scale_word, float* __restrict__ D, StatusBlock* status, uint32_t extra_tx) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   ProbeShared* sh = reinterpret_cast<ProbeShared*>(tiles + 2 * kPTileBytes);
@@ -784,7 +784,8 @@ mma_probe_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constan
     const uint32_t sf = tmem + 128;
     uint32_t phase = 0;
     for (int kb = 0; kb < kblocks; ++kb) {
-      mbar_arrive_expect_tx(smem_u32(&sh->full), 2 * kPTileBytes);
+      // extra_tx > 0 (test aid): the barrier expects bytes that nobody sends, so the bounded wait below runs out
+      mbar_arrive_expect_tx(smem_u32(&sh->full), 2 * kPTileBytes + extra_tx);
       tma_load_2d(base, &map_p, smem_u32(&sh->full), kb * kTileKBytes, 0);
       tma_load_2d(base + kPTileBytes, &map_q, smem_u32(&sh->full), kb * kTileKBytes, 0);
       const uint64_t t0 = global_timer_ns();
@@ -1037,7 +1038,8 @@ ozk_status gemm_oz1_passes(const uint8_t* planes_a, const uint8_t* planes_b, int
   return launch_limb_gemm<4, 3, W, 2, Int64BlockEpilogue>(map_p, map_q, core, ep, st);
 }
 
-ozk_status gemm_probe(const uint8_t* P, const uint8_t* Q, int64_t K, int scale_byte, float* D, uint8_t* ws, cudaStream_t st) {
+ozk_status gemm_probe(const uint8_t* P, const uint8_t* Q, int64_t K, int scale_byte, float* D, uint8_t* ws, cudaStream_t st,
+                      bool let_wait_expire) {
   CUtensorMap map_p, map_q;
   if (!make_plane_map(&map_p, P, K / 2, kTileRows, 0, 0, kTileRows)) return OZK_ERR_CUDA;
   if (!make_plane_map(&map_q, Q, K / 2, kTileRows, 0, 0, kTileRows)) return OZK_ERR_CUDA;
@@ -1046,7 +1048,7 @@ ozk_status gemm_probe(const uint8_t* P, const uint8_t* Q, int64_t K, int scale_b
     return OZK_ERR_CUDA;
   const uint32_t b = (uint32_t)(scale_byte & 0xFF);
   mma_probe_kernel<<<1, 192, smem, st>>>(map_p, map_q, (int)(K / kTileKNibbles), b * 0x01010101u, D,
-                                        reinterpret_cast<StatusBlock*>(ws));
+                                        reinterpret_cast<StatusBlock*>(ws), let_wait_expire ? 16u : 0u);
   return cudaGetLastError() == cudaSuccess ? OZK_OK : OZK_ERR_CUDA;
 }
 

@@ -83,3 +83,20 @@ def test_adversarial_accumulation_is_exact(K):
     want = reference(Pc, Qc, 0x80)
     assert np.abs(want).max() == 64 * K
     assert np.array_equal(got, want)
+
+
+def test_bounded_wait_expires_cleanly():
+    """A barrier that expects 16 bytes nobody sends: the kernel's wait gives up after its time limit, the status word
+    reads OZK_ERR_DEVICE_TIMEOUT exactly once, tensor memory is released and the next calls work as before."""
+    import time
+    from oracle import ozaki2
+    from paper_2608_06812_b200 import inputs
+    gu.ensure_workspace(1 << 20)
+    t0 = time.perf_counter()
+    ozk.check(ozk.ozk_stage_wait_probe(gu.stream()), "ozk_stage_wait_probe")
+    assert ozk.ozk_get_async_status(gu.stream()) == ozk.OZK_ERR_DEVICE_TIMEOUT
+    assert 1.0 < time.perf_counter() - t0 < 10.0             # the limit is two seconds
+    assert ozk.ozk_get_async_status(gu.stream()) == ozk.OZK_OK   # reading the status cleared it
+    A = inputs.lognormal_matrix(130, 300, 1.0, seed=1)
+    B = inputs.lognormal_matrix(300, 260, 1.0, seed=2)
+    assert gu.bits_equal(gu.dgemm(A, B, 19), ozaki2.dgemm(A, B, 19).C)
