@@ -399,7 +399,7 @@ def run_ozk(args, rank: int, local_rank: int, world: int) -> None:
             del x
         except Exception as exc:                          # out of memory on small boxes: context is optional
             line["native_fp64_tflops_context"] = f"unavailable: {type(exc).__name__}"
-    if not args.no_cpu_baseline:
+    if not args.no_cpu_baseline and world == 1:            # the oracle leg runs on rank 0 of a single-GPU run only
         tf, secs, sample, threads = oracle_sample_tflops(A, B, L, 512)
         line["cpu_baseline"] = {"value": tf, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample, "seconds": secs}
     print(json.dumps(line), flush=True)
