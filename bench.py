@@ -34,7 +34,7 @@ PAPER_TOTAL_TFLOPS = {4096: 10.81, 8192: 13.52, 16384: 15.26}   # the paper's en
 FP4_PER_BF16 = 4.0                                               # nominal dense FP4 : BF16 ratio on B200
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the limb GEMM, from ncu captures of this
 # command at the same size (see profiles/): (size, moduli) -> bytes
-DRAM_TRAFFIC_BYTES = {(16384, 19): 61.0e9 + 5.1e9, (4096, 19): 0.638e9 + 0.301e9}
+DRAM_TRAFFIC_BYTES = {(16384, 19): 53.4e9 + 5.1e9, (4096, 19): 0.638e9 + 0.301e9}
 KERNELS_PER_STEP = 9   # lut, scan_rows, scan_cols, 2 x finalize, encode_rows, encode_cols, limb GEMM, CRT
 
 

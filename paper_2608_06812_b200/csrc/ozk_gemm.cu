@@ -603,6 +603,7 @@ residue_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
+      const uint64_t pol_keep = l2_policy_evict_last(), pol_stream = l2_policy_evict_first();
       for (int item = pair; item < total_items && ok; item += npairs) {
         int l, tp, tq;
         decode_item(p, item, l, tp, tq);
@@ -621,15 +622,17 @@ residue_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
           if (rank == 0) mbar_arrive_expect_tx(smem_u32(&sh->full[stage]), 2 * kPairStageBytes);
           const int x = kb * kTileKBytes;
           const int prow = (2 * tp + (int)rank) * kTileRows;
-          tma_load_3d_pair(dst + 0 * kPTileBytes, &map_p, leader_full, x, prow, 2 * l + 0);
-          tma_load_3d_pair(dst + 1 * kPTileBytes, &map_p, leader_full, x, prow, 2 * l + 1);
+          // L2 priorities: the column-side tiles of the band are reused by every row tile of the band and
+          // should stay; the row-side tiles are shared only within the current wave and may leave first
+          tma_load_3d_pair_hint(dst + 0 * kPTileBytes, &map_p, leader_full, x, prow, 2 * l + 0, pol_keep);
+          tma_load_3d_pair_hint(dst + 1 * kPTileBytes, &map_p, leader_full, x, prow, 2 * l + 1, pol_keep);
           if (p.skip_top_first && l == 0) {
             // m = 169 needs p0 q0, p0 q1, p1 q0 only: three 128-column instructions, for which this CTA
             // supplies rows [64 rank, 64 rank + 64) of q0 and of q1 instead of all of one of them
             tma_load_3d_pair(dst + 2 * kPTileBytes, &map_qh, leader_full, x, tq * W + 64 * (int)rank, 0);
             tma_load_3d_pair(dst + 2 * kPTileBytes + kPTileBytes / 2, &map_qh, leader_full, x, tq * W + 64 * (int)rank, 1);
           } else {
-            tma_load_3d_pair(dst + 2 * kPTileBytes, &map_q, leader_full, x, tq * W, 2 * l + (int)rank);
+            tma_load_3d_pair_hint(dst + 2 * kPTileBytes, &map_q, leader_full, x, tq * W, 2 * l + (int)rank, pol_stream);
           }
           if (++stage == kPairStages) stage = 0, phase ^= 1u;
         }
