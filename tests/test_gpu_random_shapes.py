@@ -97,3 +97,18 @@ def test_cuda_graph_capture_and_replay():
     torch.cuda.synchronize()
     assert gu.bits_equal(gu.from_dev_colmajor(dC, M, N), ozaki2.dgemm(A2, B2, L).C)
     ozk.check(ozk.ozk_get_async_status(gu.stream()), "status")
+
+
+@pytest.mark.parametrize("M,N,K", [(70000, 40, 96), (40, 60000, 96), (66000, 300, 20)])
+def test_very_tall_and_very_wide_outputs(M, N, K):
+    """Grid dimensions beyond 65535 blocks in either direction; sampled rows and columns against the oracle
+    (shifts are per row / per column, so sub-matrices reproduce the same elements)."""
+    L = 19
+    A = inputs.lognormal_matrix(M, K, 1.0, seed=M % 97)
+    B = inputs.lognormal_matrix(K, N, 1.0, seed=N % 89)
+    C = gu.dgemm(A, B, L)
+    rng = np.random.default_rng(5)
+    rows = np.unique(np.concatenate([[0, 1, M - 2, M - 1], rng.integers(0, M, 60)]))
+    cols = np.unique(np.concatenate([[0, 1, N - 2, N - 1], rng.integers(0, N, 60)]))
+    assert gu.bits_equal(C[np.ix_(rows, cols)], ozaki2.dgemm(A[rows], B[:, cols], L).C)
+    assert np.isfinite(C).all()
