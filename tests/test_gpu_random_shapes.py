@@ -112,3 +112,39 @@ def test_very_tall_and_very_wide_outputs(M, N, K):
     cols = np.unique(np.concatenate([[0, 1, N - 2, N - 1], rng.integers(0, N, 60)]))
     assert gu.bits_equal(C[np.ix_(rows, cols)], ozaki2.dgemm(A[rows], B[:, cols], L).C)
     assert np.isfinite(C).all()
+
+
+def test_random_shapes_with_special_inputs():
+    """Random shapes combined with zero rows / columns, global scalings across the FP64 exponent range, rows and
+    columns in the subnormal range, integer data, single huge columns, and (for L >= 19) widths beyond 53 bits."""
+    from oracle import moduli
+    rng = np.random.default_rng(77)
+    done = 0
+    while done < 40:
+        M, N, K = int(rng.integers(1, 400)), int(rng.integers(1, 500)), int(rng.integers(1, 1500))
+        L = int(rng.integers(2, 28))
+        if moduli.capacity_bits(K, L) < 1:
+            continue
+        phi = float(rng.choice([0.5, 1.0, 4.0, 8.0]))
+        A = inputs.lognormal_matrix(M, K, phi, seed=int(rng.integers(1 << 30)))
+        B = inputs.lognormal_matrix(K, N, phi, seed=int(rng.integers(1 << 30)))
+        kind = done % 6
+        if kind == 1:
+            A[rng.integers(0, M), :] = 0.0
+            B[:, rng.integers(0, N)] = 0.0
+        elif kind == 2:
+            A *= 2.0 ** int(rng.integers(-900, 900))
+        elif kind == 3:
+            A[rng.integers(0, M), :] *= 2.0 ** -1040
+            B[:, rng.integers(0, N)] *= 2.0 ** -1030
+        elif kind == 4:
+            A, B = np.rint(A * 1000), np.rint(B * 1000)
+        elif kind == 5:
+            A[:, rng.integers(0, K)] *= 2.0 ** 60
+        max_bits = int(rng.integers(54, 63)) if (L >= 19 and rng.random() < 0.3) else None
+        with np.errstate(all="ignore"):
+            ref = ozaki2.dgemm(A, B, L, max_bits=max_bits or 53).C
+        C = gu.dgemm(A, B, L, lda=M + int(rng.integers(0, 4)), ldb=K + int(rng.integers(0, 4)), ldc=M + int(rng.integers(0, 4)),
+                     max_bits=max_bits)
+        assert gu.bits_equal(C, ref), (M, N, K, L, phi, kind, max_bits)
+        done += 1
