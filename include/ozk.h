@@ -79,7 +79,7 @@ size_t ozk_dgemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int num_moduli
 size_t ozk_igemm_i8_workspace_bytes(int64_t M, int64_t N, int64_t K);
 
 /* Registers the caller-owned device buffer used by all later compute calls of this
- * process.  `dev_ptr` must be 1024-byte aligned (any cudaMalloc / PyTorch allocation is).
+ * process.  `dev_ptr` must be 256-byte aligned (any cudaMalloc / PyTorch allocation is).
  * The library never frees it.  Passing NULL unregisters. */
 ozk_status ozk_set_workspace(void* dev_ptr, size_t bytes);
 

@@ -176,7 +176,7 @@ size_t ozk_dgemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int num_moduli
 }
 
 ozk_status ozk_set_workspace(void* dev_ptr, size_t bytes) {
-  if (dev_ptr && (reinterpret_cast<uintptr_t>(dev_ptr) & 1023)) return OZK_ERR_INVALID_ARG;
+  if (dev_ptr && (reinterpret_cast<uintptr_t>(dev_ptr) & 255)) return OZK_ERR_INVALID_ARG;
   g_ws.ptr = static_cast<uint8_t*>(dev_ptr);
   g_ws.bytes = dev_ptr ? bytes : 0;
   if (dev_ptr) {

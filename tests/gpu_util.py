@@ -13,16 +13,22 @@ def stream() -> int:
     return torch.cuda.current_stream().cuda_stream
 
 
+def _register(buf: torch.Tensor, nbytes: int) -> None:
+    """Registers the buffer from an odd multiple of 256 bytes on: the least alignment the library accepts."""
+    offset = (-buf.data_ptr()) % 512 + 256
+    ozk.check(ozk.ozk_set_workspace(buf.data_ptr() + offset, nbytes), "ozk_set_workspace")
+
+
 def ensure_workspace(nbytes: int) -> None:
     """One growing device workspace shared by all tests of a process."""
     nbytes = max(int(nbytes), 1 << 20)
     buf = _ws["buf"]
-    if buf is None or buf.numel() < nbytes:
+    if buf is None or buf.numel() < nbytes + 1024:
         torch.cuda.synchronize()
         _ws["buf"] = None
-        buf = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+        buf = torch.empty(nbytes + 1024, dtype=torch.uint8, device="cuda")
         _ws["buf"] = buf
-        ozk.check(ozk.ozk_set_workspace(buf.data_ptr(), buf.numel()), "ozk_set_workspace")
+        _register(buf, buf.numel() - 1024)
 
 
 def register_small_workspace(nbytes: int = 1 << 20) -> None:
@@ -30,8 +36,8 @@ def register_small_workspace(nbytes: int = 1 << 20) -> None:
     the next ensure_workspace() call replaces it."""
     torch.cuda.synchronize()
     _ws["buf"] = None
-    buf = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
-    ozk.check(ozk.ozk_set_workspace(buf.data_ptr(), buf.numel()), "ozk_set_workspace")
+    buf = torch.empty(nbytes + 1024, dtype=torch.uint8, device="cuda")
+    _register(buf, nbytes)
     _ws["small"] = buf
 
 

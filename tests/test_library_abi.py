@@ -70,6 +70,6 @@ def test_argument_errors_need_no_gpu():
     assert ozk.ozk_dgemm(8, 8, ozk.OZK_MAX_K + 1, None, 8, None, ozk.OZK_MAX_K + 1, None, 8, 19, None) == ozk.OZK_ERR_UNSUPPORTED
     assert ozk.ozk_dgemm(8, 8, 8, None, 8, None, 8, None, 8, 1, None) == ozk.OZK_ERR_INVALID_ARG
     assert ozk.ozk_dgemm(-8, 8, 8, None, 8, None, 8, None, 8, 19, None) == ozk.OZK_ERR_INVALID_ARG
-    assert ozk.ozk_set_workspace(12345, 1 << 20) == ozk.OZK_ERR_INVALID_ARG       # not 1024-aligned
+    assert ozk.ozk_set_workspace(12345, 1 << 20) == ozk.OZK_ERR_INVALID_ARG       # not 256-byte aligned
     assert "workspace" in ozk.ozk_status_string(ozk.OZK_ERR_WORKSPACE)
     assert "sm_100a" in ozk.ozk_version()
