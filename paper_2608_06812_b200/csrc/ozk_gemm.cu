@@ -988,9 +988,12 @@ ozk_status gemm_residues(const Geometry& g, const ModulusTable& mt, uint8_t* ws,
 }
 
 // INT8 path: C (int32, column-major) from three limb planes per operand.
+// INT8 path: C (int32, column-major) from three limb planes per operand.  128 x 64 tiles: five accumulators of
+// 64 columns, three N = 192 instructions per K step, and three 72 KiB stages (an 80-wide tile leaves room for two
+// stages only and measured 5 to 11 % slower).
 ozk_status gemm_int8(const uint8_t* planes_a, const uint8_t* planes_b, int64_t M, int64_t N, int64_t Mp, int64_t Np, int64_t Kp,
                      int32_t* C, int64_t ldc, StatusBlock* status, cudaStream_t st) {
-  constexpr int W = 80;
+  constexpr int W = 64;
   CUtensorMap map_p, map_q;
   if (!make_plane_map(&map_p, planes_b, Kp / 2, Np, 3, (size_t)Np * (size_t)(Kp / 2), kTileRows)) return OZK_ERR_CUDA;
   if (!make_plane_map(&map_q, planes_a, Kp / 2, Mp, 3, (size_t)Mp * (size_t)(Kp / 2), W)) return OZK_ERR_CUDA;
@@ -1011,7 +1014,7 @@ ozk_status gemm_int8(const uint8_t* planes_a, const uint8_t* planes_b, int64_t M
   ep.ldc = ldc;
   ep.M = M;
   ep.N = N;
-  return launch_limb_gemm<3, 3, W, 2, Int32Epilogue>(map_p, map_q, core, ep, st);
+  return launch_limb_gemm<3, 3, W, 3, Int32Epilogue>(map_p, map_q, core, ep, st);
 }
 
 // Scheme-I passes: 16 row-side limb planes (the 16th all zero) in 4 groups of 4, 15 column-side planes in
