@@ -375,9 +375,14 @@ cudaError_t launch_crt(const Geometry& g, const CrtTable& ct, const uint8_t* res
     else                                                                                                           \
       crt4_kernel<WW, NW, false, kMaxModuli><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc); \
   } while (0)
-    if (ct.words <= 5 && ww <= 4 && ct.p_bits >= 101 && ct.p_bits <= 126 && ct.L == 19)
-      crt4_kernel<4, 5, true, 19, true><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc);
-    else if (ct.words <= 5 && ww <= 4 && ct.p_bits >= 101 && ct.p_bits <= 126)
+    const bool lean = ct.words <= 5 && ww <= 4 && ct.p_bits >= 101 && ct.p_bits <= 126;  // 16 to 19 moduli
+#define OZK_CRT_LEAN(LL) crt4_kernel<4, 5, true, LL, true><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc)
+    if (lean && ct.L == 19) OZK_CRT_LEAN(19);
+    else if (lean && ct.L == 18) OZK_CRT_LEAN(18);
+    else if (lean && ct.L == 17) OZK_CRT_LEAN(17);
+    else if (lean && ct.L == 16) OZK_CRT_LEAN(16);
+#undef OZK_CRT_LEAN
+    else if (lean)
       crt4_kernel<4, 5, true, 19><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc);
     else if (ct.words == 5 && ww <= 4) OZK_CRT4(4, 5);
     else if (ct.words <= 2) OZK_CRT4(2, 2);
