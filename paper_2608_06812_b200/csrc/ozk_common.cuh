@@ -63,6 +63,7 @@ struct CrtTable {
   uint32_t halfP[kCrtWords];               // floor(P / 2)
   double inv_P;                            // 1 / P rounded to double
   double q_scale;                          // (2^96 / P) (1 - 2^-30): quotient estimate from the words above bit 96
+  double q_scale128;                       // (2^128 / P) (1 - 2^-30): the same from the words above bit 128
   int p_bits;                              // bit length of P
 };
 

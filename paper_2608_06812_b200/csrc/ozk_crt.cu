@@ -201,10 +201,81 @@ __device__ __forceinline__ double reconstruct_lean(const unsigned long long (&ac
   return over ? -r : r;
 }
 
+// The same for 2^128 <= P < 2^158 (20 to 23 moduli): S has six words and arrives as five 64-bit column sums,
+// the quotient estimate uses the words above bit 128 (q_scale128 = (2^128 / P)(1 - 2^-30); the part of S below
+// bit 128 is less than P, so the estimate is again the true quotient or one below it), x has five words.
+__device__ __forceinline__ double reconstruct_lean5(const unsigned long long (&acc)[5], const CrtTable& ct, int shift) {
+  const uint32_t a0l = (uint32_t)acc[0], a0h = (uint32_t)(acc[0] >> 32), a1l = (uint32_t)acc[1], a1h = (uint32_t)(acc[1] >> 32);
+  const uint32_t a2l = (uint32_t)acc[2], a2h = (uint32_t)(acc[2] >> 32), a3l = (uint32_t)acc[3], a3h = (uint32_t)(acc[3] >> 32);
+  const uint32_t a4l = (uint32_t)acc[4], a4h = (uint32_t)(acc[4] >> 32);
+  uint32_t S1, S2, S3, S4, S5;
+  asm("add.cc.u32 %0, %5, %6;\n\t"
+      "addc.cc.u32 %1, %7, %8;\n\t"
+      "addc.cc.u32 %2, %9, %10;\n\t"
+      "addc.cc.u32 %3, %11, %12;\n\t"
+      "addc.u32 %4, %13, 0;"
+      : "=r"(S1), "=r"(S2), "=r"(S3), "=r"(S4), "=r"(S5)
+      : "r"(a0h), "r"(a1l), "r"(a1h), "r"(a2l), "r"(a2h), "r"(a3l), "r"(a3h), "r"(a4l), "r"(a4h));
+  const uint32_t S0 = a0l;
+  const unsigned long long top = ((unsigned long long)S5 << 32) | S4;
+  const uint32_t q = __double2uint_rz(__ull2double_rz(top) * ct.q_scale128);
+  const unsigned long long m0 = (unsigned long long)q * ct.P[0];
+  const unsigned long long m1 = (unsigned long long)q * ct.P[1] + (m0 >> 32);
+  const unsigned long long m2 = (unsigned long long)q * ct.P[2] + (m1 >> 32);
+  const unsigned long long m3 = (unsigned long long)q * ct.P[3] + (m2 >> 32);
+  const unsigned long long m4 = (unsigned long long)q * ct.P[4] + (m3 >> 32);
+  uint32_t x0, x1, x2, x3, x4;
+  asm("sub.cc.u32 %0, %5, %10;\n\t"
+      "subc.cc.u32 %1, %6, %11;\n\t"
+      "subc.cc.u32 %2, %7, %12;\n\t"
+      "subc.cc.u32 %3, %8, %13;\n\t"
+      "subc.u32 %4, %9, %14;"
+      : "=r"(x0), "=r"(x1), "=r"(x2), "=r"(x3), "=r"(x4)
+      : "r"(S0), "r"(S1), "r"(S2), "r"(S3), "r"(S4), "r"((uint32_t)m0), "r"((uint32_t)m1), "r"((uint32_t)m2), "r"((uint32_t)m3),
+        "r"((uint32_t)m4));
+  const uint32_t P0 = ct.P[0], P1 = ct.P[1], P2 = ct.P[2], P3 = ct.P[3], P4 = ct.P[4];
+  uint32_t d0, d1, d2, d3, d4, below;  // d = x - P; below = all ones if x < P
+  asm("sub.cc.u32 %0, %6, %11;\n\t"
+      "subc.cc.u32 %1, %7, %12;\n\t"
+      "subc.cc.u32 %2, %8, %13;\n\t"
+      "subc.cc.u32 %3, %9, %14;\n\t"
+      "subc.cc.u32 %4, %10, %15;\n\t"
+      "subc.u32 %5, 0, 0;"
+      : "=r"(d0), "=r"(d1), "=r"(d2), "=r"(d3), "=r"(d4), "=r"(below)
+      : "r"(x0), "r"(x1), "r"(x2), "r"(x3), "r"(x4), "r"(P0), "r"(P1), "r"(P2), "r"(P3), "r"(P4));
+  if (!below) x0 = d0, x1 = d1, x2 = d2, x3 = d3, x4 = d4;
+  uint32_t e0, e1, e2, e3, e4;  // e = P - x
+  asm("sub.cc.u32 %0, %5, %10;\n\t"
+      "subc.cc.u32 %1, %6, %11;\n\t"
+      "subc.cc.u32 %2, %7, %12;\n\t"
+      "subc.cc.u32 %3, %8, %13;\n\t"
+      "subc.u32 %4, %9, %14;"
+      : "=r"(e0), "=r"(e1), "=r"(e2), "=r"(e3), "=r"(e4)
+      : "r"(P0), "r"(P1), "r"(P2), "r"(P3), "r"(P4), "r"(x0), "r"(x1), "r"(x2), "r"(x3), "r"(x4));
+  uint32_t u0, u1, u2, u3, u4, over;  // halfP - x borrows exactly when x > P/2
+  asm("sub.cc.u32 %0, %6, %11;\n\t"
+      "subc.cc.u32 %1, %7, %12;\n\t"
+      "subc.cc.u32 %2, %8, %13;\n\t"
+      "subc.cc.u32 %3, %9, %14;\n\t"
+      "subc.cc.u32 %4, %10, %15;\n\t"
+      "subc.u32 %5, 0, 0;"
+      : "=r"(u0), "=r"(u1), "=r"(u2), "=r"(u3), "=r"(u4), "=r"(over)
+      : "r"(ct.halfP[0]), "r"(ct.halfP[1]), "r"(ct.halfP[2]), "r"(ct.halfP[3]), "r"(ct.halfP[4]), "r"(x0), "r"(x1), "r"(x2), "r"(x3),
+        "r"(x4));
+  uint32_t mag[5];
+  mag[0] = over ? e0 : x0;
+  mag[1] = over ? e1 : x1;
+  mag[2] = over ? e2 : x2;
+  mag[3] = over ? e3 : x3;
+  mag[4] = over ? e4 : x4;
+  const double r = round_scaled_fast<5>(mag, shift);
+  return over ? -r : r;
+}
+
 // LMAX bounds the unrolled loops over the moduli (iterations beyond ct.L are predicated off but still
 // issue, so the common case of at most 19 moduli gets its own instantiation).
 // EXACT: ct.L equals LMAX, no per-modulus guard at all.
-template <int WW, int NW, bool LEAN, int LMAX, bool EXACT = false>
+template <int WW, int NW, int LEAN, int LMAX, bool EXACT = false>
 __global__ void __launch_bounds__(256, LEAN ? 4 : 2) crt4_kernel(const __grid_constant__ CrtTable ct, const uint8_t* __restrict__ res,
                                                    int64_t res_ld, size_t res_stride, const int32_t* __restrict__ s,
                                                    const int32_t* __restrict__ t, int64_t M, int64_t N,
@@ -241,12 +312,20 @@ __global__ void __launch_bounds__(256, LEAN ? 4 : 2) crt4_kernel(const __grid_co
     double out[4];
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-      if constexpr (LEAN) {
-        static_assert(!LEAN || (WW == 4 && NW == 5), "the lean tail is written for 4 weight words, 5 sum words");
+      if constexpr (LEAN == 4) {
+        static_assert(LEAN != 4 || (WW == 4 && NW == 5), "this lean tail is written for 4 weight words, 5 sum words");
         unsigned long long a4[4];
 #pragma unroll
         for (int k = 0; k < 4; ++k) a4[k] = acc[e][k < WW ? k : 0];
         out[e] = reconstruct_lean(a4, ct, sh[e]);
+        continue;
+      }
+      if constexpr (LEAN == 5) {
+        static_assert(LEAN != 5 || (WW == 5 && NW == 6), "this lean tail is written for 5 weight words, 6 sum words");
+        unsigned long long a5[5];
+#pragma unroll
+        for (int k = 0; k < 5; ++k) a5[k] = acc[e][k < WW ? k : 0];
+        out[e] = reconstruct_lean5(a5, ct, sh[e]);
         continue;
       }
       uint32_t S[NW];
@@ -371,19 +450,27 @@ cudaError_t launch_crt(const Geometry& g, const CrtTable& ct, const uint8_t* res
 #define OZK_CRT4(WW, NW)                                                                                             \
   do {                                                                                                             \
     if (ct.L <= 19)                                                                                                \
-      crt4_kernel<WW, NW, false, 19><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc);   \
+      crt4_kernel<WW, NW, 0, 19><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc);   \
     else                                                                                                           \
-      crt4_kernel<WW, NW, false, kMaxModuli><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc); \
+      crt4_kernel<WW, NW, 0, kMaxModuli><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc); \
   } while (0)
     const bool lean = ct.words <= 5 && ww <= 4 && ct.p_bits >= 101 && ct.p_bits <= 126;  // 16 to 19 moduli
-#define OZK_CRT_LEAN(LL) crt4_kernel<4, 5, true, LL, true><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc)
+    const bool lean5 = ct.words <= 6 && ww <= 5 && ct.p_bits >= 129 && ct.p_bits <= 158;  // 20 to 23 moduli
+#define OZK_CRT_LEAN5(LL) crt4_kernel<5, 6, 5, LL, true><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc)
+    if (lean5 && ct.L == 20) OZK_CRT_LEAN5(20);
+    else if (lean5 && ct.L == 21) OZK_CRT_LEAN5(21);
+    else if (lean5 && ct.L == 22) OZK_CRT_LEAN5(22);
+    else if (lean5 && ct.L == 23) OZK_CRT_LEAN5(23);
+#undef OZK_CRT_LEAN5
+    else
+#define OZK_CRT_LEAN(LL) crt4_kernel<4, 5, 4, LL, true><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc)
     if (lean && ct.L == 19) OZK_CRT_LEAN(19);
     else if (lean && ct.L == 18) OZK_CRT_LEAN(18);
     else if (lean && ct.L == 17) OZK_CRT_LEAN(17);
     else if (lean && ct.L == 16) OZK_CRT_LEAN(16);
 #undef OZK_CRT_LEAN
     else if (lean)
-      crt4_kernel<4, 5, true, 19><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc);
+      crt4_kernel<4, 5, 4, 19><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc);
     else if (ct.words == 5 && ww <= 4) OZK_CRT4(4, 5);
     else if (ct.words <= 2) OZK_CRT4(2, 2);
     else if (ct.words == 3) OZK_CRT4(3, 3);

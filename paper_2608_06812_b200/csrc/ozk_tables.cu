@@ -255,6 +255,7 @@ bool build_crt_table(int L, CrtTable* t) {
   for (int i = 0; i < kCrtWords; ++i) t->halfP[i] = h.w[i];
   t->inv_P = 1.0 / big_to_double(P);
   t->q_scale = ldexp(t->inv_P, 96) * (1.0 - ldexp(1.0, -30));
+  t->q_scale128 = ldexp(t->inv_P, 128) * (1.0 - ldexp(1.0, -30));
   t->p_bits = big_bits(P);
   return true;
 }
