@@ -3,6 +3,8 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <atomic>
+
 #include "ozk_common.cuh"
 
 namespace ozk {
@@ -86,17 +88,6 @@ ozk_status check_common(int64_t M, int64_t N, int64_t K, int L, Geometry* g, int
   return OZK_OK;
 }
 
-bool device_is_sm100() {
-  static int cached = -1;
-  if (cached < 0) {
-    int dev = 0, major = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return false;
-    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return false;
-    cached = (major == 10) ? 1 : 0;
-  }
-  return cached == 1;
-}
-
 ozk_status run_preprocess(const Geometry& g, const ModulusTable& mt, const double* A, int64_t lda, const double* B,
                           int64_t ldb, int64_t* At_out, int64_t* Bt_out, cudaStream_t st) {
   if (launch_build_lut(mt, g_ws.ptr + g.off_lut, st) != cudaSuccess) return OZK_ERR_CUDA;
@@ -109,6 +100,37 @@ ozk_status run_preprocess(const Geometry& g, const ModulusTable& mt, const doubl
 
 bool make_geometry(int64_t M, int64_t N, int64_t K, int L, Geometry* g, int max_bits) {
   return make_geometry_impl(M, N, K, L, g, max_bits);
+}
+
+// Facts about the current device, looked up once per device ordinal (a process may use several devices).
+namespace {
+constexpr int kMaxDevices = 64;
+struct DeviceFacts {
+  std::atomic<int> sm_count{-1};
+  std::atomic<int> major{-1};
+};
+DeviceFacts g_device_facts[kMaxDevices];
+DeviceFacts* current_device_facts() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  DeviceFacts* f = &g_device_facts[dev];
+  if (f->sm_count.load(std::memory_order_acquire) < 0) {
+    int n = 0, major = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return nullptr;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return nullptr;
+    f->major.store(major, std::memory_order_release);
+    f->sm_count.store(n, std::memory_order_release);
+  }
+  return f;
+}
+}  // namespace
+int device_sm_count() {
+  DeviceFacts* f = current_device_facts();
+  return f ? f->sm_count.load(std::memory_order_acquire) : 0;
+}
+bool device_is_sm100() {
+  DeviceFacts* f = current_device_facts();
+  return f && f->major.load(std::memory_order_acquire) == 10;
 }
 
 // Limb GEMM over all of K: one launch per k range of at most kChunkK (the FP32 accumulators stay exact

@@ -65,7 +65,16 @@ struct CrtTable {
   double q_scale;                          // (2^96 / P) (1 - 2^-30): quotient estimate from the words above bit 96
   double q_scale128;                       // (2^128 / P) (1 - 2^-30): the same from the words above bit 128
   int p_bits;                              // bit length of P
+  // B fragments of the reconstruction kernel's mma.sync.m16n8k32 (u8): tile, lane, register.  Lane (g, q) holds
+  // column g of the tile; byte n of register 0 / 1 is the digit for modulus q + 4 n / q + 16 + 4 n.  Column c
+  // of tile 0 carries digit (byte) 4 (c / 2) + c % 2 of the weights, of tile 1 digit 4 (c / 2) + 2 + c % 2, of
+  // tile 2 digit 16 + c.
+  uint32_t bfrag[3][32][2];
 };
+
+// per-device facts, cached per device ordinal (ozk_api.cu)
+int device_sm_count();      // multiprocessors of the current device (0 on error)
+bool device_is_sm100();     // compute capability 10.x
 
 // registered workspace and layout (ozk_api.cu)
 uint8_t* workspace_ptr();

@@ -7,6 +7,8 @@
 //                      C = RN_even(x * 2^-(s_i + t_j))
 // Everything is column-major with the row index fastest, so one thread per element
 // coalesces the residue bytes, the shifts and the FP64 stores alike.
+#include <algorithm>
+
 #include "ozk_common.cuh"
 #include "ozk_round.cuh"
 
@@ -16,11 +18,11 @@ namespace {
 template <int NW>
 __global__ void __launch_bounds__(256) crt_kernel(CrtTable ct, const uint8_t* __restrict__ res, int64_t res_ld,
                                                   size_t res_stride, const int32_t* __restrict__ s,
-                                                  const int32_t* __restrict__ t, int64_t M, double* __restrict__ C,
-                                                  int64_t ldc, uint32_t* __restrict__ x_out) {
+                                                  const int32_t* __restrict__ t, int64_t M, int64_t N,
+                                                  double* __restrict__ C, int64_t ldc, uint32_t* __restrict__ x_out) {
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  const int64_t j = blockIdx.y;
   if (i >= M) return;
+  for (int64_t j = blockIdx.y; j < N; j += gridDim.y) {
   const uint8_t* rp = res + (size_t)j * (size_t)res_ld + (size_t)i;
   uint32_t S[NW];
 #pragma unroll
@@ -92,6 +94,7 @@ __global__ void __launch_bounds__(256) crt_kernel(CrtTable ct, const uint8_t* __
       }
       xo[k] = w;
     }
+  }
   }
 }
 
@@ -272,120 +275,235 @@ __device__ __forceinline__ double reconstruct_lean5(const unsigned long long (&a
   return over ? -r : r;
 }
 
-// LMAX bounds the unrolled loops over the moduli (iterations beyond ct.L are predicated off but still
-// issue, so the common case of at most 19 moduli gets its own instantiation).
-// EXACT: ct.L equals LMAX, no per-modulus guard at all.
-template <int WW, int NW, int LEAN, int LMAX, bool EXACT = false>
-__global__ void __launch_bounds__(256, LEAN ? 4 : 2) crt4_kernel(const __grid_constant__ CrtTable ct, const uint8_t* __restrict__ res,
-                                                   int64_t res_ld, size_t res_stride, const int32_t* __restrict__ s,
-                                                   const int32_t* __restrict__ t, int64_t M, int64_t N,
-                                                   double* __restrict__ C, int64_t ldc) {
-  const int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
-  if (i >= M) return;
-  for (int64_t j = blockIdx.y; j < N; j += gridDim.y) {
-    const uint8_t* rp = res + (size_t)j * (size_t)res_ld + (size_t)i;
-    unsigned long long acc[4][WW];
+// Tail shared by the reconstruction kernels: from the 64-bit column sums acc[k] = sum_l r_l w_l[k] (weight
+// word k, no carries yet) to C_ij.  LEAN = 4 / 5 selects the carry-chain tails above, 0 the generic
+// multiword route (any modulus count).
+template <int WW, int NW, int LEAN>
+__device__ __forceinline__ double finish_element(const unsigned long long (&acc)[WW], const CrtTable& ct, int shift) {
+  if constexpr (LEAN == 4) {
+    static_assert(LEAN != 4 || (WW == 4 && NW == 5), "this lean tail is written for 4 weight words, 5 sum words");
+    unsigned long long a4[4];
 #pragma unroll
-    for (int e = 0; e < 4; ++e)
+    for (int k = 0; k < 4; ++k) a4[k] = acc[k < WW ? k : 0];
+    return reconstruct_lean(a4, ct, shift);
+  } else if constexpr (LEAN == 5) {
+    static_assert(LEAN != 5 || (WW >= 5 && NW == 6), "this lean tail is written for 5 weight words, 6 sum words");
+    unsigned long long a5[5];
 #pragma unroll
-      for (int k = 0; k < WW; ++k) acc[e][k] = 0ull;
-    // all residue loads are issued before the first use: 19..27 independent 128-byte requests per
-    // warp in flight instead of one (the streams of the moduli are 'res_stride' bytes apart)
-    uint32_t r4[LMAX];
+    for (int k = 0; k < 5; ++k) a5[k] = acc[k < WW ? k : 0];
+    return reconstruct_lean5(a5, ct, shift);
+  } else {
+    uint32_t S[NW];
+    unsigned long long carry = 0ull;
 #pragma unroll
-    for (int l = 0; l < LMAX; ++l)
-      r4[l] = (EXACT || l < ct.L) ? __ldg(reinterpret_cast<const uint32_t*>(rp + (size_t)l * res_stride)) : 0u;
+    for (int k = 0; k < NW; ++k) {
+      const unsigned long long v = (k < WW ? acc[k < WW ? k : 0] : 0ull) + carry;
+      S[k] = (uint32_t)v;
+      carry = v >> 32;
+    }
+    // quotient estimate from the three top words (truncation error << 1), exact correction
+    double Sd = (double)S[NW - 1];
+    if (NW >= 2) Sd = Sd * 4294967296.0 + (double)S[NW - 2];
+    if (NW >= 3) Sd = Sd * 4294967296.0 + (double)S[NW - 3];
+    if (NW > 3) Sd *= __longlong_as_double((long long)(1023 + 32 * (NW - 3)) << 52);
+    const uint32_t q = (uint32_t)(Sd * ct.inv_P);
+    uint32_t borrow = 0, mc = 0;
 #pragma unroll
-    for (int l = 0; l < LMAX; ++l) {
-      if (EXACT || l < ct.L) {
+    for (int k = 0; k < NW; ++k) {
+      const unsigned long long prod = (unsigned long long)q * ct.P[k] + mc;
+      mc = (uint32_t)(prod >> 32);
+      const unsigned long long d = (unsigned long long)S[k] - (uint32_t)prod - borrow;
+      S[k] = (uint32_t)d;
+      borrow = (uint32_t)(d >> 63);
+    }
+    uint32_t signw = 0u - mc - borrow;
+#pragma unroll 1
+    for (int it = 0; it < 2 && signw != 0; ++it) {
+      uint32_t c2 = 0;
 #pragma unroll
-        for (int k = 0; k < WW; ++k) {
-          const uint32_t w = ct.w[l][k];
+      for (int k = 0; k < NW; ++k) {
+        const unsigned long long v = (unsigned long long)S[k] + ct.P[k] + c2;
+        S[k] = (uint32_t)v;
+        c2 = (uint32_t)(v >> 32);
+      }
+      signw += c2;
+    }
+#pragma unroll 1
+    for (int it = 0; it < 2 && ge<NW>(S, ct.P); ++it) sub_in_place<NW>(S, ct.P);
+    bool neg = false;
+    if (gt<NW>(S, ct.halfP)) {
+      uint32_t tmp[NW];
 #pragma unroll
-          for (int e = 0; e < 4; ++e) acc[e][k] += (unsigned long long)__byte_perm(r4[l], 0u, 0x4440u + e) * w;
+      for (int k = 0; k < NW; ++k) tmp[k] = ct.P[k];
+      sub_in_place<NW>(tmp, S);
+#pragma unroll
+      for (int k = 0; k < NW; ++k) S[k] = tmp[k];
+      neg = true;
+    }
+    const double mag = round_scaled_fast<NW>(S, shift);
+    return neg ? -mag : mag;
+  }
+}
+
+// ------------------------------------------------------------------------------------
+// Production kernel: the contraction S = sum_l r_l w_l (Section 5.2) runs on the tensor cores.
+//
+// With the weights cut into bytes, S = sum_d 2^(8d) sum_l r_l digit_d(w_l): a [rows x moduli] by
+// [moduli x digits] product of bytes, every digit sum below 27 * 255 * 255 < 2^21.  A warp takes 128
+// consecutive rows i of one column j (one 128-byte line of residues per modulus) and runs
+// mma.sync.m16n8k32 (u8 x u8 -> s32) on them:
+//   * quad g (four lanes) owns rows 16 g .. 16 g + 15; lane q of the quad loads the 16 residue bytes of the
+//     moduli q, q + 4, q + 8, ... with one 16-byte load each and transposes 4 x 4 byte blocks in registers,
+//     which yields its share of the A fragments (k slot 4 q + n holds modulus q + 4 n, slot 16 + 4 q + n
+//     modulus q + 16 + 4 n); two rows of the quad are the MMA rows g and g + 8
+//   * the B fragments are constants (host-built, CrtTable::bfrag): tiles 0 and 1 give lane q' of the quad
+//     the digit sums 4 q' .. 4 q' + 3, i.e. the 64-bit column sum of weight word q'; a third tile carries the
+//     digits 16 .. 23 (16 bits per lane) for more than 19 moduli
+//   * the column sums of a row are then spread over the quad, so they cross once through shared memory
+//     (layout below: neither the 8-byte writes nor the 16-byte reads have bank conflicts) and every lane
+//     finishes four consecutive rows with the tails above.
+// ------------------------------------------------------------------------------------
+constexpr int kXposeQuadBytes = 16 * 32 + 4 * 16;              // 16 rows x 32 bytes, 16 bytes of padding per 4 rows
+constexpr int kXposeWarpBytes = 8 * kXposeQuadBytes + 4 * 32;  // + 32 bytes per pair of quads
+__device__ __forceinline__ uint32_t xpose_quad_offset(int g) { return (uint32_t)(g * kXposeQuadBytes + 32 * (g >> 1)); }
+__device__ __forceinline__ constexpr uint32_t xpose_row_offset(int n) { return (uint32_t)(32 * n + 16 * (n >> 2)); }
+
+__device__ __forceinline__ void mma_u8_16832(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                             uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+               : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(0));
+}
+__device__ __forceinline__ void sts64(uint32_t addr, unsigned long long v) {
+  asm volatile("st.shared.u64 [%0], %1;" ::"r"(addr), "l"(v) : "memory");
+}
+__device__ __forceinline__ void lds128(uint32_t addr, unsigned long long& a, unsigned long long& b) {
+  asm volatile("ld.shared.v2.u64 {%0, %1}, [%2];" : "=l"(a), "=l"(b) : "r"(addr) : "memory");
+}
+
+// NT: digit tiles (2: weights of up to 128 bits, 3: up to 192); NHI: moduli beyond the 16th held per lane;
+// WW / NW / LEAN as in finish_element.
+template <int NT, int NHI, int WW, int NW, int LEAN>
+__global__ void __launch_bounds__(256) crt_mma_kernel(const __grid_constant__ CrtTable ct, const uint8_t* __restrict__ res,
+                                                      size_t res_ld, size_t res_stride, const int32_t* __restrict__ s,
+                                                      const int32_t* __restrict__ t, int64_t M, int64_t N, int64_t rows_readable,
+                                                      double* __restrict__ C, int64_t ldc) {
+  static_assert(WW <= 2 * NT && NT >= 2 && NT <= 3 && NHI >= 0 && NHI <= 3, "tile counts");
+  __shared__ __align__(16) uint8_t xpose[8][kXposeWarpBytes];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int g = lane >> 2, q = lane & 3;
+  uint32_t bf[NT][2];
+#pragma unroll
+  for (int tl = 0; tl < NT; ++tl) bf[tl][0] = ct.bfrag[tl][lane][0], bf[tl][1] = ct.bfrag[tl][lane][1];
+  const uint32_t xw = (uint32_t)__cvta_generic_to_shared(&xpose[warp][0]) + xpose_quad_offset(g);
+  const uint32_t x_write = xw + 8u * q;   // + row offset: this lane's column sum for row n of the quad
+  const uint32_t x_read = xw + 144u * q;  // rows 4 q .. 4 q + 3 of the quad, all four lanes' sums
+  const int64_t row_blocks = (M + 127) / 128;
+  const int64_t units = row_blocks * N;
+  const int64_t warps_total = (int64_t)gridDim.x * 8;
+  const bool vec_store = ((reinterpret_cast<uintptr_t>(C) & 15) == 0) && ((ldc & 1) == 0);
+  for (int64_t u = (int64_t)blockIdx.x * 8 + warp; u < units; u += warps_total) {
+    const int64_t j = u / row_blocks;
+    const int64_t seg = (u - j * row_blocks) * 128 + 16 * g;  // first of this quad's 16 rows
+    const bool readable = seg < rows_readable;
+    const uint8_t* rp = res + (size_t)j * res_ld + (size_t)seg;
+    uint32_t W[4 + NHI][4];
+#pragma unroll
+    for (int n = 0; n < 4 + NHI; ++n) {
+      const int l = n < 4 ? q + 4 * n : q + 16 + 4 * (n - 4);
+      uint4 v = make_uint4(0u, 0u, 0u, 0u);
+      if (readable && l < ct.L) v = __ldg(reinterpret_cast<const uint4*>(rp + (size_t)l * res_stride));
+      W[n][0] = v.x, W[n][1] = v.y, W[n][2] = v.z, W[n][3] = v.w;
+    }
+    uint32_t top16[NT == 3 ? 16 : 1];  // digits 16 + 2 q, 17 + 2 q of all 16 rows (third tile)
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      // 4 x 4 byte transposes: lo[r] / hi[r] = residues of row 4 c + r for this lane's moduli
+      uint32_t lo[4], hi[4];
+      {
+        const uint32_t u0 = __byte_perm(W[0][c], W[1][c], 0x5140), u1 = __byte_perm(W[0][c], W[1][c], 0x7362);
+        const uint32_t v0 = __byte_perm(W[2][c], W[3][c], 0x5140), v1 = __byte_perm(W[2][c], W[3][c], 0x7362);
+        lo[0] = __byte_perm(u0, v0, 0x5410), lo[1] = __byte_perm(u0, v0, 0x7632);
+        lo[2] = __byte_perm(u1, v1, 0x5410), lo[3] = __byte_perm(u1, v1, 0x7632);
+      }
+      if constexpr (NHI == 0) {
+        hi[0] = hi[1] = hi[2] = hi[3] = 0u;
+      } else if constexpr (NHI == 1) {
+#pragma unroll
+        for (int r = 0; r < 4; ++r) hi[r] = __byte_perm(W[4][c], 0u, 0x4440 + r);
+      } else {
+        const uint32_t w6 = NHI == 3 ? W[4 + (NHI == 3 ? 2 : 0)][c] : 0u;
+        const uint32_t u0 = __byte_perm(W[4][c], W[4 + (NHI >= 2 ? 1 : 0)][c], 0x5140);
+        const uint32_t u1 = __byte_perm(W[4][c], W[4 + (NHI >= 2 ? 1 : 0)][c], 0x7362);
+        const uint32_t v0 = __byte_perm(w6, 0u, 0x4140), v1 = __byte_perm(w6, 0u, 0x4342);
+        hi[0] = __byte_perm(u0, v0, 0x5410), hi[1] = __byte_perm(u0, v0, 0x7632);
+        hi[2] = __byte_perm(u1, v1, 0x5410), hi[3] = __byte_perm(u1, v1, 0x7632);
+      }
+#pragma unroll
+      for (int pr = 0; pr < 2; ++pr) {
+        const int ra = 4 * c + 2 * pr, rb = ra + 1;  // rows of the quad on MMA rows g and g + 8
+        int d0[4], d1[4];
+        mma_u8_16832(d0, lo[2 * pr], lo[2 * pr + 1], hi[2 * pr], hi[2 * pr + 1], bf[0][0], bf[0][1]);
+        mma_u8_16832(d1, lo[2 * pr], lo[2 * pr + 1], hi[2 * pr], hi[2 * pr + 1], bf[1][0], bf[1][1]);
+        // digits 4 q .. 4 q + 3 of row ra (d[0], d[1]) and of row rb (d[2], d[3]): sum_d 2^(8 d) D_d < 2^46
+        const unsigned long long Ta = (unsigned long long)(uint32_t)(d0[0] + (d0[1] << 8)) +
+                                      ((unsigned long long)(uint32_t)(d1[0] + (d1[1] << 8)) << 16);
+        const unsigned long long Tb = (unsigned long long)(uint32_t)(d0[2] + (d0[3] << 8)) +
+                                      ((unsigned long long)(uint32_t)(d1[2] + (d1[3] << 8)) << 16);
+        sts64(x_write + xpose_row_offset(ra), Ta);
+        sts64(x_write + xpose_row_offset(rb), Tb);
+        if constexpr (NT == 3) {
+          int d2[4];
+          mma_u8_16832(d2, lo[2 * pr], lo[2 * pr + 1], hi[2 * pr], hi[2 * pr + 1], bf[NT - 1][0], bf[NT - 1][1]);
+          top16[ra] = (uint32_t)(d2[0] + (d2[1] << 8));
+          top16[rb] = (uint32_t)(d2[2] + (d2[3] << 8));
         }
       }
     }
-    const int tj = t[j];
-    const int4 s4 = *reinterpret_cast<const int4*>(s + i);
-    const int sh[4] = {s4.x + tj, s4.y + tj, s4.z + tj, s4.w + tj};
-    double out[4];
+    __syncwarp();
+    unsigned long long acc[4][2 * NT];
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-      if constexpr (LEAN == 4) {
-        static_assert(LEAN != 4 || (WW == 4 && NW == 5), "this lean tail is written for 4 weight words, 5 sum words");
-        unsigned long long a4[4];
-#pragma unroll
-        for (int k = 0; k < 4; ++k) a4[k] = acc[e][k < WW ? k : 0];
-        out[e] = reconstruct_lean(a4, ct, sh[e]);
-        continue;
-      }
-      if constexpr (LEAN == 5) {
-        static_assert(LEAN != 5 || (WW == 5 && NW == 6), "this lean tail is written for 5 weight words, 6 sum words");
-        unsigned long long a5[5];
-#pragma unroll
-        for (int k = 0; k < 5; ++k) a5[k] = acc[e][k < WW ? k : 0];
-        out[e] = reconstruct_lean5(a5, ct, sh[e]);
-        continue;
-      }
-      uint32_t S[NW];
-      unsigned long long carry = 0ull;
-#pragma unroll
-      for (int k = 0; k < NW; ++k) {
-        const unsigned long long v = (k < WW ? acc[e][k] : 0ull) + carry;
-        S[k] = (uint32_t)v;
-        carry = v >> 32;
-      }
-      // quotient estimate from the three top words (truncation error << 1), exact correction
-      double Sd = (double)S[NW - 1];
-      if (NW >= 2) Sd = Sd * 4294967296.0 + (double)S[NW - 2];
-      if (NW >= 3) Sd = Sd * 4294967296.0 + (double)S[NW - 3];
-      if (NW > 3) Sd *= __longlong_as_double((long long)(1023 + 32 * (NW - 3)) << 52);
-      const uint32_t q = (uint32_t)(Sd * ct.inv_P);
-      uint32_t borrow = 0, mc = 0;
-#pragma unroll
-      for (int k = 0; k < NW; ++k) {
-        const unsigned long long prod = (unsigned long long)q * ct.P[k] + mc;
-        mc = (uint32_t)(prod >> 32);
-        const unsigned long long d = (unsigned long long)S[k] - (uint32_t)prod - borrow;
-        S[k] = (uint32_t)d;
-        borrow = (uint32_t)(d >> 63);
-      }
-      uint32_t signw = 0u - mc - borrow;
-#pragma unroll 1
-      for (int it = 0; it < 2 && signw != 0; ++it) {
-        uint32_t c2 = 0;
-#pragma unroll
-        for (int k = 0; k < NW; ++k) {
-          const unsigned long long v = (unsigned long long)S[k] + ct.P[k] + c2;
-          S[k] = (uint32_t)v;
-          c2 = (uint32_t)(v >> 32);
-        }
-        signw += c2;
-      }
-#pragma unroll 1
-      for (int it = 0; it < 2 && ge<NW>(S, ct.P); ++it) sub_in_place<NW>(S, ct.P);
-      bool neg = false;
-      if (gt<NW>(S, ct.halfP)) {
-        uint32_t tmp[NW];
-#pragma unroll
-        for (int k = 0; k < NW; ++k) tmp[k] = ct.P[k];
-        sub_in_place<NW>(tmp, S);
-#pragma unroll
-        for (int k = 0; k < NW; ++k) S[k] = tmp[k];
-        neg = true;
-      }
-      const double mag = round_scaled_fast<NW>(S, sh[e]);
-      out[e] = neg ? -mag : mag;
+      lds128(x_read + 32 * e, acc[e][0], acc[e][1]);
+      lds128(x_read + 32 * e + 16, acc[e][2], acc[e][3]);
     }
-    double* dst = C + i + j * ldc;
-    if (i + 4 <= M && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0)) {
-      reinterpret_cast<double2*>(dst)[0] = make_double2(out[0], out[1]);
-      reinterpret_cast<double2*>(dst)[1] = make_double2(out[2], out[3]);
-    } else {
+    __syncwarp();
+    if constexpr (NT == 3) {
+      // second crossing for the 16-bit sums above bit 128: word 4 = lanes 0 and 1, word 5 = lanes 2 and 3
 #pragma unroll
-      for (int e = 0; e < 4; ++e)
-        if (i + e < M) dst[e] = out[e];
+      for (int n = 0; n < 16; ++n) sts64(x_write + xpose_row_offset(n), (unsigned long long)top16[n]);
+      __syncwarp();
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        unsigned long long u0, u1, u2, u3;
+        lds128(x_read + 32 * e, u0, u1);
+        lds128(x_read + 32 * e + 16, u2, u3);
+        acc[e][4] = u0 + (u1 << 16);
+        acc[e][5] = u2 + (u3 << 16);
+      }
+      __syncwarp();
+    }
+    const int64_t i0 = seg + 4 * q;
+    if (i0 < M) {
+      const int tj = t[j];
+      double out[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int sh = (i0 + e < M ? s[i0 + e] : 0) + tj;
+        unsigned long long a[WW];
+#pragma unroll
+        for (int k = 0; k < WW; ++k) a[k] = acc[e][k];
+        out[e] = finish_element<WW, NW, LEAN>(a, ct, sh);
+      }
+      double* dst = C + i0 + j * ldc;
+      if (i0 + 4 <= M && vec_store) {
+        reinterpret_cast<double2*>(dst)[0] = make_double2(out[0], out[1]);
+        reinterpret_cast<double2*>(dst)[1] = make_double2(out[2], out[3]);
+      } else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          if (i0 + e < M) dst[e] = out[e];
+      }
     }
   }
 }
@@ -393,11 +511,11 @@ __global__ void __launch_bounds__(256, LEAN ? 4 : 2) crt4_kernel(const __grid_co
 __global__ void copy_residues_kernel(const uint8_t* __restrict__ res, int64_t Mp, size_t res_stride, int64_t M, int64_t N,
                                      uint8_t* __restrict__ out) {
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  const int64_t j = blockIdx.y;
   const int64_t l = blockIdx.z;
   if (i >= M) return;
-  out[(size_t)l * (size_t)M * (size_t)N + (size_t)j * (size_t)M + (size_t)i] =
-      res[(size_t)l * res_stride + (size_t)j * (size_t)Mp + (size_t)i];
+  for (int64_t j = blockIdx.y; j < N; j += gridDim.y)
+    out[(size_t)l * (size_t)M * (size_t)N + (size_t)j * (size_t)M + (size_t)i] =
+        res[(size_t)l * res_stride + (size_t)j * (size_t)Mp + (size_t)i];
 }
 
 // acc = (acc + chunk) mod m for one modulus per blockIdx.y: sums the residues of two k ranges
@@ -437,62 +555,55 @@ cudaError_t launch_add_residues(const Geometry& g, const ModulusTable& mt, uint8
 
 cudaError_t launch_crt(const Geometry& g, const CrtTable& ct, const uint8_t* res, int64_t res_ld, size_t res_stride,
                        const int32_t* s, const int32_t* t, double* C, int64_t ldc, uint32_t* x_out, cudaStream_t st) {
-  // weight words actually used, and whether the four-row kernel's vector loads are legal here
+  // weight words actually used
   int ww = 1;
   for (int l = 0; l < ct.L; ++l)
     for (int k = 0; k < kCrtWords; ++k)
       if (ct.w[l][k] && k + 1 > ww) ww = k + 1;
-  const bool s_padded = (const void*)s == (const void*)(workspace_ptr() + g.off_s);  // the workspace copy has Mp entries
-  const bool fast = !x_out && (res_ld % 4 == 0) && (res_stride % 4 == 0) && ((reinterpret_cast<uintptr_t>(res) & 3) == 0) &&
-                    ((reinterpret_cast<uintptr_t>(s) & 15) == 0) && (g.M % 4 == 0 || s_padded);
-  if (fast) {
-    dim3 grid((unsigned)((g.M + 1023) / 1024), (unsigned)(g.N < 65535 ? g.N : 65535));
-#define OZK_CRT4(WW, NW)                                                                                             \
-  do {                                                                                                             \
-    if (ct.L <= 19)                                                                                                \
-      crt4_kernel<WW, NW, 0, 19><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc);   \
-    else                                                                                                           \
-      crt4_kernel<WW, NW, 0, kMaxModuli><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc); \
-  } while (0)
-    const bool lean = ct.words <= 5 && ww <= 4 && ct.p_bits >= 101 && ct.p_bits <= 126;  // 16 to 19 moduli
+  // The tensor-core kernel reads 16 residue bytes per load: aligned columns, and either a row count that is a
+  // multiple of 16 or columns padded to one (the workspace layout).
+  const int64_t rows16 = round_up(g.M, 16);
+  const bool aligned = !x_out && (res_ld % 16 == 0) && (res_stride % 16 == 0) && ((reinterpret_cast<uintptr_t>(res) & 15) == 0) &&
+                       res_ld >= rows16;
+  if (aligned) {
+    const int64_t units = ((g.M + 127) / 128) * g.N;
+    const int64_t cap = (int64_t)device_sm_count() * 6;
+    const unsigned grid = (unsigned)std::min<int64_t>((units + 7) / 8, cap);
+    const int nhi = ct.L <= 16 ? 0 : ct.L <= 20 ? 1 : ct.L <= 24 ? 2 : 3;
+    const bool lean = ct.words <= 5 && ww <= 4 && ct.p_bits >= 101 && ct.p_bits <= 126;   // 16 to 19 moduli
     const bool lean5 = ct.words <= 6 && ww <= 5 && ct.p_bits >= 129 && ct.p_bits <= 158;  // 20 to 23 moduli
-#define OZK_CRT_LEAN5(LL) crt4_kernel<5, 6, 5, LL, true><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc)
-    if (lean5 && ct.L == 20) OZK_CRT_LEAN5(20);
-    else if (lean5 && ct.L == 21) OZK_CRT_LEAN5(21);
-    else if (lean5 && ct.L == 22) OZK_CRT_LEAN5(22);
-    else if (lean5 && ct.L == 23) OZK_CRT_LEAN5(23);
-#undef OZK_CRT_LEAN5
-    else
-#define OZK_CRT_LEAN(LL) crt4_kernel<4, 5, 4, LL, true><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc)
-    if (lean && ct.L == 19) OZK_CRT_LEAN(19);
-    else if (lean && ct.L == 18) OZK_CRT_LEAN(18);
-    else if (lean && ct.L == 17) OZK_CRT_LEAN(17);
-    else if (lean && ct.L == 16) OZK_CRT_LEAN(16);
-#undef OZK_CRT_LEAN
-    else if (lean)
-      crt4_kernel<4, 5, 4, 19><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc);
-    else if (ct.words == 5 && ww <= 4) OZK_CRT4(4, 5);
-    else if (ct.words <= 2) OZK_CRT4(2, 2);
-    else if (ct.words == 3) OZK_CRT4(3, 3);
-    else if (ct.words == 4) OZK_CRT4(4, 4);
-    else if (ct.words == 5) OZK_CRT4(5, 5);
-    else OZK_CRT4(6, 6);
-#undef OZK_CRT4
-    return cudaGetLastError();
+#define OZK_CRT_MMA(NT, NHI, WW, NW, LEAN)                                                                           \
+  crt_mma_kernel<NT, NHI, WW, NW, LEAN><<<grid, 256, 0, st>>>(ct, res, (size_t)res_ld, res_stride, s, t, g.M, g.N, rows16, C, ldc)
+    bool launched = true;
+    if (lean && nhi == 0) OZK_CRT_MMA(2, 0, 4, 5, 4);
+    else if (lean && nhi == 1) OZK_CRT_MMA(2, 1, 4, 5, 4);
+    else if (lean5 && nhi == 1) OZK_CRT_MMA(3, 1, 5, 6, 5);
+    else if (lean5 && nhi == 2) OZK_CRT_MMA(3, 2, 5, 6, 5);
+    else if (ww <= 4 && nhi == 0 && ct.words <= 2) OZK_CRT_MMA(2, 0, 4, 2, 0);
+    else if (ww <= 4 && nhi == 0 && ct.words == 3) OZK_CRT_MMA(2, 0, 4, 3, 0);
+    else if (ww <= 4 && nhi == 0 && ct.words == 4) OZK_CRT_MMA(2, 0, 4, 4, 0);
+    else if (ww <= 4 && nhi == 0 && ct.words == 5) OZK_CRT_MMA(2, 0, 4, 5, 0);
+    else if (ww <= 4 && nhi == 1 && ct.words == 5) OZK_CRT_MMA(2, 1, 4, 5, 0);
+    else if (nhi == 1 && ct.words == 6) OZK_CRT_MMA(3, 1, 6, 6, 0);
+    else if (nhi == 2 && ct.words == 6) OZK_CRT_MMA(3, 2, 6, 6, 0);
+    else if (nhi == 3 && ct.words == 6) OZK_CRT_MMA(3, 3, 6, 6, 0);
+    else launched = false;
+#undef OZK_CRT_MMA
+    if (launched) return cudaGetLastError();
   }
-  dim3 grid((unsigned)((g.M + 255) / 256), (unsigned)g.N);
+  dim3 grid((unsigned)((g.M + 255) / 256), (unsigned)(g.N < 65535 ? g.N : 65535));
   switch (ct.words) {
-    case 2: crt_kernel<2><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, C, ldc, x_out); break;
-    case 3: crt_kernel<3><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, C, ldc, x_out); break;
-    case 4: crt_kernel<4><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, C, ldc, x_out); break;
-    case 5: crt_kernel<5><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, C, ldc, x_out); break;
-    default: crt_kernel<6><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, C, ldc, x_out); break;
+    case 2: crt_kernel<2><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc, x_out); break;
+    case 3: crt_kernel<3><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc, x_out); break;
+    case 4: crt_kernel<4><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc, x_out); break;
+    case 5: crt_kernel<5><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc, x_out); break;
+    default: crt_kernel<6><<<grid, 256, 0, st>>>(ct, res, res_ld, res_stride, s, t, g.M, g.N, C, ldc, x_out); break;
   }
   return cudaGetLastError();
 }
 
 cudaError_t launch_copy_residues(const Geometry& g, const uint8_t* res, uint8_t* out, cudaStream_t st) {
-  dim3 grid((unsigned)((g.M + 255) / 256), (unsigned)g.N, (unsigned)g.L);
+  dim3 grid((unsigned)((g.M + 255) / 256), (unsigned)(g.N < 65535 ? g.N : 65535), (unsigned)g.L);
   copy_residues_kernel<<<grid, 256, 0, st>>>(res, g.Mp, (size_t)g.Mp * (size_t)g.Np, g.M, g.N, out);
   return cudaGetLastError();
 }

@@ -22,6 +22,8 @@
 #include <stdio.h>
 #include <stdlib.h>
 
+#include <atomic>
+
 #include "ozk_common.cuh"
 #include "ozk_ptx.cuh"
 
@@ -874,14 +876,12 @@ bool make_plane_map(CUtensorMap* map, const void* base, int64_t k_bytes, int64_t
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int sm_count() {
-  static int n = 0;
-  if (!n) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-  }
-  return n;
+// cudaFuncSetAttribute acts on the current device only: remember per device ordinal where it has been done.
+constexpr int kMaxDevices = 64;
+int current_device_ordinal() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return -1;
+  return dev;
 }
 
 // The CTA-pair (cta_group::2) kernel runs whenever the padded column count is a multiple of 256;
@@ -901,13 +901,17 @@ ozk_status launch_limb_gemm(const CUtensorMap& map_p, const CUtensorMap& map_q, 
   constexpr size_t kStageBytes = (size_t)NP * kPTileBytes + (size_t)NQ * W * kTileKBytes;
   const size_t smem = STAGES * kStageBytes + sizeof(GemmShared) + 1024;
   auto kernel = limb_gemm_kernel<NP, NQ, W, STAGES, Epi>;
-  static bool attr_set = false;
-  if (!attr_set) {
+  static std::atomic<bool> attr_set[kMaxDevices];
+  const int dev = current_device_ordinal();
+  if (dev < 0) return OZK_ERR_CUDA;
+  if (!attr_set[dev].load(std::memory_order_acquire)) {
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return OZK_ERR_CUDA;
-    attr_set = true;
+    attr_set[dev].store(true, std::memory_order_release);
   }
+  const int sms = device_sm_count();
+  if (sms < 1) return OZK_ERR_CUDA;
   const long long items = (long long)core.L * core.tiles_p * core.tiles_q;
-  const int grid = (int)(items < sm_count() ? items : sm_count());
+  const int grid = (int)(items < sms ? items : sms);
   kernel<<<grid, 64 + 32 * Epi::kWarps, smem, st>>>(map_p, map_q, core, ep);
   return cudaGetLastError() == cudaSuccess ? OZK_OK : OZK_ERR_CUDA;
 }
@@ -958,13 +962,17 @@ ozk_status gemm_residues(const Geometry& g, const ModulusTable& mt, uint8_t* ws,
     if (!make_plane_map(&map_qh, planes_a, klen / 2, g.Mp, 2 * g.L, g.plane_bytes_a, 64, g.pitch)) return OZK_ERR_CUDA;
     pc.wave_counter = reinterpret_cast<unsigned int*>(ws + g.off_status + 512);
     const size_t smem = (size_t)kPairStages * kPairStageBytes + kPairZeroBytes + sizeof(GemmShared) + 1024;
-    static int max_pairs = -1;
-    if (max_pairs < 0) {
+    static std::atomic<bool> attr_set[kMaxDevices];
+    const int dev = current_device_ordinal();
+    if (dev < 0) return OZK_ERR_CUDA;
+    if (!attr_set[dev].load(std::memory_order_acquire)) {
       if (cudaFuncSetAttribute(residue_gemm_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
           cudaFuncSetAttribute(residue_gemm_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return OZK_ERR_CUDA;
-      max_pairs = sm_count() / 2;
+      attr_set[dev].store(true, std::memory_order_release);
     }
+    const int max_pairs = device_sm_count() / 2;
+    if (max_pairs < 1) return OZK_ERR_CUDA;
     const long long items = (long long)pc.L * pc.tiles_p * pc.tiles_q;
     const int pairs = (int)(items < max_pairs ? items : max_pairs);
     if (cudaMemsetAsync(pc.wave_counter, 0, 4, st) != cudaSuccess) return OZK_ERR_CUDA;

@@ -257,6 +257,19 @@ bool build_crt_table(int L, CrtTable* t) {
   t->q_scale = ldexp(t->inv_P, 96) * (1.0 - ldexp(1.0, -30));
   t->q_scale128 = ldexp(t->inv_P, 128) * (1.0 - ldexp(1.0, -30));
   t->p_bits = big_bits(P);
+  for (int tile = 0; tile < 3; ++tile)
+    for (int lane = 0; lane < 32; ++lane) {
+      const int col = lane >> 2, q = lane & 3;
+      const int digit = tile < 2 ? 4 * (col / 2) + 2 * tile + col % 2 : 16 + col;
+      for (int reg = 0; reg < 2; ++reg) {
+        uint32_t v = 0;
+        for (int n = 0; n < 4; ++n) {
+          const int l = q + 16 * reg + 4 * n;
+          if (l < L && digit < 4 * kCrtWords) v |= ((t->w[l][digit / 4] >> (8 * (digit % 4))) & 0xFFu) << (8 * n);
+        }
+        t->bfrag[tile][lane][reg] = v;
+      }
+    }
   return true;
 }
 

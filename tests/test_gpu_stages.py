@@ -111,11 +111,12 @@ def words_to_int(words: np.ndarray) -> int:
 
 
 @pytest.mark.parametrize("fast", [False, True])
-@pytest.mark.parametrize("L", [2, 12, 14, 19, 20, 23, 24, 27])
+@pytest.mark.parametrize("L", [2, 9, 12, 14, 16, 17, 18, 19, 20, 21, 22, 23, 24, 27])
 def test_crt_stage_matches_oracle_on_arbitrary_residues(L, fast):
     """fast=False: one element per thread, with the reconstructed integers exported; fast=True: the
-    four-rows-per-thread kernel the full pipeline uses (row count a multiple of 4, no export)."""
-    M, N, K = (40, 29, 16) if fast else (37, 29, 16)
+    tensor-core kernel the full pipeline uses (row count a multiple of 16: one full block of 128 rows and a
+    ragged one; no export)."""
+    M, N, K = (144, 9, 16) if fast else (37, 29, 16)
     mods = moduli.select_moduli(L)
     P = moduli.product(mods)
     rng = np.random.default_rng(L)
@@ -127,6 +128,9 @@ def test_crt_stage_matches_oracle_on_arbitrary_residues(L, fast):
             xs[idx] = 0
     xs[0, 0], xs[1, 0], xs[2, 0], xs[3, 0] = 0, (P - 1) // 2, -((P - 1) // 2), 1
     xs[4, 0], xs[5, 0] = 2 ** 53 + 1, -(2 ** 54 + 2 ** 0 + 2)             # ties and near-ties of the final rounding
+    # every residue m_l - 1 (the largest weighted sum and quotient), and the neighbours of the range's ends
+    xs[6, 0], xs[7, 0], xs[12, 0], xs[13, 0] = -1, 1 - P // 2, P // 2 - 1, -2
+    xs[M - 1, N - 1], xs[M - 2, N - 1] = -1, (P - 1) // 2
     for idx in np.ndindex(M, N):
         if 2 * abs(xs[idx]) >= P:
             xs[idx] = 0
