@@ -61,10 +61,14 @@ struct CrtTable {
   uint32_t w[kMaxModuli][kCrtWords];       // w_l little endian
   uint32_t P[kCrtWords];
   uint32_t halfP[kCrtWords];               // floor(P / 2)
+  uint32_t negP[4];                        // 2^128 - P (used when P < 2^128)
   double inv_P;                            // 1 / P rounded to double
-  double q_scale;                          // (2^96 / P) (1 - 2^-30): quotient estimate from the words above bit 96
-  double q_scale128;                       // (2^128 / P) (1 - 2^-30): the same from the words above bit 128
   int p_bits;                              // bit length of P
+  // Integer quotient estimate of the carry-chain tails (P of at least 2^100, at most 2047 for floor(S / P)):
+  // top = floor(S / 2^q_shift) < 2^32 with q_shift = p_bits - 21 = 32 q_word + q_bit, and
+  // q_mul = floor(2^(52 + q_shift) / P * (1 - 2^-28)) < 2^32; (top * q_mul) >> 52 is floor(S / P) or one less.
+  uint32_t q_mul;
+  int q_word, q_bit;
   // B fragments of the reconstruction kernel's mma.sync.m16n8k32 (u8): tile, lane, register.  Lane (g, q) holds
   // column g of the tile; byte n of register 0 / 1 is the digit for modulus q + 4 n / q + 16 + 4 n.  Column c
   // of tile 0 carries digit (byte) 4 (c / 2) + c % 2 of the weights, of tile 1 digit 4 (c / 2) + 2 + c % 2, of

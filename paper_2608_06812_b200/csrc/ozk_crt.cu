@@ -109,19 +109,26 @@ __global__ void __launch_bounds__(256) crt_kernel(CrtTable ct, const uint8_t* __
 // ------------------------------------------------------------------------------------
 template <int NW>
 __device__ __forceinline__ double round_scaled_fast(const uint32_t (&mag)[NW], int shift) {
-  // top non-zero word and the two words below it
-  int top = -1;
+  // top non-zero word and the two words below it; the usual case (top word in use) needs no search
+  int top = NW - 1;
+  uint32_t w2 = mag[NW - 1], w1 = NW >= 2 ? mag[NW >= 2 ? NW - 2 : 0] : 0u, w0 = NW >= 3 ? mag[NW >= 3 ? NW - 3 : 0] : 0u, rest = 0;
+  if (w2 != 0) {
 #pragma unroll
-  for (int i = 0; i < NW; ++i)
-    if (mag[i]) top = i;
-  if (top < 0) return 0.0;
-  uint32_t w2 = 0, w1 = 0, w0 = 0, rest = 0;
+    for (int i = 0; i < NW - 3; ++i) rest |= mag[i];
+  } else {
+    top = -1;
 #pragma unroll
-  for (int i = 0; i < NW; ++i) {
-    if (i == top) w2 = mag[i];
-    if (i == top - 1) w1 = mag[i];
-    if (i == top - 2) w0 = mag[i];
-    if (i < top - 2) rest |= mag[i];
+    for (int i = 0; i < NW; ++i)
+      if (mag[i]) top = i;
+    if (top < 0) return 0.0;
+    w2 = w1 = w0 = 0;
+#pragma unroll
+    for (int i = 0; i < NW; ++i) {
+      if (i == top) w2 = mag[i];
+      if (i == top - 1) w1 = mag[i];
+      if (i == top - 2) w0 = mag[i];
+      if (i < top - 2) rest |= mag[i];
+    }
   }
   const int lz = __clz(w2);
   const int bitlen = 32 * top + 32 - lz;
@@ -141,72 +148,78 @@ __device__ __forceinline__ double round_scaled_fast(const uint32_t (&mag)[NW], i
 }
 
 
-// Lean reconstruction for 2^100 <= P < 2^126 (16 to 19 moduli): the weighted sum S (five words)
-// arrives as four 64-bit column sums; everything after the quotient estimate is 128-bit arithmetic
-// written as explicit carry chains.
-//   q  = floor((S >> 96) * (2^96 / P) * (1 - 2^-30))  is the true quotient or one below it, so
-//   x  = S - q P  lies in [0, 2P) and fits 128 bits; one conditional subtraction brings it below P.
+// Lean reconstruction for 2^100 <= P < 2^126 (16 to 19 moduli): the weighted sum S (up to 137 bits)
+// arrives as four 64-bit column sums acc[k] (weight 2^(32 k), no carries yet).
+//   q  = ((S >> (p_bits - 21)) * q_mul) >> 52 is the true quotient floor(S / P) or one below it.  The 32 bits
+//        of S it needs come from the two top column sums alone: the carries left out are worth less than
+//        2^98 < P / 4 and only lower the estimate, which keeps it in {floor(S / P) - 1, floor(S / P)}.
+//   x  = S - q P in [0, 2P) is formed column by column as acc[k] + q n_k with n = 2^128 - P (one wide
+//        multiply-add per word, then a single carry pass), modulo 2^128.
+//   The two comparisons (x >= P, x > P / 2) look at the top word first; the full comparison runs only when
+//   the top words are equal.  The rounding builds the FP64 bit pattern from the top three words directly;
+//   magnitudes below 2^96 and results outside the normal range take the general routine.
 __device__ __forceinline__ double reconstruct_lean(const unsigned long long (&acc)[4], const CrtTable& ct, int shift) {
-  const uint32_t a0l = (uint32_t)acc[0], a0h = (uint32_t)(acc[0] >> 32), a1l = (uint32_t)acc[1], a1h = (uint32_t)(acc[1] >> 32);
-  const uint32_t a2l = (uint32_t)acc[2], a2h = (uint32_t)(acc[2] >> 32), a3l = (uint32_t)acc[3], a3h = (uint32_t)(acc[3] >> 32);
-  uint32_t S1, S2, S3, S4;
-  asm("add.cc.u32 %0, %4, %5;\n\t"
-      "addc.cc.u32 %1, %6, %7;\n\t"
-      "addc.cc.u32 %2, %8, %9;\n\t"
-      "addc.u32 %3, %10, 0;"
-      : "=r"(S1), "=r"(S2), "=r"(S3), "=r"(S4)
-      : "r"(a0h), "r"(a1l), "r"(a1h), "r"(a2l), "r"(a2h), "r"(a3l), "r"(a3h));
-  const uint32_t S0 = a0l;
-  const unsigned long long top = ((unsigned long long)S4 << 32) | S3;
-  const uint32_t q = __double2uint_rz(__ull2double_rz(top) * ct.q_scale);
-  const unsigned long long m0 = (unsigned long long)q * ct.P[0];
-  const unsigned long long m1 = (unsigned long long)q * ct.P[1] + (m0 >> 32);
-  const unsigned long long m2 = (unsigned long long)q * ct.P[2] + (m1 >> 32);
-  const unsigned long long m3 = (unsigned long long)q * ct.P[3] + (m2 >> 32);
-  uint32_t x0, x1, x2, x3;
-  asm("sub.cc.u32 %0, %4, %8;\n\t"
-      "subc.cc.u32 %1, %5, %9;\n\t"
-      "subc.cc.u32 %2, %6, %10;\n\t"
-      "subc.u32 %3, %7, %11;"
-      : "=r"(x0), "=r"(x1), "=r"(x2), "=r"(x3)
-      : "r"(S0), "r"(S1), "r"(S2), "r"(S3), "r"((uint32_t)m0), "r"((uint32_t)m1), "r"((uint32_t)m2), "r"((uint32_t)m3));
+  const uint32_t a3l = (uint32_t)acc[3], a3h = (uint32_t)(acc[3] >> 32), a2h = (uint32_t)(acc[2] >> 32);
+  uint32_t t_lo, t_hi;
+  asm("add.cc.u32 %0, %2, %4;\n\taddc.u32 %1, %3, 0;" : "=r"(t_lo), "=r"(t_hi) : "r"(a3l), "r"(a3h), "r"(a2h));
+  uint32_t top;
+  if (ct.q_word == 3) {
+    top = __funnelshift_r(t_lo, t_hi, ct.q_bit);
+  } else {
+    const unsigned long long a64 = ((unsigned long long)t_hi << 32) | t_lo;
+    const unsigned long long b64 = (a64 << 32) + (uint32_t)acc[2] + (acc[1] >> 32);
+    top = (uint32_t)(b64 >> ct.q_bit);
+  }
+  const uint32_t q = __umulhi(top, ct.q_mul) >> 20;
   const uint32_t P0 = ct.P[0], P1 = ct.P[1], P2 = ct.P[2], P3 = ct.P[3];
-  uint32_t d0, d1, d2, d3, below;  // d = x - P; below = all ones if x < P
-  asm("sub.cc.u32 %0, %5, %9;\n\t"
-      "subc.cc.u32 %1, %6, %10;\n\t"
-      "subc.cc.u32 %2, %7, %11;\n\t"
-      "subc.cc.u32 %3, %8, %12;\n\t"
-      "subc.u32 %4, 0, 0;"
-      : "=r"(d0), "=r"(d1), "=r"(d2), "=r"(d3), "=r"(below)
-      : "r"(x0), "r"(x1), "r"(x2), "r"(x3), "r"(P0), "r"(P1), "r"(P2), "r"(P3));
-  if (!below) x0 = d0, x1 = d1, x2 = d2, x3 = d3;
-  uint32_t e0, e1, e2, e3;  // e = P - x
-  asm("sub.cc.u32 %0, %4, %8;\n\t"
-      "subc.cc.u32 %1, %5, %9;\n\t"
-      "subc.cc.u32 %2, %6, %10;\n\t"
-      "subc.u32 %3, %7, %11;"
-      : "=r"(e0), "=r"(e1), "=r"(e2), "=r"(e3)
-      : "r"(P0), "r"(P1), "r"(P2), "r"(P3), "r"(x0), "r"(x1), "r"(x2), "r"(x3));
-  uint32_t u0, u1, u2, u3, over;  // halfP - x borrows exactly when x > P/2
-  asm("sub.cc.u32 %0, %5, %9;\n\t"
-      "subc.cc.u32 %1, %6, %10;\n\t"
-      "subc.cc.u32 %2, %7, %11;\n\t"
-      "subc.cc.u32 %3, %8, %12;\n\t"
-      "subc.u32 %4, 0, 0;"
-      : "=r"(u0), "=r"(u1), "=r"(u2), "=r"(u3), "=r"(over)
-      : "r"(ct.halfP[0]), "r"(ct.halfP[1]), "r"(ct.halfP[2]), "r"(ct.halfP[3]), "r"(x0), "r"(x1), "r"(x2), "r"(x3));
-  uint32_t mag[4];
-  mag[0] = over ? e0 : x0;
-  mag[1] = over ? e1 : x1;
-  mag[2] = over ? e2 : x2;
-  mag[3] = over ? e3 : x3;
-  const double r = round_scaled_fast<4>(mag, shift);
-  return over ? -r : r;
+  const unsigned long long c0 = acc[0] + (unsigned long long)q * ct.negP[0];  // negP = 2^128 - P
+  const unsigned long long c1 = acc[1] + (unsigned long long)q * ct.negP[1];
+  const unsigned long long c2 = acc[2] + (unsigned long long)q * ct.negP[2];
+  const unsigned long long c3 = acc[3] + (unsigned long long)q * ct.negP[3];
+  uint32_t x0 = (uint32_t)c0, x1, x2, x3;
+  asm("add.cc.u32 %0, %3, %4;\n\taddc.cc.u32 %1, %5, %6;\n\taddc.u32 %2, %7, %8;"
+      : "=r"(x1), "=r"(x2), "=r"(x3)
+      : "r"((uint32_t)(c0 >> 32)), "r"((uint32_t)c1), "r"((uint32_t)(c1 >> 32)), "r"((uint32_t)c2), "r"((uint32_t)(c2 >> 32)), "r"((uint32_t)c3));
+  if (x3 >= P3) {  // rarely true: x >= P needs the full comparison
+    uint32_t d0, d1, d2, d3, below;
+    asm("sub.cc.u32 %0, %5, %9;\n\tsubc.cc.u32 %1, %6, %10;\n\tsubc.cc.u32 %2, %7, %11;\n\tsubc.cc.u32 %3, %8, %12;\n\tsubc.u32 %4, 0, 0;"
+        : "=r"(d0), "=r"(d1), "=r"(d2), "=r"(d3), "=r"(below)
+        : "r"(x0), "r"(x1), "r"(x2), "r"(x3), "r"(P0), "r"(P1), "r"(P2), "r"(P3));
+    if (!below) x0 = d0, x1 = d1, x2 = d2, x3 = d3;
+  }
+  const uint32_t h3 = ct.halfP[3];
+  bool over = x3 > h3;
+  if (x3 == h3) {
+    uint32_t u0, u1, u2, u3, bw;
+    asm("sub.cc.u32 %0, %5, %9;\n\tsubc.cc.u32 %1, %6, %10;\n\tsubc.cc.u32 %2, %7, %11;\n\tsubc.cc.u32 %3, %8, %12;\n\tsubc.u32 %4, 0, 0;"
+        : "=r"(u0), "=r"(u1), "=r"(u2), "=r"(u3), "=r"(bw)
+        : "r"(ct.halfP[0]), "r"(ct.halfP[1]), "r"(ct.halfP[2]), "r"(h3), "r"(x0), "r"(x1), "r"(x2), "r"(x3));
+    over = bw != 0;
+  }
+  uint32_t e0, e1, e2, e3;
+  asm("sub.cc.u32 %0, %4, %8;\n\tsubc.cc.u32 %1, %5, %9;\n\tsubc.cc.u32 %2, %6, %10;\n\tsubc.u32 %3, %7, %11;"
+      : "=r"(e0), "=r"(e1), "=r"(e2), "=r"(e3) : "r"(P0), "r"(P1), "r"(P2), "r"(P3), "r"(x0), "r"(x1), "r"(x2), "r"(x3));
+  const uint32_t m0 = over ? e0 : x0, m1 = over ? e1 : x1, m2 = over ? e2 : x2, m3 = over ? e3 : x3;
+  const int lz = __clz(m3);
+  const int e_biased = 127 + 1022 - lz - shift;  // exponent field minus one
+  if (m3 == 0u || (unsigned)e_biased >= 2046u) {
+    const uint32_t mag[4] = {m0, m1, m2, m3};
+    const double r = round_scaled_fast<4>(mag, shift);
+    return over ? -r : r;
+  }
+  const uint32_t w1 = __funnelshift_l(m2, m3, lz), w0 = __funnelshift_l(m1, m2, lz);
+  const uint32_t rest = __funnelshift_l(m0, m1, lz) | m0;
+  uint32_t lo = __funnelshift_r(w0, w1, 11), hi = w1 >> 11;
+  const uint32_t sticky = ((w0 & 0x3FFu) | rest) != 0u ? 1u : 0u;
+  const uint32_t inc = (w0 >> 10) & (sticky | lo) & 1u;
+  asm("add.cc.u32 %0, %0, %2;\n\taddc.u32 %1, %1, 0;" : "+r"(lo), "+r"(hi) : "r"(inc));
+  hi += (uint32_t)e_biased << 20;
+  if (over) hi |= 0x80000000u;
+  return __hiloint2double((int)hi, (int)lo);
 }
 
 // The same for 2^128 <= P < 2^158 (20 to 23 moduli): S has six words and arrives as five 64-bit column sums,
-// the quotient estimate uses the words above bit 128 (q_scale128 = (2^128 / P)(1 - 2^-30); the part of S below
-// bit 128 is less than P, so the estimate is again the true quotient or one below it), x has five words.
+// the quotient estimate is the same multiply-high on the 32 bits of S from bit p_bits - 21 on, x has five words.
 __device__ __forceinline__ double reconstruct_lean5(const unsigned long long (&acc)[5], const CrtTable& ct, int shift) {
   const uint32_t a0l = (uint32_t)acc[0], a0h = (uint32_t)(acc[0] >> 32), a1l = (uint32_t)acc[1], a1h = (uint32_t)(acc[1] >> 32);
   const uint32_t a2l = (uint32_t)acc[2], a2h = (uint32_t)(acc[2] >> 32), a3l = (uint32_t)acc[3], a3h = (uint32_t)(acc[3] >> 32);
@@ -220,8 +233,8 @@ __device__ __forceinline__ double reconstruct_lean5(const unsigned long long (&a
       : "=r"(S1), "=r"(S2), "=r"(S3), "=r"(S4), "=r"(S5)
       : "r"(a0h), "r"(a1l), "r"(a1h), "r"(a2l), "r"(a2h), "r"(a3l), "r"(a3h), "r"(a4l), "r"(a4h));
   const uint32_t S0 = a0l;
-  const unsigned long long top = ((unsigned long long)S5 << 32) | S4;
-  const uint32_t q = __double2uint_rz(__ull2double_rz(top) * ct.q_scale128);
+  const uint32_t top = ct.q_word == 4 ? __funnelshift_r(S4, S5, ct.q_bit) : __funnelshift_r(S3, S4, ct.q_bit);
+  const uint32_t q = __umulhi(top, ct.q_mul) >> 20;
   const unsigned long long m0 = (unsigned long long)q * ct.P[0];
   const unsigned long long m1 = (unsigned long long)q * ct.P[1] + (m0 >> 32);
   const unsigned long long m2 = (unsigned long long)q * ct.P[2] + (m1 >> 32);
@@ -365,57 +378,79 @@ __device__ __forceinline__ double finish_element(const unsigned long long (&acc)
 // ------------------------------------------------------------------------------------
 constexpr int kXposeQuadBytes = 16 * 32 + 4 * 16;              // 16 rows x 32 bytes, 16 bytes of padding per 4 rows
 constexpr int kXposeWarpBytes = 8 * kXposeQuadBytes + 4 * 32;  // + 32 bytes per pair of quads
+__host__ __device__ constexpr int kCrtWarps(int nt) { return nt == 3 ? 4 : 8; }  // warps per block: two crossing buffers per warp with three tiles
 __device__ __forceinline__ uint32_t xpose_quad_offset(int g) { return (uint32_t)(g * kXposeQuadBytes + 32 * (g >> 1)); }
 __device__ __forceinline__ constexpr uint32_t xpose_row_offset(int n) { return (uint32_t)(32 * n + 16 * (n >> 2)); }
 
 __device__ __forceinline__ void mma_u8_16832(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                              uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+  asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
                : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
                : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(0));
 }
+__device__ __forceinline__ unsigned long long mad_wide(uint32_t a, uint32_t b, uint32_t c) {  // a * b + c in 64 bits
+  unsigned long long d;
+  asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(d) : "r"(a), "r"(b), "l"((unsigned long long)c));
+  return d;
+}
 __device__ __forceinline__ void sts64(uint32_t addr, unsigned long long v) {
   asm volatile("st.shared.u64 [%0], %1;" ::"r"(addr), "l"(v) : "memory");
+}
+__device__ __forceinline__ void lds128x4(uint32_t addr, uint32_t (&w)[4]) {
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(addr) : "memory");
 }
 __device__ __forceinline__ void lds128(uint32_t addr, unsigned long long& a, unsigned long long& b) {
   asm volatile("ld.shared.v2.u64 {%0, %1}, [%2];" : "=l"(a), "=l"(b) : "r"(addr) : "memory");
 }
 
 // NT: digit tiles (2: weights of up to 128 bits, 3: up to 192); NHI: moduli beyond the 16th held per lane;
-// WW / NW / LEAN as in finish_element.
+// WW / NW / LEAN as in finish_element.  The residue loads of a warp's next unit are issued before the tails of
+// the current one, so their latency hides behind that arithmetic.
 template <int NT, int NHI, int WW, int NW, int LEAN>
-__global__ void __launch_bounds__(256) crt_mma_kernel(const __grid_constant__ CrtTable ct, const uint8_t* __restrict__ res,
-                                                      size_t res_ld, size_t res_stride, const int32_t* __restrict__ s,
-                                                      const int32_t* __restrict__ t, int64_t M, int64_t N, int64_t rows_readable,
-                                                      double* __restrict__ C, int64_t ldc) {
+__global__ void __launch_bounds__(kCrtWarps(NT) * 32, NT == 3 ? 4 : 3)
+crt_mma_kernel(const __grid_constant__ CrtTable ct, const uint8_t* __restrict__ res, size_t res_ld, size_t res_stride,
+               const int32_t* __restrict__ s, const int32_t* __restrict__ t, int64_t M, int64_t N, int64_t rows_readable,
+               double* __restrict__ C, int64_t ldc) {
   static_assert(WW <= 2 * NT && NT >= 2 && NT <= 3 && NHI >= 0 && NHI <= 3, "tile counts");
-  __shared__ __align__(16) uint8_t xpose[8][kXposeWarpBytes];
+  constexpr int kWarps = kCrtWarps(NT);
+  constexpr int NLD = 4 + NHI;  // 16-byte loads per lane and unit: moduli q, q + 4, ...
+  __shared__ __align__(16) uint8_t xpose[NT == 3 ? 2 : 1][kWarps][kXposeWarpBytes];  // [1]: the third tile's sums
+  constexpr uint32_t kUOffset = kWarps * kXposeWarpBytes;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, q = lane & 3;
   uint32_t bf[NT][2];
 #pragma unroll
   for (int tl = 0; tl < NT; ++tl) bf[tl][0] = ct.bfrag[tl][lane][0], bf[tl][1] = ct.bfrag[tl][lane][1];
-  const uint32_t xw = (uint32_t)__cvta_generic_to_shared(&xpose[warp][0]) + xpose_quad_offset(g);
+  const uint32_t xw = (uint32_t)__cvta_generic_to_shared(&xpose[0][warp][0]) + xpose_quad_offset(g);
   const uint32_t x_write = xw + 8u * q;   // + row offset: this lane's column sum for row n of the quad
   const uint32_t x_read = xw + 144u * q;  // rows 4 q .. 4 q + 3 of the quad, all four lanes' sums
+  // work units (row block, column) are dealt round-robin to the warps of the grid; the position advances without
+  // a division per unit
   const int64_t row_blocks = (M + 127) / 128;
-  const int64_t units = row_blocks * N;
-  const int64_t warps_total = (int64_t)gridDim.x * 8;
+  const int64_t warps_total = (int64_t)gridDim.x * kWarps;
+  const int64_t step_j = warps_total / row_blocks, step_rb = warps_total - step_j * row_blocks;
+  const int64_t first = (int64_t)blockIdx.x * kWarps + warp;
+  int64_t j = first / row_blocks, rb = first - j * row_blocks;
   const bool vec_store = ((reinterpret_cast<uintptr_t>(C) & 15) == 0) && ((ldc & 1) == 0);
-  for (int64_t u = (int64_t)blockIdx.x * 8 + warp; u < units; u += warps_total) {
-    const int64_t j = u / row_blocks;
-    const int64_t seg = (u - j * row_blocks) * 128 + 16 * g;  // first of this quad's 16 rows
-    const bool readable = seg < rows_readable;
-    const uint8_t* rp = res + (size_t)j * res_ld + (size_t)seg;
-    uint32_t W[4 + NHI][4];
+  const int n_mine = (ct.L - q + 3) >> 2;  // this lane's moduli: q + 4 n for n < n_mine
+  const uint8_t* lane_base = res + (size_t)q * res_stride + (size_t)(16 * g);
+  const size_t stride4 = 4 * res_stride;
+  uint32_t W[NLD][4];
+  auto issue_loads = [&](int64_t jj, int64_t rr) {
+    const bool readable = rr * 128 + 16 * g < rows_readable;
+    const uint8_t* p = lane_base + (size_t)jj * res_ld + (size_t)(rr * 128);
 #pragma unroll
-    for (int n = 0; n < 4 + NHI; ++n) {
-      const int l = n < 4 ? q + 4 * n : q + 16 + 4 * (n - 4);
+    for (int n = 0; n < NLD; ++n) {
       uint4 v = make_uint4(0u, 0u, 0u, 0u);
-      if (readable && l < ct.L) v = __ldg(reinterpret_cast<const uint4*>(rp + (size_t)l * res_stride));
+      if (readable && n < n_mine) v = __ldg(reinterpret_cast<const uint4*>(p));
       W[n][0] = v.x, W[n][1] = v.y, W[n][2] = v.z, W[n][3] = v.w;
+      p += stride4;
     }
-    uint32_t top16[NT == 3 ? 16 : 1];  // digits 16 + 2 q, 17 + 2 q of all 16 rows (third tile)
+  };
+  bool have = j < N;
+  if (have) issue_loads(j, rb);
+  while (have) {
+    const int64_t cur_j = j, i0 = rb * 128 + 16 * g + 4 * q;  // this lane finishes rows i0 .. i0 + 3 of column cur_j
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
       // 4 x 4 byte transposes: lo[r] / hi[r] = residues of row 4 c + r for this lane's moduli
@@ -430,81 +465,74 @@ __global__ void __launch_bounds__(256) crt_mma_kernel(const __grid_constant__ Cr
         hi[0] = hi[1] = hi[2] = hi[3] = 0u;
       } else if constexpr (NHI == 1) {
 #pragma unroll
-        for (int r = 0; r < 4; ++r) hi[r] = __byte_perm(W[4][c], 0u, 0x4440 + r);
+        for (int r = 0; r < 4; ++r) hi[r] = __byte_perm(W[NLD - 1][c], 0u, 0x4440 + r);
       } else {
-        const uint32_t w6 = NHI == 3 ? W[4 + (NHI == 3 ? 2 : 0)][c] : 0u;
-        const uint32_t u0 = __byte_perm(W[4][c], W[4 + (NHI >= 2 ? 1 : 0)][c], 0x5140);
-        const uint32_t u1 = __byte_perm(W[4][c], W[4 + (NHI >= 2 ? 1 : 0)][c], 0x7362);
+        const uint32_t w5 = W[NHI >= 2 ? 5 : 0][c], w6 = NHI == 3 ? W[NHI == 3 ? 6 : 0][c] : 0u;
+        const uint32_t u0 = __byte_perm(W[4][c], w5, 0x5140), u1 = __byte_perm(W[4][c], w5, 0x7362);
         const uint32_t v0 = __byte_perm(w6, 0u, 0x4140), v1 = __byte_perm(w6, 0u, 0x4342);
         hi[0] = __byte_perm(u0, v0, 0x5410), hi[1] = __byte_perm(u0, v0, 0x7632);
         hi[2] = __byte_perm(u1, v1, 0x5410), hi[3] = __byte_perm(u1, v1, 0x7632);
       }
 #pragma unroll
       for (int pr = 0; pr < 2; ++pr) {
-        const int ra = 4 * c + 2 * pr, rb = ra + 1;  // rows of the quad on MMA rows g and g + 8
+        const int ra = 4 * c + 2 * pr, rb2 = ra + 1;  // rows of the quad on MMA rows g and g + 8
         int d0[4], d1[4];
         mma_u8_16832(d0, lo[2 * pr], lo[2 * pr + 1], hi[2 * pr], hi[2 * pr + 1], bf[0][0], bf[0][1]);
         mma_u8_16832(d1, lo[2 * pr], lo[2 * pr + 1], hi[2 * pr], hi[2 * pr + 1], bf[1][0], bf[1][1]);
-        // digits 4 q .. 4 q + 3 of row ra (d[0], d[1]) and of row rb (d[2], d[3]): sum_d 2^(8 d) D_d < 2^46
-        const unsigned long long Ta = (unsigned long long)(uint32_t)(d0[0] + (d0[1] << 8)) +
-                                      ((unsigned long long)(uint32_t)(d1[0] + (d1[1] << 8)) << 16);
-        const unsigned long long Tb = (unsigned long long)(uint32_t)(d0[2] + (d0[3] << 8)) +
-                                      ((unsigned long long)(uint32_t)(d1[2] + (d1[3] << 8)) << 16);
-        sts64(x_write + xpose_row_offset(ra), Ta);
-        sts64(x_write + xpose_row_offset(rb), Tb);
+        // digits 4 q .. 4 q + 3 of row ra (d[0], d[1]) and of row rb2 (d[2], d[3]): sum_d 2^(8 d) D_d < 2^46
+        sts64(x_write + xpose_row_offset(ra), mad_wide((uint32_t)(d1[0] + (d1[1] << 8)), 65536u, (uint32_t)(d0[0] + (d0[1] << 8))));
+        sts64(x_write + xpose_row_offset(rb2), mad_wide((uint32_t)(d1[2] + (d1[3] << 8)), 65536u, (uint32_t)(d0[2] + (d0[3] << 8))));
         if constexpr (NT == 3) {
           int d2[4];
           mma_u8_16832(d2, lo[2 * pr], lo[2 * pr + 1], hi[2 * pr], hi[2 * pr + 1], bf[NT - 1][0], bf[NT - 1][1]);
-          top16[ra] = (uint32_t)(d2[0] + (d2[1] << 8));
-          top16[rb] = (uint32_t)(d2[2] + (d2[3] << 8));
+          sts64(x_write + kUOffset + xpose_row_offset(ra), (unsigned long long)(uint32_t)(d2[0] + (d2[1] << 8)));
+          sts64(x_write + kUOffset + xpose_row_offset(rb2), (unsigned long long)(uint32_t)(d2[2] + (d2[3] << 8)));
         }
       }
     }
+    // next unit of this warp: its loads fly while the tails below run
+    j += step_j, rb += step_rb;
+    if (rb >= row_blocks) rb -= row_blocks, ++j;
+    have = j < N;
+    if (have) issue_loads(j, rb);
     __syncwarp();
-    unsigned long long acc[4][2 * NT];
+    // every lane finishes its four rows two at a time (a rolled loop: the column sums are read just before use,
+    // which keeps the register count low enough for three blocks per SM)
+    const int tj = t[cur_j];
+    double* dst = C + i0 + cur_j * ldc;
+#pragma unroll 1
+    for (int h = 0; h < 2; ++h) {
+      double out[2];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      lds128(x_read + 32 * e, acc[e][0], acc[e][1]);
-      lds128(x_read + 32 * e + 16, acc[e][2], acc[e][3]);
-    }
-    __syncwarp();
-    if constexpr (NT == 3) {
-      // second crossing for the 16-bit sums above bit 128: word 4 = lanes 0 and 1, word 5 = lanes 2 and 3
+      for (int e = 0; e < 2; ++e) {
+        const uint32_t xr = x_read + 64 * h + 32 * e;
+        unsigned long long a[2 * NT];
+        lds128(xr, a[0], a[1]);
+        lds128(xr + 16, a[2], a[3]);
+        if constexpr (NT == 3) {
+          // 16-bit sums above bit 128: word 4 from lanes 0 and 1, word 5 from lanes 2 and 3
+          unsigned long long u0, u1, u2, u3;
+          lds128(xr + kUOffset, u0, u1);
+          lds128(xr + kUOffset + 16, u2, u3);
+          a[4] = u0 + (u1 << 16);
+          a[5] = u2 + (u3 << 16);
+        }
+        const int64_t i = i0 + 2 * h + e;
+        const int sh = (i < M ? s[i] : 0) + tj;
+        unsigned long long aw[WW];
 #pragma unroll
-      for (int n = 0; n < 16; ++n) sts64(x_write + xpose_row_offset(n), (unsigned long long)top16[n]);
-      __syncwarp();
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        unsigned long long u0, u1, u2, u3;
-        lds128(x_read + 32 * e, u0, u1);
-        lds128(x_read + 32 * e + 16, u2, u3);
-        acc[e][4] = u0 + (u1 << 16);
-        acc[e][5] = u2 + (u3 << 16);
+        for (int k = 0; k < WW; ++k) aw[k] = a[k];
+        out[e] = finish_element<WW, NW, LEAN>(aw, ct, sh);
       }
-      __syncwarp();
-    }
-    const int64_t i0 = seg + 4 * q;
-    if (i0 < M) {
-      const int tj = t[j];
-      double out[4];
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int sh = (i0 + e < M ? s[i0 + e] : 0) + tj;
-        unsigned long long a[WW];
-#pragma unroll
-        for (int k = 0; k < WW; ++k) a[k] = acc[e][k];
-        out[e] = finish_element<WW, NW, LEAN>(a, ct, sh);
-      }
-      double* dst = C + i0 + j * ldc;
-      if (i0 + 4 <= M && vec_store) {
-        reinterpret_cast<double2*>(dst)[0] = make_double2(out[0], out[1]);
-        reinterpret_cast<double2*>(dst)[1] = make_double2(out[2], out[3]);
+      const int64_t i = i0 + 2 * h;
+      if (i + 2 <= M && vec_store) {
+        *reinterpret_cast<double2*>(dst + 2 * h) = make_double2(out[0], out[1]);
       } else {
-#pragma unroll
-        for (int e = 0; e < 4; ++e)
-          if (i0 + e < M) dst[e] = out[e];
+        if (i < M) dst[2 * h] = out[0];
+        if (i + 1 < M) dst[2 * h + 1] = out[1];
       }
     }
+    __syncwarp();  // the crossing buffer is rewritten by the next unit
   }
 }
 
@@ -567,13 +595,15 @@ cudaError_t launch_crt(const Geometry& g, const CrtTable& ct, const uint8_t* res
                        res_ld >= rows16;
   if (aligned) {
     const int64_t units = ((g.M + 127) / 128) * g.N;
-    const int64_t cap = (int64_t)device_sm_count() * 6;
-    const unsigned grid = (unsigned)std::min<int64_t>((units + 7) / 8, cap);
+    // persistent grid: as many blocks as stay resident (three of eight warps, or four of four with three digit tiles)
+    const int64_t wpb = ww <= 4 ? kCrtWarps(2) : kCrtWarps(3);
+    const int64_t cap = (int64_t)device_sm_count() * (ww <= 4 ? 3 : 4);
+    const unsigned grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>((units + wpb - 1) / wpb, cap));
     const int nhi = ct.L <= 16 ? 0 : ct.L <= 20 ? 1 : ct.L <= 24 ? 2 : 3;
     const bool lean = ct.words <= 5 && ww <= 4 && ct.p_bits >= 101 && ct.p_bits <= 126;   // 16 to 19 moduli
     const bool lean5 = ct.words <= 6 && ww <= 5 && ct.p_bits >= 129 && ct.p_bits <= 158;  // 20 to 23 moduli
 #define OZK_CRT_MMA(NT, NHI, WW, NW, LEAN)                                                                           \
-  crt_mma_kernel<NT, NHI, WW, NW, LEAN><<<grid, 256, 0, st>>>(ct, res, (size_t)res_ld, res_stride, s, t, g.M, g.N, rows16, C, ldc)
+  crt_mma_kernel<NT, NHI, WW, NW, LEAN><<<grid, kCrtWarps(NT) * 32, 0, st>>>(ct, res, (size_t)res_ld, res_stride, s, t, g.M, g.N, rows16, C, ldc)
     bool launched = true;
     if (lean && nhi == 0) OZK_CRT_MMA(2, 0, 4, 5, 4);
     else if (lean && nhi == 1) OZK_CRT_MMA(2, 1, 4, 5, 4);

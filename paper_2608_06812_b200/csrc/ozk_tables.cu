@@ -253,10 +253,30 @@ bool build_crt_table(int L, CrtTable* t) {
   for (int i = 0; i < kCrtWords; ++i) t->P[i] = P.w[i];
   Big h = big_div_small(P, 2, nullptr);
   for (int i = 0; i < kCrtWords; ++i) t->halfP[i] = h.w[i];
+  {
+    uint64_t borrow = 0;
+    for (int i = 0; i < 4; ++i) {
+      const uint64_t d = (uint64_t)0 - P.w[i] - borrow;
+      t->negP[i] = (uint32_t)d;
+      borrow = (d >> 32) & 1u;
+    }
+  }
   t->inv_P = 1.0 / big_to_double(P);
-  t->q_scale = ldexp(t->inv_P, 96) * (1.0 - ldexp(1.0, -30));
-  t->q_scale128 = ldexp(t->inv_P, 128) * (1.0 - ldexp(1.0, -30));
   t->p_bits = big_bits(P);
+  t->q_mul = 0, t->q_word = 0, t->q_bit = 0;
+  if (t->p_bits >= 100 && t->p_bits <= 160) {
+    // largest c with c P 2^28 <= 2^(52 + shift) (2^28 - 1), by bisection
+    const int shift = t->p_bits - 21;
+    const Big rhs = big_shl(big_from((1ull << 28) - 1), 52 + shift);
+    uint64_t lo = 0, hi = 0xFFFFFFFFull;
+    while (lo < hi) {
+      const uint64_t mid = (lo + hi + 1) / 2;
+      if (big_cmp(big_shl(big_mul_small(P, (uint32_t)mid), 28), rhs) <= 0) lo = mid; else hi = mid - 1;
+    }
+    t->q_mul = (uint32_t)lo;
+    t->q_word = shift / 32;
+    t->q_bit = shift % 32;
+  }
   for (int tile = 0; tile < 3; ++tile)
     for (int lane = 0; lane < 32; ++lane) {
       const int col = lane >> 2, q = lane & 3;
