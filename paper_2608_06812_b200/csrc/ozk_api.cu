@@ -50,7 +50,7 @@ bool make_geometry_impl(int64_t M, int64_t N, int64_t K, int L, Geometry* g, int
   g->off_status = off;
   off += align_up(sizeof(StatusBlock), 1024);
   g->off_lut = off;
-  off += align_up((size_t)kMaxModuli * kLutStride * sizeof(uint16_t), 1024);
+  off += align_up(kEncTableBytes, 1024);
   g->off_amax_a = off;
   off += (size_t)g->Mp * 8;
   g->off_amax_b = off;

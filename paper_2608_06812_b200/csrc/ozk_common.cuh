@@ -14,8 +14,16 @@ constexpr int kTileKNibbles = 256;   // k extent of one pipeline stage: 256 E2M1
 constexpr int kTileKBytes = 128;
 constexpr int kMaxModuli = OZK_MAX_MODULI;
 constexpr int kCrtWords = 6;         // 192-bit integers cover sum r_l w_l for all 27 moduli
-constexpr int kLutStride = 192;      // 16-bit entries per modulus in the limb-pair table: centred residues -96 .. 95
-constexpr int kLutOffset = 96;
+// Encoder tables in the workspace (rebuilt by a small kernel at every call):
+//   limb-pair tables   per modulus two byte tables of kLimbTabStride entries indexed by (residue + 2^62) mod m: the
+//                      E2M1 codes of a limb pair (c0, c1), c0 + 13 c1 = residue (mod m), as code(c0) | code(c1) << 4 for
+//                      elements at even k and code(c1) | code(c0) << 4 for elements at odd k
+//   B fragments        of the encoder's mma.sync (kEncTiles tiles of two moduli, 32 lanes, two registers)
+constexpr int kLimbTabStride = 176;  // >= 169, a multiple of 16
+constexpr int kEncTiles = (kMaxModuli + 1) / 2;
+constexpr size_t kLimbTabBytes = (size_t)kMaxModuli * 2 * kLimbTabStride;
+constexpr size_t kEncFragBytes = (size_t)kEncTiles * 32 * 2 * sizeof(uint32_t);
+constexpr size_t kEncTableBytes = kLimbTabBytes + kEncFragBytes;
 constexpr int64_t kChunkK = OZK_CHUNK_K;  // longest k range of one limb-GEMM launch: 128 K <= 2^24 keeps FP32 sums exact (|limb| <= 8)
 constexpr int64_t kMaxK = OZK_MAX_K;      // 16 ranges; the grid limits of the O(N^2) kernels lie beyond it
 
@@ -47,11 +55,11 @@ struct ModulusTable {
   int L;
   int m[kMaxModuli];
   uint32_t recip[kMaxModuli];      // floor(2^32 / m)
-  // encoder constants (FP32 arithmetic on exact small integers): centred residues of 2^14, 2^28, 2^42
-  float c14[kMaxModuli], c28[kMaxModuli], c42[kMaxModuli];
-  float c56[kMaxModuli];           // centred residue of 2^56: fifth piece of integers wider than 56 bits
-  float inv_m[kMaxModuli];         // 1 / m rounded to FP32
-  float m_f[kMaxModuli];           // m
+  // encoder constants: the residue of a converted integer a is taken from the bytes b_p of a + 2^62 (non-negative) as
+  //   t = sum_p b_p c8[p] < 2^19,  t = a + 2^62 (mod m);   t mod m = t - mulhi(t, floor(2^32 / m) + 1) m
+  // (the limb-pair tables are indexed by t mod m, i.e. shifted by 2^62 mod m)
+  uint8_t c8[kMaxModuli][8];       // 2^(8 p) mod m
+  int off62[kMaxModuli];           // 2^62 mod m
 };
 
 struct CrtTable {

@@ -27,4 +27,21 @@ __device__ __forceinline__ unsigned long long to_integer_magnitude(double x, int
   return q + ((rem > half) || (rem == half && (q & 1ull)) ? 1ull : 0ull);
 }
 
+// The same conversion on the FP64 pipe: round(x * 2^s) with ties to even as a signed 64-bit integer.  Scaling by
+// a power of two is exact as long as the product is a normal number, so x * 2^s is formed in two exact steps
+// (2^s itself is not a double for s beyond 1023: rows of tiny or huge numbers) and rounded once by the
+// conversion instruction.  An intermediate that falls into the subnormal range belongs to an element at least
+// 2^900 below its row maximum: its converted value is 0 either way.  Requires |x * 2^s| <= 2^62.
+struct ScalePair {
+  double f1, f2;  // 2^s = f1 * f2, both normal powers of two
+};
+__device__ __forceinline__ ScalePair make_scale(int s) {
+  const int s1 = max(-1000, min(1000, s));
+  ScalePair p;
+  p.f1 = __longlong_as_double((long long)(s1 + 1023) << 52);
+  p.f2 = __longlong_as_double((long long)(s - s1 + 1023) << 52);
+  return p;
+}
+__device__ __forceinline__ long long to_integer_rne(double x, const ScalePair& p) { return __double2ll_rn(x * p.f1 * p.f2); }
+
 }  // namespace ozk

@@ -93,7 +93,7 @@ bool make_host_layout(int64_t M, int64_t N, int64_t K, int L, HostLayout* h) {
   h->off_status = off;
   off += 1024;
   h->off_lut = off;
-  off += up((size_t)kMaxModuli * kLutStride * sizeof(uint16_t));
+  off += up(kEncTableBytes);
   h->stride_amax_a = up((size_t)g.Mp * 8);
   h->stride_s = up((size_t)g.Mp * 4);
   h->off_amax_a = off;

@@ -19,36 +19,61 @@ namespace {
 __device__ __constant__ int8_t kDoubledE2M1[8] = {0, 1, 2, 3, 4, 6, 8, 12};
 
 // ------------------------------------------------------------------------------------
-// Limb-pair table: for modulus m and every centred residue r in [-96, 96) one 16-bit entry (index
-// r + 96) holding the E2M1 codes of a limb pair (c0, c1) with c0 + 13 c1 = r (mod m): code(c0) in bits
-// 0..3, code(c1) in bits 8..11.  Both limbs are in S with |c| <= 8; among the valid pairs the one with the
-// fewest negative limbs, then the smallest max(|c0|,|c1|), then the smallest |c0|+|c1| is taken.  The encoder's residue is centred (|r| <= m/2 + 2 <= 87), so the sign of the converted
-// integer needs no separate handling.
+// Encoder tables (layout in ozk_common.cuh).  Limb pairs: for modulus m and every residue r in [0, m) the E2M1
+// codes of a pair (c0, c1) with c0 + 13 c1 = r (mod m), both limbs in S with |c| <= 8; among the valid pairs the one
+// with the fewest negative limbs, then the smallest max(|c0|, |c1|), then the smallest |c0| + |c1| is taken.
+// The tables are indexed by t = (residue + 2^62) mod m, the value the encoder's contraction yields.
+// Block l < L writes the two byte tables of modulus l; block L writes the B fragments of the encoder's MMA.
 // ------------------------------------------------------------------------------------
-__global__ void build_lut_kernel(ModulusTable mt, uint16_t* __restrict__ lut) {
+__global__ void build_lut_kernel(ModulusTable mt, uint8_t* __restrict__ tables) {
   const int l = blockIdx.x;
+  if (l == mt.L) {
+    // B fragments (m16n8k32, u8 x u8): tile T holds the moduli 2 T and 2 T + 1.  Column n of a tile belongs to
+    // lane n / 2 of every quad and to modulus 2 T + n % 2: it is non-zero only in the k slots of that lane (bytes 0..3
+    // of its element in slots 4 q .. 4 q + 3, bytes 4..7 in slots 16 + 4 q ..), where it holds 2^(8 p) mod m.  Lane (g, q) stores column g of the tile: register 0 = its slots 4 q .., register 1 = slots 16 + 4 q ...
+    uint32_t* frag = reinterpret_cast<uint32_t*>(tables + kLimbTabBytes);
+    for (int x = threadIdx.x; x < kEncTiles * 32; x += blockDim.x) {
+      const int T = x >> 5, lane = x & 31, g = lane >> 2, q = lane & 3;
+      const int mod = 2 * T + (g & 1);
+      uint32_t r0 = 0, r1 = 0;
+      if ((g >> 1) == q && mod < mt.L) {
+        for (int p = 0; p < 4; ++p) {
+          r0 |= (uint32_t)mt.c8[mod][p] << (8 * p);
+          r1 |= (uint32_t)mt.c8[mod][4 + p] << (8 * p);
+        }
+      }
+      frag[2 * x] = r0;
+      frag[2 * x + 1] = r1;
+    }
+    return;
+  }
   const int m = mt.m[l];
-  for (int x = threadIdx.x; x < kLutStride; x += blockDim.x) {
-    const int rho = ((x - kLutOffset) % m + m) % m;
-    int best_key = 1 << 30, best = 0;
-    for (int i1 = 0; i1 < 16; ++i1) {
-      for (int i0 = 0; i0 < 16; ++i0) {
-        if ((i0 == 8) || (i1 == 8)) continue;  // skip the negative-zero codes
-        const int c0 = kDoubledE2M1[i0 & 7] * ((i0 & 8) ? -1 : 1);
-        const int c1 = kDoubledE2M1[i1 & 7] * ((i1 & 8) ? -1 : 1);
-        if ((c0 + 13 * c1 - rho) % m != 0) continue;
-        const int a0 = abs(c0), a1 = abs(c1);
-        if (max(a0, a1) > 8) continue;  // every class of every modulus has a pair with |c| <= 8 (keeps 128 K <= 2^24)
-        // fewest negative limbs first (sign changes in the operand streams cost power on the tensor pipe:
-        // a few per cent of the limb GEMM's time under the power cap), then smallest magnitudes
-        const int key = 2000 * ((c0 < 0) + (c1 < 0)) + max(a0, a1) * 64 + (a0 + a1);
-        if (key < best_key) {
-          best_key = key;
-          best = (i1 << 8) | i0;
+  uint8_t* even = tables + (size_t)l * 2 * kLimbTabStride;
+  uint8_t* odd = even + kLimbTabStride;
+  for (int idx = threadIdx.x; idx < kLimbTabStride; idx += blockDim.x) {
+    int best_key = 1 << 30, best0 = 0, best1 = 0;
+    if (idx < m) {
+      const int rho = (idx - mt.off62[l] + m) % m;  // the residue whose shifted value is idx
+      for (int i1 = 0; i1 < 16; ++i1) {
+        for (int i0 = 0; i0 < 16; ++i0) {
+          if ((i0 == 8) || (i1 == 8)) continue;  // skip the negative-zero codes
+          const int c0 = kDoubledE2M1[i0 & 7] * ((i0 & 8) ? -1 : 1);
+          const int c1 = kDoubledE2M1[i1 & 7] * ((i1 & 8) ? -1 : 1);
+          if ((c0 + 13 * c1 - rho) % m != 0) continue;
+          const int a0 = abs(c0), a1 = abs(c1);
+          if (max(a0, a1) > 8) continue;  // every class of every modulus has a pair with |c| <= 8 (keeps 128 K <= 2^24)
+          // fewest negative limbs first (sign changes in the operand streams cost power on the tensor pipe:
+          // a few per cent of the limb GEMM's time under the power cap), then smallest magnitudes
+          const int key = 2000 * ((c0 < 0) + (c1 < 0)) + max(a0, a1) * 64 + (a0 + a1);
+          if (key < best_key) {
+            best_key = key;
+            best0 = i0, best1 = i1;
+          }
         }
       }
     }
-    lut[l * kLutStride + x] = (uint16_t)best;
+    even[idx] = (uint8_t)(best0 | (best1 << 4));
+    odd[idx] = (uint8_t)(best1 | (best0 << 4));
   }
 }
 
@@ -136,122 +161,152 @@ __global__ void finalize_shifts_kernel(const unsigned long long* __restrict__ am
   shifts[i] = s;
 }
 
-// Eight consecutive-k integers of one plane row as signed 14-bit pieces, held in FP32
-// (a = x3 2^42 + x2 2^28 + x1 2^14 + x0, every piece carrying the sign of a).  Integers of up to 56 bits
-// need four pieces; kWide adds x4 2^56 for the extended-capacity mode (up to 62 bits).
-template <bool kWide>
-struct Piece8 {
-  float x0[8], x1[8], x2[8], x3[8], x4[kWide ? 8 : 1];
-};
+// ------------------------------------------------------------------------------------
+// Residues and limb codes of eight consecutive-k integers per thread, all moduli (Section 5.1), with the
+// residue contraction on the tensor cores.
+//
+// The converted integer a (|a| <= 2^62) is shifted to v = a + 2^62 >= 0, whose eight bytes b_p give
+//   t_l = sum_p b_p (2^(8 p) mod m_l)  =  a + 2^62  (mod m_l),   0 <= t_l < 2^19:
+// an [elements x 8 bytes] by [8 bytes x moduli] product of bytes, run as mma.sync.m16n8k32 (u8 x u8 -> s32).
+// The two 32-bit halves of v ARE the A fragments: a lane puts the halves of two of its elements into its own k
+// slots of MMA rows g and g + 8, and the B fragments are block-sparse (a column answers only to the k slots of
+// the lane that will read it, see build_lut_kernel), so the accumulators a lane gets back belong to its own
+// elements: no data crosses lanes.  One MMA yields 2 elements x 2 moduli per lane; a tile of two moduli takes
+// four MMAs for the thread's eight elements.  Then per element and modulus: t mod m = t - mulhi(t, recip1) m,
+// one byte read from the limb-pair table, which is indexed by that shifted residue (byte tables keep a warp's 32
+// reads within 32 to 43 words: almost no bank conflicts), and the nibbles of eight elements are merged into the
+// two 32-bit plane words with byte permutes and three logic operations.
+// ------------------------------------------------------------------------------------
+__device__ __forceinline__ void mma_u8u8_16832(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                               uint32_t b1) {
+  asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+      : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(0));
+}
 
-template <bool kWide>
-__device__ __forceinline__ void split8(const unsigned long long (&mag)[8], const bool (&neg)[8], Piece8<kWide>& p) {
+// v = (converted integer) + 2^62 of the thread's eight elements, as low and high words
+struct Shifted8 {
+  uint32_t lo[8], hi[8];
+};
+__device__ __forceinline__ void shift8(const long long (&a)[8], Shifted8& v) {
 #pragma unroll
   for (int e = 0; e < 8; ++e) {
-    const float sgn = neg[e] ? -1.0f : 1.0f;
-    p.x0[e] = sgn * (float)(uint32_t)(mag[e] & 0x3FFFull);
-    p.x1[e] = sgn * (float)(uint32_t)((mag[e] >> 14) & 0x3FFFull);
-    p.x2[e] = sgn * (float)(uint32_t)((mag[e] >> 28) & 0x3FFFull);
-    if (kWide) {
-      p.x3[e] = sgn * (float)(uint32_t)((mag[e] >> 42) & 0x3FFFull);
-      p.x4[e] = sgn * (float)(uint32_t)(mag[e] >> 56);  // <= 2^6
-    } else {
-      p.x3[e] = sgn * (float)(uint32_t)(mag[e] >> 42);  // < 2^14
-    }
+    const unsigned long long x = (unsigned long long)a[e] + (1ull << 62);
+    v.lo[e] = (uint32_t)x;
+    v.hi[e] = (uint32_t)(x >> 32);
   }
 }
 
-// Residues of the eight values mod m_l and their limb codes packed as 8 nibbles per limb, on the FP32
-// pipe (the integer pipes of this GPU run at half its rate).  All quantities are small exact integers:
-//   t = x0 + x1 c14 + x2 c28 + x3 c42 (+ x4 c56)   |t| < 2^22   (c = centred residues of 2^14, 2^28, ...;
-//                                                  |c| <= 84: 16383 (1 + 3 * 84) + 63 * 84 < 2^22)
-//   q = round(t / m) by the add-2^23 trick,  r = t - q m   centred residue, |r| <= m/2 + 2
-//   byte offset of the table entry = 2 (r + 96), read from the low bits of 2 r + 192 + 1.5 * 2^23
-// Two neighbouring k share a byte: entry(even k) | entry(odd k) << 4 has the byte of limb 0 in bits
-// 0..7 and the byte of limb 1 in bits 8..15.
-template <bool kWide>
-__device__ __forceinline__ void encode8(const Piece8<kWide>& p, float c14, float c28, float c42, float c56, float inv_m, float m_f,
-                                        const uint16_t* __restrict__ lut_l, uint32_t& w0, uint32_t& w1) {
-  constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23 (bit pattern 0x4B400000): adding it rounds to an integer in the low mantissa bits
-  // shared-memory address of the table minus the bit pattern of the magic constant: one integer add turns the
-  // float below into the address of its entry
-  const uint32_t delta = (uint32_t)__cvta_generic_to_shared(lut_l) - 0x4B400000u;
-  uint32_t pair[4];
+// The moduli as compile-time constants: the loop over the moduli below is fully unrolled, so that the modulus, its
+// reciprocal and the shared-memory address of its table are immediates of the three instructions per element and
+// modulus.  This is the list the selection rule of Section 5.1 produces (169 first, then descending, pairwise
+// coprime, two-limb representable); the launcher checks it against the host's own search before every launch.
+__host__ __device__ constexpr int enc_modulus(int l) {
+  constexpr int kList[kMaxModuli + 1] = {169, 115, 113, 112, 111, 109, 107, 103, 101, 97, 89, 83, 79, 73,
+                                         71,  67,  61,  59,  53,  47,  43,  41,  31,  29, 19, 17, 11, 1};
+  return kList[l < kMaxModuli ? l : kMaxModuli];
+}
+bool enc_moduli_match(const ModulusTable& mt) {
+  for (int l = 0; l < mt.L; ++l)
+    if (mt.m[l] != enc_modulus(l)) return false;
+  return true;
+}
+
+// Shared-memory copy of the encoder tables (static arrays of the calling kernel: their addresses are compile-time
+// constants): limb-pair byte tables of the first L moduli and the B fragments.
+struct EncTables {
+  uint8_t limb[kMaxModuli][2][kLimbTabStride];
+  uint2 frag[kEncTiles][32];
+};
+static_assert(sizeof(EncTables) == kLimbTabBytes + kEncFragBytes, "shared copy mirrors the workspace layout");
+__device__ __forceinline__ void load_tables(const uint8_t* __restrict__ tables, int L, EncTables* tab) {
+  const int limb_vec = L * 2 * kLimbTabStride / 16, frag_vec = (int)(kEncFragBytes / 16);
+  const uint4* src = reinterpret_cast<const uint4*>(tables);
+  const uint4* src_frag = reinterpret_cast<const uint4*>(tables + kLimbTabBytes);
+  uint4* dst = reinterpret_cast<uint4*>(tab->limb);
+  uint4* dst_frag = reinterpret_cast<uint4*>(tab->frag);
+  for (int i = threadIdx.x; i < limb_vec; i += blockDim.x) dst[i] = src[i];
+  for (int i = threadIdx.x; i < frag_vec; i += blockDim.x) dst_frag[i] = src_frag[i];
+}
+
+// Plane words of the thread's eight elements for every modulus, stored at dst + plane * plane_bytes.
+// Warp-collective (all 32 lanes must call it).
+__device__ __forceinline__ void encode_planes(const Shifted8& v, int L, const EncTables& tab, uint8_t* dst, size_t plane_bytes) {
+  const int lane = threadIdx.x & 31;
 #pragma unroll
-  for (int h = 0; h < 4; ++h) {
-    uint32_t v[2];
+  for (int T = 0; T < kEncTiles; ++T) {
+    if (2 * T >= L) break;
+    const uint2 b = tab.frag[T][lane];
+    int d[4][4];  // d[h]: elements 2 h (d[h][0], d[h][1]: moduli 2 T, 2 T + 1) and 2 h + 1 (d[h][2], d[h][3])
 #pragma unroll
-    for (int o = 0; o < 2; ++o) {
-      const int e = 2 * h + o;
-      float t = fmaf(p.x3[e], c42, fmaf(p.x2[e], c28, fmaf(p.x1[e], c14, p.x0[e])));
-      if (kWide) t = fmaf(p.x4[e], c56, t);
-      const float q = fmaf(t, inv_m, kMagic) - kMagic;
-      const float r = fmaf(-q, m_f, t);
-      const uint32_t addr = __float_as_uint(fmaf(r, 2.0f, kMagic + 2.0f * kLutOffset)) + delta;  // table + 2 (r + 96)
-      asm("ld.shared.u16 %0, [%1];" : "=r"(v[o]) : "r"(addr));
+    for (int h = 0; h < 4; ++h) mma_u8u8_16832(d[h], v.lo[2 * h], v.lo[2 * h + 1], v.hi[2 * h], v.hi[2 * h + 1], b.x, b.y);
+#pragma unroll
+    for (int mm = 0; mm < 2; ++mm) {
+      const int l = 2 * T + mm;
+      if (l >= kMaxModuli || l >= L) break;  // odd modulus count: the last tile has one modulus only
+      const uint32_t m = (uint32_t)enc_modulus(l), recip1 = (uint32_t)(0x100000000ull / (unsigned long long)enc_modulus(l)) + 1u;
+      const uint8_t* even = tab.limb[l][0];
+      const uint8_t* odd = tab.limb[l][1];
+      uint32_t ea[4], eb[4];  // table bytes of the elements at even / odd k
+#pragma unroll
+      for (int h = 0; h < 4; ++h) {
+        const uint32_t t0 = (uint32_t)d[h][mm], t1 = (uint32_t)d[h][2 + mm];
+        ea[h] = even[t0 - __umulhi(t0, recip1) * m];
+        eb[h] = odd[t1 - __umulhi(t1, recip1) * m];
+      }
+      const uint32_t xa = __byte_perm(__byte_perm(ea[0], ea[1], 0x0040), __byte_perm(ea[2], ea[3], 0x0040), 0x5410);
+      const uint32_t xb = __byte_perm(__byte_perm(eb[0], eb[1], 0x0040), __byte_perm(eb[2], eb[3], 0x0040), 0x5410);
+      // even table: code(c0) | code(c1) << 4, odd table: code(c1) | code(c0) << 4
+      *reinterpret_cast<uint32_t*>(dst + (size_t)(2 * l) * plane_bytes) = (xa & 0x0F0F0F0Fu) | (xb & 0xF0F0F0F0u);
+      *reinterpret_cast<uint32_t*>(dst + (size_t)(2 * l + 1) * plane_bytes) = ((xa >> 4) & 0x0F0F0F0Fu) | ((xb << 4) & 0xF0F0F0F0u);
     }
-    pair[h] = v[1] * 16u + v[0];  // the nibbles do not overlap: one multiply-add instead of shift and or
   }
-  const uint32_t t0 = __byte_perm(pair[0], pair[1], 0x5410), t1 = __byte_perm(pair[2], pair[3], 0x5410);
-  w0 = __byte_perm(t0, t1, 0x6420);
-  w1 = __byte_perm(t0, t1, 0x7531);
 }
 
 // ------------------------------------------------------------------------------------
 // B side: plane row = column j of B, source already K-contiguous.
-// Block = 256 threads = 2048 consecutive k of one column; thread = 8 consecutive k.
+// Block = 256 threads = 2048 consecutive k of one column; thread = 8 consecutive k (a warp = 256 k: whole warps
+// lie inside or outside the padded K, which is a multiple of 256).
 // ------------------------------------------------------------------------------------
-template <bool kWide>
 __global__ void __launch_bounds__(256) encode_cols_kernel(const double* __restrict__ B, int64_t ldb, int64_t N, int64_t K,
-                                                          int64_t Kp, ModulusTable mt, const uint16_t* __restrict__ lut,
+                                                          int64_t Kp, int L, const uint8_t* __restrict__ tables,
                                                           const int32_t* __restrict__ shifts, uint8_t* __restrict__ planes,
                                                           size_t plane_bytes, size_t pitch, int64_t* __restrict__ int_out, int reps) {
-  extern __shared__ __align__(16) uint16_t lut_s[];
-  {  // the table is copied once per block and reused for `reps` chunks of 2048 k
-    const uint4* src = reinterpret_cast<const uint4*>(lut);
-    uint4* dst = reinterpret_cast<uint4*>(lut_s);
-    for (int i = threadIdx.x; i < mt.L * kLutStride / 8; i += blockDim.x) dst[i] = src[i];
-  }
+  __shared__ __align__(16) EncTables tab;
+  load_tables(tables, L, &tab);  // copied once per block and reused for `reps` chunks of 2048 k
   __syncthreads();
   const int64_t j = blockIdx.x;
   for (int rep = 0; rep < reps; ++rep) {
-  const int64_t k = (((int64_t)blockIdx.y * reps + rep) * blockDim.x + threadIdx.x) * 8;
-  if (k >= Kp) return;
-  unsigned long long mag[8];
-  bool neg[8];
+    const int64_t k = (((int64_t)blockIdx.y * reps + rep) * blockDim.x + threadIdx.x) * 8;
+    if (k >= Kp) return;  // warp-uniform
+    long long a[8];
 #pragma unroll
-  for (int e = 0; e < 8; ++e) mag[e] = 0, neg[e] = false;
-  if (j < N && k < K) {
-    const int s = shifts[j];
-    const double* src = B + j * ldb + k;
-    if (k + 8 <= K && ((reinterpret_cast<uintptr_t>(src) & 15) == 0)) {
-      const double2* s2 = reinterpret_cast<const double2*>(src);
+    for (int e = 0; e < 8; ++e) a[e] = 0;
+    if (j < N && k < K) {
+      const ScalePair sc = make_scale(shifts[j]);
+      const double* src = B + j * ldb + k;
+      if (k + 8 <= K && ((reinterpret_cast<uintptr_t>(src) & 15) == 0)) {
+        const double2* s2 = reinterpret_cast<const double2*>(src);
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const double2 v = __ldg(s2 + e);
-        mag[2 * e] = to_integer_magnitude(v.x, s, &neg[2 * e]);
-        mag[2 * e + 1] = to_integer_magnitude(v.y, s, &neg[2 * e + 1]);
+        for (int e = 0; e < 4; ++e) {
+          const double2 x = __ldg(s2 + e);
+          a[2 * e] = to_integer_rne(x.x, sc);
+          a[2 * e + 1] = to_integer_rne(x.y, sc);
+        }
+      } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+          if (k + e < K) a[e] = to_integer_rne(__ldg(src + e), sc);
       }
-    } else {
+      if (int_out) {
 #pragma unroll
-      for (int e = 0; e < 8; ++e)
-        if (k + e < K) mag[e] = to_integer_magnitude(__ldg(src + e), s, &neg[e]);
+        for (int e = 0; e < 8; ++e)
+          if (k + e < K) int_out[j * K + k + e] = a[e];
+      }
     }
-    if (int_out) {
-#pragma unroll
-      for (int e = 0; e < 8; ++e)
-        if (k + e < K) int_out[j * K + k + e] = neg[e] ? -(long long)mag[e] : (long long)mag[e];
-    }
-  }
-  Piece8<kWide> p;
-  split8<kWide>(mag, neg, p);
-  uint8_t* dst = planes + (size_t)j * pitch + (size_t)(k / 2);
-  for (int l = 0; l < mt.L; ++l) {
-    uint32_t w0, w1;
-    encode8<kWide>(p, mt.c14[l], mt.c28[l], mt.c42[l], mt.c56[l], mt.inv_m[l], mt.m_f[l], lut_s + l * kLutStride, w0, w1);
-    *reinterpret_cast<uint32_t*>(dst + (size_t)(2 * l) * plane_bytes) = w0;
-    *reinterpret_cast<uint32_t*>(dst + (size_t)(2 * l + 1) * plane_bytes) = w1;
-  }
+    Shifted8 v;
+    shift8(a, v);
+    encode_planes(v, L, tab, planes + (size_t)j * pitch + (size_t)(k / 2), plane_bytes);
   }
 }
 
@@ -268,25 +323,18 @@ constexpr int kRowTileK = 128;
 constexpr int kGroupStride = 9;                                         // doubles per group of 8 k (8 used)
 constexpr int kRowStride = (kRowTileK / 8) * kGroupStride + 1;          // doubles per row: 145, odd
 
-template <bool kWide>
 __global__ void __launch_bounds__(256) encode_rows_kernel(const double* __restrict__ A, int64_t lda, int64_t M, int64_t K,
-                                                          int64_t Kp, ModulusTable mt, const uint16_t* __restrict__ lut,
+                                                          int64_t Kp, int L, const uint8_t* __restrict__ tables,
                                                           const int32_t* __restrict__ shifts, uint8_t* __restrict__ planes,
                                                           size_t plane_bytes, size_t pitch, int64_t* __restrict__ int_out, int reps) {
-  extern __shared__ __align__(16) uint8_t smem[];
-  uint16_t* lut_s = reinterpret_cast<uint16_t*>(smem);                          // L * kLutStride entries
-  const int lut_bytes = (mt.L * kLutStride * (int)sizeof(uint16_t) + 15) & ~15;
-  double* in_s = reinterpret_cast<double*>(smem + lut_bytes);                    // [16][145] doubles
+  __shared__ __align__(16) EncTables tab;
+  __shared__ double in_s[kRowTile * kRowStride];
   const int t = threadIdx.x;
   const int64_t i0 = (int64_t)blockIdx.x * kRowTile;
-  {  // the table is copied once per block and reused for `reps` tiles along k
-    const uint4* src = reinterpret_cast<const uint4*>(lut);
-    uint4* dst = reinterpret_cast<uint4*>(lut_s);
-    for (int i = t; i < mt.L * kLutStride / 8; i += blockDim.x) dst[i] = src[i];
-  }
+  load_tables(tables, L, &tab);  // copied once per block and reused for `reps` tiles along k
   const int r = t >> 4, g = t & 15;  // encode role: row r, k group g
   const int64_t i = i0 + r;
-  const int s = shifts[i];           // shifts has Mp entries; padded rows hold 0
+  const ScalePair sc = make_scale(shifts[i]);  // shifts has Mp entries; padded rows hold 0
   for (int rep = 0; rep < reps; ++rep) {
     const int64_t k0 = ((int64_t)blockIdx.y * reps + rep) * kRowTileK;
     if (k0 >= Kp) break;        // uniform over the block
@@ -302,26 +350,19 @@ __global__ void __launch_bounds__(256) encode_rows_kernel(const double* __restri
       }
     }
     __syncthreads();
-    unsigned long long mag[8];
-    bool neg[8];
+    long long a[8];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) mag[e] = to_integer_magnitude(in_s[r * kRowStride + g * kGroupStride + e], s, &neg[e]);
+    for (int e = 0; e < 8; ++e) a[e] = to_integer_rne(in_s[r * kRowStride + g * kGroupStride + e], sc);
     if (int_out && i < M) {
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
         const int64_t k = k0 + 8 * g + e;
-        if (k < K) int_out[i + k * M] = neg[e] ? -(long long)mag[e] : (long long)mag[e];
+        if (k < K) int_out[i + k * M] = a[e];
       }
     }
-    Piece8<kWide> p;
-    split8<kWide>(mag, neg, p);
-    uint8_t* dst = planes + (size_t)i * pitch + (size_t)(k0 / 2) + 4 * g;
-    for (int l = 0; l < mt.L; ++l) {
-      uint32_t w0, w1;
-      encode8<kWide>(p, mt.c14[l], mt.c28[l], mt.c42[l], mt.c56[l], mt.inv_m[l], mt.m_f[l], lut_s + l * kLutStride, w0, w1);
-      *reinterpret_cast<uint32_t*>(dst + (size_t)(2 * l) * plane_bytes) = w0;
-      *reinterpret_cast<uint32_t*>(dst + (size_t)(2 * l + 1) * plane_bytes) = w1;
-    }
+    Shifted8 v;
+    shift8(a, v);
+    encode_planes(v, L, tab, planes + (size_t)i * pitch + (size_t)(k0 / 2) + 4 * g, plane_bytes);
   }
 }
 
@@ -340,7 +381,7 @@ __global__ void decode_plane_kernel(const uint8_t* __restrict__ plane, int64_t r
 }  // namespace
 
 cudaError_t launch_build_lut(const ModulusTable& mt, uint8_t* lut, cudaStream_t st) {
-  build_lut_kernel<<<mt.L, 192, 0, st>>>(mt, reinterpret_cast<uint16_t*>(lut));
+  build_lut_kernel<<<mt.L + 1, kLimbTabStride, 0, st>>>(mt, lut);
   return cudaGetLastError();
 }
 
@@ -383,23 +424,17 @@ cudaError_t launch_scan_and_shifts(const Geometry& g, const double* A, int64_t l
 // Limb planes of A (which = 0, rows of A) or of B (which = 1, columns of B).
 cudaError_t launch_encode_operand(const Geometry& g, const ModulusTable& mt, int which, const double* X, int64_t ldx,
                                   uint8_t* ws, int64_t* int_out, cudaStream_t st) {
-  const uint16_t* lut = reinterpret_cast<const uint16_t*>(ws + g.off_lut);
-  const int lut_bytes = (mt.L * kLutStride * (int)sizeof(uint16_t) + 15) & ~15;
+  const uint8_t* tables = ws + g.off_lut;
+  if (!enc_moduli_match(mt)) return cudaErrorInvalidValue;  // the kernels carry the modulus list as constants
   const int reps = 4;
-  const bool wide = g.c_bits > 56;  // integers beyond 56 bits take a fifth 14-bit piece
   if (which == 0) {
-    const size_t smem = lut_bytes + (size_t)kRowTile * kRowStride * sizeof(double);
-    auto* kernel = wide ? encode_rows_kernel<true> : encode_rows_kernel<false>;
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
     dim3 grid((unsigned)(g.Mp / kRowTile), (unsigned)((g.Kp / kRowTileK + reps - 1) / reps));
-    kernel<<<grid, 256, smem, st>>>(X, ldx, g.M, g.K, g.Kp, mt, lut, reinterpret_cast<const int32_t*>(ws + g.off_s),
-                                    ws + g.off_planes_a, g.plane_bytes_a, g.pitch, int_out, reps);
+    encode_rows_kernel<<<grid, 256, 0, st>>>(X, ldx, g.M, g.K, g.Kp, mt.L, tables, reinterpret_cast<const int32_t*>(ws + g.off_s),
+                                             ws + g.off_planes_a, g.plane_bytes_a, g.pitch, int_out, reps);
   } else {
     dim3 grid((unsigned)g.Np, (unsigned)(((g.Kp + 2047) / 2048 + reps - 1) / reps));
-    auto* kernel = wide ? encode_cols_kernel<true> : encode_cols_kernel<false>;
-    kernel<<<grid, 256, lut_bytes, st>>>(X, ldx, g.N, g.K, g.Kp, mt, lut, reinterpret_cast<const int32_t*>(ws + g.off_t),
-                                         ws + g.off_planes_b, g.plane_bytes_b, g.pitch, int_out, reps);
+    encode_cols_kernel<<<grid, 256, 0, st>>>(X, ldx, g.N, g.K, g.Kp, mt.L, tables, reinterpret_cast<const int32_t*>(ws + g.off_t),
+                                             ws + g.off_planes_b, g.plane_bytes_b, g.pitch, int_out, reps);
   }
   return cudaGetLastError();
 }

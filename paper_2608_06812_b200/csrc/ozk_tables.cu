@@ -208,19 +208,19 @@ bool build_modulus_table(int L, ModulusTable* t) {
   for (int i = 0; i < L; ++i) {
     uint32_t m = (uint32_t)t->m[i];
     t->recip[i] = (uint32_t)(0x100000000ull / m);
-    auto centred = [m](unsigned long long v) {
-      const long long r = (long long)(v % m);
-      return (float)(r > (long long)(m / 2) ? r - (long long)m : r);
-    };
-    t->c14[i] = centred(1ull << 14);
-    t->c28[i] = centred(1ull << 28);
-    t->c42[i] = centred(1ull << 42);
-    t->c56[i] = centred(1ull << 56);
-    t->inv_m[i] = 1.0f / (float)m;
-    t->m_f[i] = (float)m;
+    for (int p = 0; p < 8; ++p) {
+      unsigned long long pw = 1;  // 2^(8 p) mod m
+      for (int k = 0; k < 8 * p; ++k) pw = pw * 2 % m;
+      t->c8[i][p] = (uint8_t)pw;
+    }
+    unsigned long long off = 1;  // 2^62 mod m
+    for (int k = 0; k < 62; ++k) off = off * 2 % m;
+    t->off62[i] = (int)off;
   }
-  for (int i = L; i < kMaxModuli; ++i)
-    t->m[i] = 1, t->recip[i] = 0, t->c14[i] = t->c28[i] = t->c42[i] = t->c56[i] = 0.0f, t->inv_m[i] = 1.0f, t->m_f[i] = 1.0f;
+  for (int i = L; i < kMaxModuli; ++i) {
+    t->m[i] = 1, t->recip[i] = 0, t->off62[i] = 0;
+    for (int p = 0; p < 8; ++p) t->c8[i][p] = 0;
+  }
   return true;
 }
 
