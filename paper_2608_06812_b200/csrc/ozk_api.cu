@@ -146,6 +146,7 @@ ozk_status gemm_residues_chunked(const Geometry& g, const ModulusTable& mt, uint
   }
   return OZK_OK;
 }
+bool stage_timing_enabled() { return g_timing.enabled; }
 uint8_t* workspace_ptr() { return g_ws.ptr; }
 size_t workspace_bytes() { return g_ws.bytes; }
 
@@ -214,8 +215,6 @@ ozk_status ozk_get_async_status(void* stream) {
   if (cudaStreamSynchronize(st) != cudaSuccess) return OZK_ERR_CUDA;
   StatusBlock sb;
   if (cudaMemcpy(&sb, g_ws.ptr, sizeof sb, cudaMemcpyDeviceToHost) != cudaSuccess) return OZK_ERR_CUDA;
-  if (getenv("OZK_DEBUG_TIMING"))
-    fprintf(stderr, "ozk dbg: mma thread total %d, wait tmem_empty %d, wait full %d (x256 clk)\n", sb.pad[0], sb.pad[1], sb.pad[2]);
   if (sb.code != 0) {
     if (sb.code == OZK_ERR_DEVICE_TIMEOUT) fprintf(stderr, "ozk: bounded wait expired at 0x%x\n", sb.where);
     cudaMemset(g_ws.ptr, 0, sizeof(StatusBlock));

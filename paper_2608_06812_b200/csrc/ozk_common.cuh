@@ -31,8 +31,12 @@ constexpr int64_t kMaxK = OZK_MAX_K;      // 16 ranges; the grid limits of the O
 struct StatusBlock {
   int code;          // 0, OZK_ERR_NONFINITE or OZK_ERR_DEVICE_TIMEOUT (first writer wins on severity)
   int where;         // which wait gave up (role * 256 + barrier id), for diagnostics
-  int pad[62];
+  // measurement aid (written only while stage timing is enabled): clocks of the limb GEMM's issuing thread in the
+  // first CTA pair, in total and spent waiting for free tensor memory / for operand stages
+  long long mma_clk_total, mma_clk_wait_tmem, mma_clk_wait_operands;
+  int pad[56];
 };
+static_assert(sizeof(StatusBlock) == 256, "the wave counter of the limb GEMM sits at byte 512 of the same kibibyte");
 
 // ---- problem geometry ---------------------------------------------------------------
 struct Geometry {
@@ -87,6 +91,7 @@ struct CrtTable {
 // per-device facts, cached per device ordinal (ozk_api.cu)
 int device_sm_count();      // multiprocessors of the current device (0 on error)
 bool device_is_sm100();     // compute capability 10.x
+bool stage_timing_enabled();  // ozk_stage_timing_enable state (ozk_api.cu)
 
 // registered workspace and layout (ozk_api.cu)
 uint8_t* workspace_ptr();

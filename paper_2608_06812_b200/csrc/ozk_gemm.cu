@@ -48,6 +48,7 @@ struct GemmCore {
   int q_groups;        // 0: both operands use plane group l; n > 0: row side uses l / n, column side l % n
   unsigned int* wave_counter;  // optional: producers of all CTAs meet here before every wave of items
   int fast_combine;    // K <= 17476: D1 + 13 D2 stays below 2^24 and may be formed in FP32 before the release
+  int count_cycles;    // measurement aid: the issuing thread of pair 0 records where its clocks went (status block)
   StatusBlock* status;
   uint32_t scale_word;  // four copies of the UE8M0 scale byte
 };
@@ -437,22 +438,17 @@ limb_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constan
       constexpr uint32_t kIdescAll = idesc_mxf4(NQ * W);
       constexpr uint32_t kIdescButLast = idesc_mxf4(NQ > 1 ? (NQ - 1) * W : W);
       bool ok = true;
-      long long dbg_t0 = clock64(), dbg_empty = 0, dbg_full = 0;
       for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
         int l, tp, tq;
         decode_item(p, item, l, tp, tq);
         const bool skip_top = p.skip_top_first && l == 0;
-        long long dbg_a = clock64();
         if (!wait_bounded(smem_u32(&sh->tmem_empty), acc_phase ^ 1u, sh, p.status, 0x100)) break;
-        dbg_empty += clock64() - dbg_a;
         tc_fence_after();
         for (int kb = 0; kb < p.kblocks; ++kb) {
-          dbg_a = clock64();
           if (!wait_bounded(smem_u32(&sh->full[stage]), phase, sh, p.status, 0x110 + stage)) {
             ok = false;
             break;
           }
-          dbg_full += clock64() - dbg_a;
           tc_fence_after();
           const uint32_t pbase = smem_u32(tiles + stage * kStageBytes);
           const uint32_t qbase = pbase + NP * kPTileBytes;
@@ -488,11 +484,6 @@ limb_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constan
         if (!ok) break;
         mma_commit(smem_u32(&sh->tmem_full));
         acc_phase ^= 1u;
-      }
-      if (blockIdx.x == 0) {
-        p.status->pad[0] = (int)((clock64() - dbg_t0) >> 8);
-        p.status->pad[1] = (int)(dbg_empty >> 8);
-        p.status->pad[2] = (int)(dbg_full >> 8);
       }
       if (sh->abort) {  // wait for the tensor pipe to go idle before TMEM is released
         mma_commit(smem_u32(&sh->drained));
@@ -648,22 +639,23 @@ residue_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
       const uint32_t sf = tmem + kScaleCol;
       constexpr uint32_t kIdesc = idesc_mxf4_pair(2 * W);
       bool ok = true;
-      long long dbg_t0 = clock64(), dbg_empty = 0, dbg_full = 0;
+      const bool count = p.count_cycles != 0;
+      long long clk_start = count ? clock64() : 0, clk_empty = 0, clk_full = 0, clk_a = 0;
       for (int item = pair; item < total_items && ok; item += npairs) {
         int l, tp, tq;
         decode_item(p, item, l, tp, tq);
         const bool three = p.skip_top_first && l == 0;
-        long long dbg_a = clock64();
+        if (count) clk_a = clock64();
         if (!wait_bounded(smem_u32(&sh->tmem_empty), acc_phase ^ 1u, sh, p.status, 0x400)) break;
-        dbg_empty += clock64() - dbg_a;
+        if (count) clk_empty += clock64() - clk_a;
         tc_fence_after();
         for (int kb = 0; kb < p.kblocks; ++kb) {
-          dbg_a = clock64();
+          if (count) clk_a = clock64();
           if (!wait_bounded(smem_u32(&sh->full[stage]), phase, sh, p.status, 0x410 + stage)) {
             ok = false;
             break;
           }
-          dbg_full += clock64() - dbg_a;
+          if (count) clk_full += clock64() - clk_a;
           tc_fence_after();
           const uint32_t base = smem_u32(tiles + stage * kPairStageBytes);
           if (three) {
@@ -697,10 +689,10 @@ residue_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
         mma_commit_pair(smem_u32(&sh->tmem_full), (uint16_t)3);
         acc_phase ^= 1u;
       }
-      if (blockIdx.x == 0) {
-        p.status->pad[0] = (int)((clock64() - dbg_t0) >> 8);
-        p.status->pad[1] = (int)(dbg_empty >> 8);
-        p.status->pad[2] = (int)(dbg_full >> 8);
+      if (count && blockIdx.x == 0) {  // measurement aid: where the issuing thread of pair 0 spent its clocks
+        p.status->mma_clk_total = clock64() - clk_start;
+        p.status->mma_clk_wait_tmem = clk_empty;
+        p.status->mma_clk_wait_operands = clk_full;
       }
       if (sh->abort) {
         mma_commit_pair(smem_u32(&sh->drained), (uint16_t)1);
@@ -895,6 +887,17 @@ bool pair_kernel_enabled() {
   return v == 1;
 }
 
+// OZK_GEMM_THREE=0 in the environment makes the CTA-pair kernel run modulus 169 like the others (four products in two
+// instructions, the 13^2 term cancelling in the epilogue) instead of three narrower instructions: a measurement aid.
+bool three_product_enabled() {
+  static int v = -1;
+  if (v < 0) {
+    const char* e = getenv("OZK_GEMM_THREE");
+    v = (e && e[0] == '0') ? 0 : 1;
+  }
+  return v == 1;
+}
+
 template <int NP, int NQ, int W, int STAGES, class Epi>
 ozk_status launch_limb_gemm(const CUtensorMap& map_p, const CUtensorMap& map_q, const GemmCore& core,
                             const typename Epi::Params& ep, cudaStream_t st) {
@@ -939,6 +942,7 @@ ozk_status gemm_residues(const Geometry& g, const ModulusTable& mt, uint8_t* ws,
   core.skip_top_first = (mt.m[0] == 169) ? 1 : 0;  // 13^2 a1 b1 vanishes mod 169 (Section 5.1)
   core.q_groups = 0;
   core.fast_combine = (g.K <= 17476 || klen <= 17408) ? 1 : 0;  // 128 K + 13 * 64 K = 960 K < 2^24
+  core.count_cycles = 0;
   core.wave_counter = nullptr;
   core.status = reinterpret_cast<StatusBlock*>(ws + g.off_status);
   core.scale_word = 0x80808080u;  // UE8M0 byte 0x80 = 2: both operands doubled, accumulators hold integers
@@ -957,7 +961,8 @@ ozk_status gemm_residues(const Geometry& g, const ModulusTable& mt, uint8_t* ws,
     GemmCore pc = core;
     pc.tiles_p = (int)(g.Np / 256);
     pc.group = 8;  // 8 column tiles of 256: the same 2048-column band as the single-CTA kernel
-    pc.skip_top_first = (mt.m[0] == 169) ? 1 : 0;  // 13^2 a1 b1 vanishes mod 169 (Section 5.1)
+    pc.skip_top_first = (mt.m[0] == 169 && three_product_enabled()) ? 1 : 0;  // 13^2 a1 b1 vanishes mod 169 (Section 5.1)
+    pc.count_cycles = stage_timing_enabled() ? 1 : 0;
     CUtensorMap map_qh;  // 64-row boxes of the A-side planes, for the three-product form of m = 169
     if (!make_plane_map(&map_qh, planes_a, klen / 2, g.Mp, 2 * g.L, g.plane_bytes_a, 64, g.pitch)) return OZK_ERR_CUDA;
     pc.wave_counter = reinterpret_cast<unsigned int*>(ws + g.off_status + 512);
@@ -1015,6 +1020,7 @@ ozk_status gemm_int8(const uint8_t* planes_a, const uint8_t* planes_b, int64_t M
   core.q_groups = 0;
   core.wave_counter = nullptr;
   core.fast_combine = 0;
+  core.count_cycles = 0;
   core.status = status;
   core.scale_word = 0x80808080u;
   Int32Epilogue::Params ep;
@@ -1043,6 +1049,7 @@ ozk_status gemm_oz1_passes(const uint8_t* planes_a, const uint8_t* planes_b, int
   core.q_groups = 5;
   core.wave_counter = nullptr;
   core.fast_combine = 0;
+  core.count_cycles = 0;
   core.status = status;
   core.scale_word = 0x80808080u;
   Int64BlockEpilogue::Params ep;

@@ -30,7 +30,8 @@ __global__ void build_lut_kernel(ModulusTable mt, uint8_t* __restrict__ tables) 
   if (l == mt.L) {
     // B fragments (m16n8k32, u8 x u8): tile T holds the moduli 2 T and 2 T + 1.  Column n of a tile belongs to
     // lane n / 2 of every quad and to modulus 2 T + n % 2: it is non-zero only in the k slots of that lane (bytes 0..3
-    // of its element in slots 4 q .. 4 q + 3, bytes 4..7 in slots 16 + 4 q ..), where it holds 2^(8 p) mod m.  Lane (g, q) stores column g of the tile: register 0 = its slots 4 q .., register 1 = slots 16 + 4 q ...
+    // of its element in slots 4 q .. 4 q + 3, bytes 4..7 in slots 16 + 4 q ..), where it holds 2^(8 p) mod m.
+    // Lane (g, q) stores column g of the tile: register 0 = its slots 4 q .., register 1 = slots 16 + 4 q ...
     uint32_t* frag = reinterpret_cast<uint32_t*>(tables + kLimbTabBytes);
     for (int x = threadIdx.x; x < kEncTiles * 32; x += blockDim.x) {
       const int T = x >> 5, lane = x & 31, g = lane >> 2, q = lane & 3;
@@ -47,33 +48,36 @@ __global__ void build_lut_kernel(ModulusTable mt, uint8_t* __restrict__ tables) 
     }
     return;
   }
+  // one thread per candidate pair (c0, c1): the best pair of every residue class by an atomic minimum on
+  // key * 256 + pair id (equal keys: the smaller id, i.e. the smaller code of c1, then of c0)
+  __shared__ unsigned int best[kLimbTabStride];
   const int m = mt.m[l];
+  for (int idx = threadIdx.x; idx < kLimbTabStride; idx += blockDim.x) best[idx] = 0xFFFFFFFFu;
+  __syncthreads();
+  {
+    const int i1 = threadIdx.x >> 4, i0 = threadIdx.x & 15;
+    if (i0 != 8 && i1 != 8) {  // skip the negative-zero codes
+      const int c0 = kDoubledE2M1[i0 & 7] * ((i0 & 8) ? -1 : 1);
+      const int c1 = kDoubledE2M1[i1 & 7] * ((i1 & 8) ? -1 : 1);
+      const int a0 = abs(c0), a1 = abs(c1);
+      if (max(a0, a1) <= 8) {  // every class of every modulus has a pair with |c| <= 8 (keeps 128 K <= 2^24)
+        // fewest negative limbs first (sign changes in the operand streams cost power on the tensor pipe:
+        // a few per cent of the limb GEMM's time under the power cap), then smallest magnitudes
+        const int key = 2000 * ((c0 < 0) + (c1 < 0)) + max(a0, a1) * 64 + (a0 + a1);
+        const int rho = ((c0 + 13 * c1) % m + m) % m;
+        const int idx = (rho + mt.off62[l]) % m;  // the tables are indexed by the shifted residue
+        atomicMin(&best[idx], (unsigned int)key * 256u + (unsigned int)threadIdx.x);
+      }
+    }
+  }
+  __syncthreads();
   uint8_t* even = tables + (size_t)l * 2 * kLimbTabStride;
   uint8_t* odd = even + kLimbTabStride;
   for (int idx = threadIdx.x; idx < kLimbTabStride; idx += blockDim.x) {
-    int best_key = 1 << 30, best0 = 0, best1 = 0;
-    if (idx < m) {
-      const int rho = (idx - mt.off62[l] + m) % m;  // the residue whose shifted value is idx
-      for (int i1 = 0; i1 < 16; ++i1) {
-        for (int i0 = 0; i0 < 16; ++i0) {
-          if ((i0 == 8) || (i1 == 8)) continue;  // skip the negative-zero codes
-          const int c0 = kDoubledE2M1[i0 & 7] * ((i0 & 8) ? -1 : 1);
-          const int c1 = kDoubledE2M1[i1 & 7] * ((i1 & 8) ? -1 : 1);
-          if ((c0 + 13 * c1 - rho) % m != 0) continue;
-          const int a0 = abs(c0), a1 = abs(c1);
-          if (max(a0, a1) > 8) continue;  // every class of every modulus has a pair with |c| <= 8 (keeps 128 K <= 2^24)
-          // fewest negative limbs first (sign changes in the operand streams cost power on the tensor pipe:
-          // a few per cent of the limb GEMM's time under the power cap), then smallest magnitudes
-          const int key = 2000 * ((c0 < 0) + (c1 < 0)) + max(a0, a1) * 64 + (a0 + a1);
-          if (key < best_key) {
-            best_key = key;
-            best0 = i0, best1 = i1;
-          }
-        }
-      }
-    }
-    even[idx] = (uint8_t)(best0 | (best1 << 4));
-    odd[idx] = (uint8_t)(best1 | (best0 << 4));
+    const unsigned int pair = idx < m ? best[idx] & 0xFFu : 0u;
+    const unsigned int i0 = pair & 15u, i1 = pair >> 4;
+    even[idx] = (uint8_t)(i0 | (i1 << 4));
+    odd[idx] = (uint8_t)(i1 | (i0 << 4));
   }
 }
 
@@ -381,7 +385,7 @@ __global__ void decode_plane_kernel(const uint8_t* __restrict__ plane, int64_t r
 }  // namespace
 
 cudaError_t launch_build_lut(const ModulusTable& mt, uint8_t* lut, cudaStream_t st) {
-  build_lut_kernel<<<mt.L + 1, kLimbTabStride, 0, st>>>(mt, lut);
+  build_lut_kernel<<<mt.L + 1, 256, 0, st>>>(mt, lut);
   return cudaGetLastError();
 }
 
