@@ -32,9 +32,12 @@ METRIC = "effective FP64 TFLOPS (2MNK/t), Ozaki scheme II on FP4, end to end inc
 UNIT = "TFLOP/s"
 PAPER_TOTAL_TFLOPS = {4096: 10.81, 8192: 13.52, 16384: 15.26}   # the paper's end-to-end numbers, L = 19, other GPU
 FP4_PER_BF16 = 4.0                                               # nominal dense FP4 : BF16 ratio on B200
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the limb GEMM, from ncu captures of this
-# command at the same size (see profiles/): (size, moduli) -> bytes
-DRAM_TRAFFIC_BYTES = {(16384, 19): 53.4e9 + 5.1e9, (4096, 19): 0.638e9 + 0.301e9}
+NOMINAL_FP4_TFLOPS = 9000.0                                      # B200 dense FP4 (NVIDIA's doubled figures are 2:4 sparsity)
+SM_COUNT = 148
+# DRAM traffic of one limb-GEMM launch comes from an ncu capture recorded in this file together with a hash of the
+# kernel source it was taken from; a capture of other source is not reported
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "limb_gemm_dram_traffic.json")
+GEMM_SOURCES = ["paper_2608_06812_b200/csrc/ozk_gemm.cu", "paper_2608_06812_b200/csrc/ozk_ptx.cuh"]
 KERNELS_PER_STEP = 9   # lut, scan_rows, scan_cols, 2 x finalize, encode_rows, encode_cols, limb GEMM, CRT
 
 
@@ -57,7 +60,31 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-fp64-context", action="store_true")
+    ap.add_argument("--launcher-selftest", action="store_true", help="CPU-only check of the multi-rank launch and reduction (no GPU work)")
     return ap.parse_args()
+
+
+def gemm_source_hash() -> str:
+    import hashlib
+    h = hashlib.sha256()
+    for rel in GEMM_SOURCES:
+        h.update(open(os.path.join(ROOT, rel), "rb").read())
+    return h.hexdigest()
+
+
+def recorded_traffic(M: int, N: int, K: int, L: int):
+    """(bytes per launch or None, note): the ncu DRAM read + write bytes of one limb-GEMM launch at this size, if a
+    capture of the current kernel source is on record."""
+    try:
+        rec = json.load(open(TRAFFIC_FILE))
+    except (OSError, ValueError):
+        return None, "no capture on record"
+    for c in rec.get("captures", []):
+        if [c.get("M"), c.get("N"), c.get("K"), c.get("moduli")] == [M, N, K, L]:
+            if c.get("gemm_source_sha256") != gemm_source_hash():
+                return None, "the capture on record is of other kernel source"
+            return float(c["dram_read_bytes"]) + float(c["dram_write_bytes"]), c.get("command", "")
+    return None, "no capture of this size on record"
 
 
 def workload_name(n: int, L: int, phi: float, shape=None) -> str:
@@ -128,6 +155,12 @@ class ClockSampler:
 # ---------------------------------------------------------------------------------------------
 # CPU oracle legs
 # ---------------------------------------------------------------------------------------------
+def threads_used(cpu_seconds: float, wall_seconds: float) -> int:
+    """Threads a timed region kept busy on average (its process CPU time over its wall time): the big-integer loops
+    of the oracle are single-threaded Python, only its float64 matrix products use the BLAS thread pool."""
+    return max(1, int(round(cpu_seconds / max(wall_seconds, 1e-9))))
+
+
 def oracle_sample_tflops(A: np.ndarray, B: np.ndarray, L: int, block: int, repeats: int = 1) -> tuple[float, float, str, int]:
     """Times the CPU oracle, as it stands, on a block x block corner of the output (full K).
     Returns (TFLOP/s, seconds per run, description of the sample, threads used)."""
@@ -135,18 +168,31 @@ def oracle_sample_tflops(A: np.ndarray, B: np.ndarray, L: int, block: int, repea
     M, K = A.shape
     b = min(block, M, B.shape[1])
     As, Bs = np.ascontiguousarray(A[:b]), np.ascontiguousarray(B[:, :b])
-    best = float("inf")
+    best, threads = float("inf"), 1
     for _ in range(repeats):
-        t0 = time.perf_counter()
+        t0, c0 = time.perf_counter(), time.process_time()
         ozaki2.dgemm(As, Bs, L)
-        best = min(best, time.perf_counter() - t0)
-    try:
-        from threadpoolctl import threadpool_info
-        threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
-    except Exception:
-        threads = os.cpu_count() or 1
+        wall, cpu = time.perf_counter() - t0, time.process_time() - c0
+        if wall < best:
+            best, threads = wall, threads_used(cpu, wall)
     sample = f"oracle.ozaki2.dgemm on the {b}x{b} leading output block, full K={K} ({2.0 * b * b * K:.3g} flop-equivalents)"
     return 2.0 * b * b * K / best / 1e12, best, sample, threads
+
+
+def oracle_full_runs(L: int, phi: float) -> dict:
+    """Whole-matrix oracle runs at small sizes (the scheme-II pipeline at 256^3 and 1024^3, the exact fl(AB) at
+    256^3), each timed once: effective FP64 GFLOP/s, seconds, threads."""
+    from oracle import exact, ozaki2
+    from paper_2608_06812_b200 import inputs
+    out = {}
+    for name, n, fn in (("ozaki2_256", 256, lambda a, b: ozaki2.dgemm(a, b, L)), ("ozaki2_1024", 1024, lambda a, b: ozaki2.dgemm(a, b, L)),
+                        ("exact_fl_matmul_256", 256, exact.fl_matmul)):
+        a, b = inputs.lognormal_matrix(n, n, phi, seed=0), inputs.lognormal_matrix(n, n, phi, seed=1)
+        t0, c0 = time.perf_counter(), time.process_time()
+        fn(a, b)
+        wall, cpu = time.perf_counter() - t0, time.process_time() - c0
+        out[name] = {"gflops": 2.0 * n ** 3 / wall / 1e9, "seconds": wall, "cores": threads_used(cpu, wall)}
+    return out
 
 
 def run_reference(args, rank: int, world: int) -> None:
@@ -170,7 +216,7 @@ def run_reference(args, rank: int, world: int) -> None:
             "warmup": args.warmup, "ms_per_step": 1e3 * t, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "int64/f64 (CPU oracle)", "data": "synthetic",
             "config": {"workload": workload_name(n, L, args.phi), "sample": sample},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample, "host_cpus": os.cpu_count()},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
@@ -303,8 +349,10 @@ def run_ozk(args, rank: int, local_rank: int, world: int) -> None:
     barrier()
     # per-stage CUDA events the library recorded on this stream inside the timed steps (a ring of the
     # last 64 calls), read after the region so that no step waits for the host
+    gemm_cycles = (0, 0, 0)
     if not oz1:
         stage_acc = np.array(ozk.ozk_stage_timing_read()) * args.steps
+        gemm_cycles = ozk.ozk_stage_gemm_cycles()      # the last timed step's limb GEMM (first CTA pair's issuing thread)
     total_ms = ev[0].elapsed_time(ev[args.steps])
     clocks = sampler.stop() if rank == 0 else None
     ozk.check(ozk.ozk_get_async_status(stream), "ozk_get_async_status")
@@ -368,13 +416,29 @@ def run_ozk(args, rank: int, local_rank: int, world: int) -> None:
     fp4_flops_exec = 2.0 * executed * M * N * K
     fp4_flops_req = 2.0 * (4 * L - 1) * M * N * K        # the 13^2 term of modulus 169 is not required
     achieved = fp4_flops_exec / (gemm_ms * 1e-3) / 1e12
-    peak = peaks["bf16_sustained"] * FP4_PER_BF16
-    roofline = {"bound": "tensor", "kernel": "residue_gemm_pair_kernel" if pair else "limb_gemm_kernel", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                "frac": achieved / peak, "traffic": DRAM_TRAFFIC_BYTES.get((n, L)),
-                "peak_source": f"{peaks['source']} bf16 sustained {peaks['bf16_sustained']:.1f} TFLOP/s x {FP4_PER_BF16:g} (nominal FP4:BF16)",
+    proxy_sustained = peaks["bf16_sustained"] * FP4_PER_BF16
+    traffic, traffic_note = recorded_traffic(M, N, K, L)
+    # per-cycle view: executed multiply-adds per SM and clock at the SM clock sampled during the timed region, against
+    # the nominal 9000 TFLOP/s at the maximum clock; and the share of its clocks the issuing thread of the first CTA
+    # pair spent issuing rather than waiting (counters of the last launch, read after the region)
+    per_cycle = None
+    if clocks and clocks.get("sm_mhz") and pair:
+        mac_per_clk_sm = fp4_flops_exec / 2.0 / k_ranges / (SM_COUNT * gemm_ms / k_ranges * 1e-3 * clocks["sm_mhz"] * 1e6)
+        nominal_mac = NOMINAL_FP4_TFLOPS * 1e12 / 2.0 / (SM_COUNT * clocks["sm_max_mhz"] * 1e6)
+        clk_total, clk_tmem, clk_operands = gemm_cycles
+        per_cycle = {"mac_per_clk_per_sm": mac_per_clk_sm, "nominal_mac_per_clk_per_sm": nominal_mac, "frac": mac_per_clk_sm / nominal_mac,
+                     "sm_mhz": clocks["sm_mhz"], "gemm_ms_x_sm_mhz": gemm_ms * clocks["sm_mhz"],
+                     "issue_thread": {"clocks": clk_total, "waiting_for_tensor_memory": clk_tmem, "waiting_for_operands": clk_operands,
+                                      "issuing_frac": (1.0 - (clk_tmem + clk_operands) / clk_total) if clk_total > 0 else None}}
+    roofline = {"bound": "tensor", "kernel": "residue_gemm_pair_kernel" if pair else "limb_gemm_kernel", "achieved": achieved,
+                "peak": NOMINAL_FP4_TFLOPS, "unit": "TFLOP/s", "frac": achieved / NOMINAL_FP4_TFLOPS, "traffic": traffic,
+                "traffic_source": traffic_note,
+                "peak_source": "nominal dense FP4 of B200 (no FP4 peak is measured on this pool; the measured BF16 proxies follow)",
                 "achieved_required_count": fp4_flops_req / (gemm_ms * 1e-3) / 1e12,
-                "frac_of_burst_peak": achieved / (peaks["bf16_burst"] * FP4_PER_BF16),
-                "frac_of_nominal_9000": achieved / 9000.0, "ms_per_launch": gemm_ms / k_ranges, "launches_per_step": k_ranges}
+                "frac_of_4x_measured_bf16_sustained": achieved / proxy_sustained,
+                "frac_of_4x_measured_bf16_burst": achieved / (peaks["bf16_burst"] * FP4_PER_BF16),
+                "measured_bf16": {"source": peaks["source"], "sustained_tflops": peaks["bf16_sustained"], "burst_tflops": peaks["bf16_burst"]},
+                "ms_per_launch": gemm_ms / k_ranges, "launches_per_step": k_ranges, "per_cycle": per_cycle}
     pre_bytes = (16 + L) * (M * K + K * N)               # scan read + convert read + one byte (two nibbles) per modulus
     crt_bytes = (L + 8) * M * N
     stages = {"preprocess_ms": float(stage_acc[0]), "limb_gemm_ms": gemm_ms, "crt_ms": float(stage_acc[2]),
@@ -401,15 +465,46 @@ def run_ozk(args, rank: int, local_rank: int, world: int) -> None:
             line["native_fp64_tflops_context"] = f"unavailable: {type(exc).__name__}"
     if not args.no_cpu_baseline and world == 1:            # the oracle leg runs on rank 0 of a single-GPU run only
         tf, secs, sample, threads = oracle_sample_tflops(A, B, L, 512)
-        line["cpu_baseline"] = {"value": tf, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample, "seconds": secs}
+        line["cpu_baseline"] = {"value": tf, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample, "seconds": secs,
+                                "host_cpus": os.cpu_count(), "full_runs": oracle_full_runs(L, args.phi)}
     print(json.dumps(line), flush=True)
+
+
+def launcher_selftest(rank: int, world: int) -> None:
+    """CPU check of the multi-rank plumbing (gloo, no GPU, no kernels): every rank contributes a made-up step
+    time and flop count, rank 0 prints the reduced line."""
+    import torch.distributed as dist
+    if world > 1:
+        dist.init_process_group("gloo")
+    ms, flops = reduce_over_ranks(10.0 + rank, 1e12, dist if world > 1 else None, None)
+    if rank == 0:
+        print(json.dumps({"selftest": "launcher", "n_gpus": world, "ms_per_step": ms, "value": flops / (ms * 1e-3) / 1e12}), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def spawn_ranks(n: int) -> int:
+    """`python bench.py --gpus N` without a launcher: start N ranks of this script on this node with torch's
+    launcher (one process per GPU, rendezvous on 127.0.0.1) and pass their output through."""
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
 
 
 def main():
     args = parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl != "reference":
+        sys.exit(spawn_ranks(args.gpus))
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.launcher_selftest:
+        launcher_selftest(rank, world)
+        return
     if args.impl == "reference":
         run_reference(args, rank, world)
         return

@@ -100,10 +100,16 @@ ozk_status ozk_get_async_status(void* stream);
  *   A: M x K, lda >= max(1,M).  B: K x N, ldb >= max(1,K).  C: M x N, ldc >= max(1,M), overwritten.
  *   num_moduli in [OZK_MIN_MODULI, OZK_MAX_MODULI]; 19 keeps all 53 bits for K <= 76549.
  *   One limb-GEMM launch covers at most 131072 values of k (FP32 accumulators stay exact
- *   integers: 128*K <= 2^24 with limbs |c| <= 8, Lemma 3 tightened); a longer K is cut into
- *   such ranges whose residues are added modulo each modulus (Section 5.1, "Exactness of the
- *   FP32 accumulation": chunking), up to OZK_MAX_K.  The capacity of ozk_capacity_bits(K, ...)
- *   always refers to the whole K.  M, N, K = 0 are allowed (K = 0 gives C = 0).
+ *   integers: 128*K <= 2^24 with limbs |c| <= 8; Lemma 3 bounds K by 58254 for limbs up to 12).
+ *   EXTENSION, not in the paper (which never splits K): a longer K is cut into such ranges, one
+ *   limb-GEMM launch each, and the residues of the ranges are added modulo each modulus (the
+ *   residue of a sum is the sum of the residues), up to OZK_MAX_K.  The capacity of
+ *   ozk_capacity_bits(K, ...) always refers to the whole K.  M, N, K = 0 are allowed (K = 0
+ *   gives C = 0).  M and N are otherwise limited only by the workspace.
+ *   The library keeps per-device launch state keyed by the device ordinal, so one process may
+ *   use several devices (each call acts on the current device, to which `stream` and all
+ *   pointers must belong); the registered workspace and the stage timing are one per process,
+ *   and calls from several host threads must be serialised by the caller.
  * Returns OZK_OK once the work is enqueued.  The call only enqueues kernels and memsets on
  * `stream` (no allocation, no synchronisation), so after one eager call, which sets the
  * kernels' attributes, it may be captured into a CUDA graph and replayed. */
@@ -213,8 +219,12 @@ ozk_status ozk_stage_crt(int64_t M, int64_t N, int64_t K, int num_moduli,
  * It computes what stage 1 computes first, the row shifts s_i = c - 1 - e_i of A
  * (c = ozk_capacity_bits(K, num_moduli), Section 4.2), and keeps its only scratch, one 64-bit
  * maximum per row, in a fixed array inside the library image: OZK_NOALLOC_MAX_ROWS rows,
- * 512 KiB, resident on every GPU that loads the library until the process exits.  Neither this
- * call nor anything it calls allocates or frees memory.
+ * 512 KiB, resident on every GPU that loads the library until the process exits.  This call and
+ * everything it calls neither allocate nor free memory; the array itself is set up by the CUDA
+ * driver when it loads the library's device code, which with lazy loading can be as late as the
+ * first call on a device: make that call at start-up (a process with no free device memory gets
+ * OZK_ERR_CUDA from it), as advised for stream capture below.  `stream` must belong to the
+ * current device.
  *   A: M x K column-major FP64 (device), lda >= M.  s_out: M int32 (device).  An all-zero row
  *   gets 0; a row containing NaN or Inf gets INT32_MIN (there is no status word to report it).
  *   M > OZK_NOALLOC_MAX_ROWS, or K beyond the limits of ozk_dgemm -> OZK_ERR_UNSUPPORTED.
@@ -235,6 +245,13 @@ ozk_status ozk_row_shifts_noalloc(int64_t M, int64_t K, const double* A, int64_t
  * timed loop need not synchronise between its calls.  No call since then -> OZK_ERR_INVALID_ARG. */
 ozk_status ozk_stage_timing_enable(int enable);
 ozk_status ozk_stage_timing_read(float* ms3);
+
+/* Measurement aid: while stage timing is enabled, the thread that issues the tensor-core
+ * instructions of the limb GEMM's first CTA pair counts its clocks (clock64): clk3[0] the whole
+ * kernel, clk3[1] waiting for tensor memory to be drained by the epilogue, clk3[2] waiting for
+ * operand stages from the TMA producer; the rest it spent issuing.  Reads the counters the most
+ * recent limb-GEMM launch left in the workspace (synchronise its stream first); host pointer. */
+ozk_status ozk_stage_gemm_cycles(long long* clk3);
 
 /* One tcgen05.mma.kind::mxf4.block_scale instruction sequence on caller-supplied packed
  * E2M1 operands, used to pin the hardware byte formats (nibble order, E2M1 codes, UE8M0

@@ -54,6 +54,7 @@ SIGNATURES = {
     "ozk_stage_wait_probe": (c_int, [c_void_p]),
     "ozk_row_shifts_noalloc": (c_int, [c_int64, c_int64, c_void_p, c_int64, c_int, c_void_p, c_void_p]),
     "ozk_stage_timing_enable": (c_int, [c_int]),
+    "ozk_stage_gemm_cycles": (c_int, [c_void_p]),
     "ozk_stage_timing_read": (c_int, [c_void_p]),
     "ozk_stage_mma_probe": (c_int, [c_void_p, c_void_p, c_int64, c_int, c_void_p, c_void_p]),
 }
@@ -175,6 +176,13 @@ def ozk_stage_timing_read() -> tuple[float, float, float]:
     ms = (ctypes.c_float * 3)()
     check(lib().ozk_stage_timing_read(ms), "ozk_stage_timing_read")
     return float(ms[0]), float(ms[1]), float(ms[2])
+
+
+def ozk_stage_gemm_cycles() -> tuple[int, int, int]:
+    """Clocks of the limb GEMM's issuing thread: (whole kernel, waiting for tensor memory, waiting for operands)."""
+    clk = (ctypes.c_longlong * 3)()
+    check(lib().ozk_stage_gemm_cycles(clk), "ozk_stage_gemm_cycles")
+    return int(clk[0]), int(clk[1]), int(clk[2])
 
 
 def ozk_stage_wait_probe(stream=0) -> int:

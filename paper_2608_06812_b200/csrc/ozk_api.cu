@@ -82,7 +82,6 @@ ozk_status check_common(int64_t M, int64_t N, int64_t K, int L, Geometry* g, int
   if (!make_geometry(M, N, K, L, g, max_bits)) return OZK_ERR_INVALID_ARG;
   if (K > kMaxK) return OZK_ERR_UNSUPPORTED;
   if (g->c_bits < 1) return OZK_ERR_UNSUPPORTED;
-  if (N > 65535 || g->Mp / 32 > 65535) return OZK_ERR_UNSUPPORTED;  // grid-dimension limits of the O(N^2) kernels
   if (!g_ws.ptr) return OZK_ERR_WORKSPACE;
   if (g_ws.bytes < g->total) return OZK_ERR_WORKSPACE;
   return OZK_OK;
@@ -352,6 +351,17 @@ ozk_status ozk_stage_timing_read(float* ms3) {
   }
   for (int i = 0; i < 3; ++i) ms3[i] = (float)(sum[i] / n);
   g_timing.calls = 0;
+  return OZK_OK;
+}
+
+ozk_status ozk_stage_gemm_cycles(long long* clk3) {
+  if (!clk3) return OZK_ERR_INVALID_ARG;
+  if (!g_ws.ptr) return OZK_ERR_WORKSPACE;
+  StatusBlock sb;
+  if (cudaMemcpy(&sb, g_ws.ptr, sizeof sb, cudaMemcpyDeviceToHost) != cudaSuccess) return OZK_ERR_CUDA;
+  clk3[0] = sb.mma_clk_total;
+  clk3[1] = sb.mma_clk_wait_tmem;
+  clk3[2] = sb.mma_clk_wait_operands;
   return OZK_OK;
 }
 

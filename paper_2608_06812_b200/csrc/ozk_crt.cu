@@ -547,7 +547,8 @@ __global__ void copy_residues_kernel(const uint8_t* __restrict__ res, int64_t Mp
 }
 
 // acc = (acc + chunk) mod m for one modulus per blockIdx.y: sums the residues of two k ranges
-// (Section 5.1: the residue of a sum is the sum of the residues).  16 bytes per thread.
+// (an extension the paper does not have: it never splits K; the residue of a sum is the sum of the residues).
+// 16 bytes per thread.
 __global__ void add_residues_kernel(uint8_t* __restrict__ acc, const uint8_t* __restrict__ chunk, size_t per_modulus,
                                     ModulusTable mt) {
   const size_t v = (size_t)blockIdx.x * blockDim.x + threadIdx.x;

@@ -5,9 +5,13 @@
 // all device memory and forbids raw cudaMalloc (it synchronises the whole device), a plug-in
 // called from a latency-critical loop, or a process that has already handed every free byte to
 // another library.  For them this entry point keeps its scratch in a fixed array that is part of
-// the library image, so nothing is allocated or freed, by this code or by a library routine, at
-// any time.  The price is a size limit, a few hundred KiB held on every GPU that loads the
-// library, and no protection between calls that overlap on the GPU.
+// the library image, so this code and the routines it calls neither allocate nor free anything.
+// (The CUDA driver sets the array up when it loads the library's device code, which with lazy
+// loading may be as late as the first call on a device: callers make that call at start-up.)
+// The price is a size limit, a few hundred KiB held on every GPU that loads the library, and no
+// protection between calls that overlap on the GPU.  The device address is looked up once per
+// device ordinal with that device current; `stream` must belong to the current device, and the
+// cached address does not survive a cudaDeviceReset.
 #include <limits.h>
 
 #include <mutex>

@@ -55,3 +55,27 @@ def test_reference_arm_only_rank0_prints():
 
 def test_workload_name_mentions_the_config():
     assert "16384" in bench.workload_name(16384, 19, 1.0) and "19 moduli" in bench.workload_name(16384, 19, 1.0)
+
+
+def test_gpus_flag_starts_the_ranks_itself():
+    """`python bench.py --gpus 2` with no launcher around it must run two ranks (here on CPU, gloo, no kernels)."""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--launcher-selftest"], env=env,
+                         capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [json.loads(l) for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1 and lines[0]["n_gpus"] == 2
+    assert lines[0]["ms_per_step"] == 11.0 and abs(lines[0]["value"] - 2e12 / 11e-3 / 1e12) < 1e-9   # max of times, sum of work
+
+
+def test_recorded_traffic_needs_a_capture_of_the_current_source(tmp_path, monkeypatch):
+    rec = {"captures": [{"M": 64, "N": 64, "K": 64, "moduli": 19, "dram_read_bytes": 10, "dram_write_bytes": 5,
+                         "gemm_source_sha256": "not the current source", "command": "x"}]}
+    path = tmp_path / "t.json"
+    path.write_text(json.dumps(rec))
+    monkeypatch.setattr(bench, "TRAFFIC_FILE", str(path))
+    assert bench.recorded_traffic(64, 64, 64, 19)[0] is None
+    assert bench.recorded_traffic(128, 64, 64, 19)[0] is None
+    rec["captures"][0]["gemm_source_sha256"] = bench.gemm_source_hash()
+    path.write_text(json.dumps(rec))
+    assert bench.recorded_traffic(64, 64, 64, 19)[0] == 15.0

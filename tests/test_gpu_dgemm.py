@@ -57,14 +57,27 @@ def test_long_inner_products_bit_exact(shape, L):
 
 @pytest.mark.parametrize("shape", [(16, 64, 140000), (16, 130, 290000)])
 def test_k_beyond_one_limb_gemm_range_bit_exact(shape):
-    """K above 131072 runs one limb GEMM per range of 131072 and adds the residues modulo each modulus
-    (Section 5.1, chunking): a short last range (fast recombination) and three ranges with a long last one."""
+    """K above 131072 runs one limb GEMM per range of 131072 and adds the residues modulo each modulus (this build's
+    extension: Lemma 3 only bounds K, the paper never splits it): a short last range (fast recombination) and
+    three ranges with a long last one."""
     M, N, K = shape
     A = inputs.lognormal_matrix(M, K, 0.5, seed=30)
     B = inputs.lognormal_matrix(K, N, 0.5, seed=31)
     A[0, :] = np.abs(A[0, :])
     B[:, 0] = np.abs(B[:, 0])
     assert gu.bits_equal(gu.dgemm(A, B, 19), ozaki2.dgemm(A, B, 19).C)
+
+
+def test_more_than_65535_columns():
+    """N beyond the y-dimension limit of a CUDA grid: the O(N^2) kernels loop over the columns.  Small integers
+    make C the exact integer product, so the whole matrix is checked against an int64 product."""
+    M, N, K = 20, 66000, 24
+    A = inputs.small_integer_matrix(M, K, 1000, seed=5)
+    B = inputs.small_integer_matrix(K, N, 1000, seed=6)
+    C = gu.dgemm(A, B, 19)
+    assert gu.bits_equal(C, (A.astype(np.int64) @ B.astype(np.int64)).astype(np.float64))
+    j = np.array([0, 1, 65534, 65535, 65536, 65999])            # a few columns also against the oracle
+    assert gu.bits_equal(C[:, j], ozaki2.dgemm(A, B[:, j], 19).C)
 
 
 def test_k_ranges_small_integers_exact_over_several_tiles():

@@ -1,10 +1,11 @@
 """ozk_row_shifts_noalloc, the entry point for callers that cannot allocate device memory (its
 scratch is a fixed array inside the library): its output must equal the shifts the regular,
-workspace-based stage 1 produces, on two calls in a row that reuse the same scratch."""
+workspace-based stage 1 produces, and the oracle's, on two calls in a row that reuse the same scratch."""
 import numpy as np
 import pytest
 import torch
 
+from oracle import moduli, ozaki2
 from paper_2608_06812_b200 import binding as ozk
 from paper_2608_06812_b200 import inputs
 from tests import gpu_util as gu
@@ -47,9 +48,30 @@ def test_two_calls_in_a_row_match_the_workspace_path():
     got2 = shifts_by_noalloc_path(A2, L)
     assert np.array_equal(got1, shifts_by_workspace_path(A1, B1, L))
     assert np.array_equal(got2, shifts_by_workspace_path(A2, B2, L))
+    assert np.array_equal(got1, ozaki2.shared_shifts(A1, 1, moduli.capacity_bits(333, L)))
+    assert np.array_equal(got2, ozaki2.shared_shifts(A2, 1, moduli.capacity_bits(200, L)))
     assert got2[5] == 0
     # and a third call on the first input again gives the first answer again
     assert np.array_equal(shifts_by_noalloc_path(A1, L), got1)
+
+
+def test_subnormal_row_maximum_and_empty_inner_dimension():
+    L = 19
+    A = inputs.lognormal_matrix(40, 12, 0.5, seed=7)
+    A[3, :] = [k * 2.0 ** -1074 for k in range(12)]          # the row maximum is subnormal
+    A[4, :] = 0.0
+    A[4, 2] = -(2.0 ** -1074)                                  # the smallest magnitude there is
+    B = inputs.lognormal_matrix(12, 8, 0.5, seed=8)
+    got = shifts_by_noalloc_path(A, L)
+    assert np.array_equal(got, shifts_by_workspace_path(A, B, L))
+    assert np.array_equal(got, ozaki2.shared_shifts(A, 1, moduli.capacity_bits(12, L)))
+    # K = 0: every row is empty, every shift 0, and nothing is read from A
+    ds = torch.full((9,), 777, dtype=torch.int32, device="cuda")
+    ozk.check(ozk.ozk_row_shifts_noalloc(9, 0, None, 9, L, ds.data_ptr(), gu.stream()), "ozk_row_shifts_noalloc")
+    torch.cuda.synchronize()
+    assert np.array_equal(ds.cpu().numpy(), np.zeros(9, dtype=np.int32))
+    # the same array serves the next call
+    assert np.array_equal(shifts_by_noalloc_path(A, L), got)
 
 
 def test_limits_and_flags():
