@@ -1,7 +1,9 @@
 """Parity at the full configured sizes, in the launch configuration bench.py times (ozk_dgemm on
 column-major device buffers): a 128x128 output block (the paper's own evaluation protocol) plus
 scattered rows and columns against the CPU oracle bit for bit, the error against exact fl(AB) on
-a sub-block, and (4096, 8192) every reconstructed integer by a Freivalds check modulo two primes."""
+a sub-block, every reconstructed integer by a Freivalds check modulo two primes (4096 and 8192 on
+the host, 16384 with the reconstructed integers left on the device), and C against the oracle's
+rounding of its own reconstructed integer on a million elements."""
 import numpy as np
 import pytest
 import torch
@@ -88,6 +90,40 @@ def x_words_by_stages(n, L, dA, dB):
     return dX.cpu().numpy(), dC2
 
 
+def freivalds_on_device(n, L, A, B, dX):
+    """The same identity with the 192-bit words left on the device (dX[j, i, 6], int32): x v = At (Bt v) modulo two
+    31-bit primes.  At, Bt come from the CPU oracle; torch int64 arithmetic on the GPU is test infrastructure."""
+    c = moduli.capacity_bits(n, L)
+    dAt = torch.from_numpy(ozaki2.to_integers(A, ozaki2.shared_shifts(A, 1, c), 1)).cuda()     # [i, k]
+    dBt = torch.from_numpy(ozaki2.to_integers(B, ozaki2.shared_shifts(B, 0, c), 0)).cuda()     # [k, j]
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(99)
+    step = 512
+    for q in (2147483647, 2147483629):
+        v = torch.randint(0, q, (n,), dtype=torch.int64, device="cuda", generator=gen)
+        Bv = torch.zeros(n, dtype=torch.int64, device="cuda")
+        for j0 in range(0, n, step):                          # every product is reduced (< 2^31) before the sum
+            Bv = (Bv + ((dBt[:, j0:j0 + step] % q) * v[None, j0:j0 + step] % q).sum(dim=1)) % q
+        right = torch.zeros(n, dtype=torch.int64, device="cuda")
+        for k0 in range(0, n, step):
+            right = (right + ((dAt[:, k0:k0 + step] % q) * Bv[None, k0:k0 + step] % q).sum(dim=1)) % q
+        pw = [pow(2, 32 * k, q) for k in range(6)]
+        left = torch.zeros(n, dtype=torch.int64, device="cuda")
+        for j0 in range(0, n, step):
+            W = dX[j0:j0 + step].to(torch.int64) & 0xFFFFFFFF                                   # [j, i, 6]
+            xm = torch.zeros(W.shape[:2], dtype=torch.int64, device="cuda")
+            for k in range(6):
+                xm = (xm + (W[:, :, k] % q) * pw[k]) % q
+            xm = (xm - (W[:, :, 5] >> 31) * pow(2, 192, q)) % q                                 # two's complement sign
+            left = (left + (xm * v[j0:j0 + step, None] % q).sum(dim=0)) % q
+        assert torch.equal(left, right)
+
+
+def words_to_int(w) -> int:
+    v = sum((int(x) & 0xFFFFFFFF) << (32 * k) for k, x in enumerate(w))
+    return v - (1 << 192) if v >> 191 else v
+
+
 def test_config2_4096_moduli_sweep():
     """M=N=K=4096, phi=0.5, moduli count 12..20: bit-exact samples for every count; the error bound
     1e-15 against fl(AB) from 17 moduli on; Freivalds over the whole matrix at 19 moduli."""
@@ -103,6 +139,17 @@ def test_config2_4096_moduli_sweep():
             X, dC2 = x_words_by_stages(n, L, dA, dB)
             assert torch.equal(dC2.view(torch.int64), dC.view(torch.int64))
             freivalds(n, L, A, B, X)
+            # C is the oracle's single rounding of the reconstructed integer, scaled by the oracle's shifts:
+            # a million random elements plus the first column
+            c = moduli.capacity_bits(n, L)
+            s_ref, t_ref = ozaki2.shared_shifts(A, 1, c), ozaki2.shared_shifts(B, 0, c)
+            C = dC.cpu().numpy()                              # [j, i]
+            rng = np.random.default_rng(7)
+            ii = np.concatenate([rng.integers(0, n, 1_000_000), np.arange(n)])
+            jj = np.concatenate([rng.integers(0, n, 1_000_000), np.zeros(n, dtype=np.int64)])
+            want = np.array([ozaki2.round_scaled_to_double(words_to_int(X[j, i]), int(s_ref[i]) + int(t_ref[j]))
+                             for i, j in zip(ii, jj)])
+            assert gu.bits_equal(C[jj, ii], want)
     assert all(errs[L] <= 1e-15 for L in range(17, 21)), errs
     assert errs[12] > errs[15] > errs[18]                     # fewer moduli keep fewer bits
 
@@ -135,3 +182,25 @@ def test_config5_16384_headline_configuration():
     err = exact.normwise_error(got[:16, :16], A[rows[:16]], B[:, cols[:16]], against_rounded=True)
     assert err <= 1e-15
     assert torch.isfinite(dC).all()
+    # every element: the reconstructed integers of the staged run (left on the device) satisfy the Freivalds
+    # identity against the oracle's converted integers, and the staged run's C equals ozk_dgemm's bit for bit
+    gu.ensure_workspace(ozk.ozk_dgemm_workspace_bytes(n, n, n, 19))
+    dX = torch.empty((n, n, 6), dtype=torch.int32, device="cuda")
+    dC2 = torch.empty((n, n), dtype=torch.float64, device="cuda")
+    ozk.check(ozk.ozk_stage_preprocess(n, n, n, dA.data_ptr(), n, dB.data_ptr(), n, 19, None, None, None, None, gu.stream()),
+              "ozk_stage_preprocess")
+    ozk.check(ozk.ozk_stage_residue_gemm(n, n, n, 19, None, gu.stream()), "ozk_stage_residue_gemm")
+    ozk.check(ozk.ozk_stage_crt(n, n, n, 19, None, None, None, dC2.data_ptr(), n, dX.data_ptr(), gu.stream()), "ozk_stage_crt")
+    ozk.check(ozk.ozk_get_async_status(gu.stream()), "status")
+    assert torch.equal(dC2.view(torch.int64), dC.view(torch.int64))
+    del dC2
+    freivalds_on_device(n, 19, A, B, dX)
+    # and C against the oracle's rounding of x on scattered elements
+    c = moduli.capacity_bits(n, 19)
+    s_ref, t_ref = ozaki2.shared_shifts(A, 1, c), ozaki2.shared_shifts(B, 0, c)
+    rng = np.random.default_rng(11)
+    ii, jj = rng.integers(0, n, 20000), rng.integers(0, n, 20000)
+    Xs = dX[torch.from_numpy(jj).cuda(), torch.from_numpy(ii).cuda()].cpu().numpy()
+    Cs = dC[torch.from_numpy(jj).cuda(), torch.from_numpy(ii).cuda()].cpu().numpy()
+    want = np.array([ozaki2.round_scaled_to_double(words_to_int(Xs[k]), int(s_ref[ii[k]]) + int(t_ref[jj[k]])) for k in range(ii.size)])
+    assert gu.bits_equal(Cs, want)

@@ -296,3 +296,21 @@ def test_scheme1_equals_integer_product_and_scheme2_bit_for_bit():
     assert all(int(X1[idx]) == int(ref[idx]) for idx in np.ndindex(*X1.shape))
     C2 = ozaki2.dgemm(A, B, 19).C
     assert np.array_equal(C1.view(np.uint64), C2.view(np.uint64))
+
+
+def test_limb_products_through_float64_are_exact_at_the_headline_k():
+    """The oracle forms the four limb products with float64 matrix products (magnitudes 288 K << 2^53, so exact).
+    At K = 16384, with adversarial limbs of one sign as well as random ones, they equal Python big-integer sums."""
+    K = 16384
+    rng = np.random.default_rng(5)
+    for m in (169, 115, 53):
+        for kind in ("random", "extreme"):
+            if kind == "random":
+                At = rng.integers(-2 ** 52, 2 ** 52, size=(3, K), dtype=np.int64)
+                Bt = rng.integers(-2 ** 52, 2 ** 52, size=(K, 2), dtype=np.int64)
+            else:                                                  # every residue the same: limb sums of one sign
+                At = np.full((3, K), 2 ** 52 - 1, dtype=np.int64)
+                Bt = np.full((K, 2), 2 ** 52 - 3, dtype=np.int64)
+            got = ozaki2.residue_product(At, Bt, m)
+            want = np.array([[sum(int(At[i, k]) * int(Bt[k, j]) for k in range(K)) % m for j in range(2)] for i in range(3)])
+            assert np.array_equal(np.asarray(got, dtype=np.int64), want), (m, kind)
