@@ -60,6 +60,8 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-fp64-context", action="store_true")
+    ap.add_argument("--karatsuba", action="store_true", help="switch the partial Karatsuba variant on (68 instead of 75 limb products "
+                    "at 19 moduli; a measured loss, not the default)")
     ap.add_argument("--launcher-selftest", action="store_true", help="CPU-only check of the multi-rank launch and reduction (no GPU work)")
     return ap.parse_args()
 
@@ -310,6 +312,8 @@ def run_ozk(args, rank: int, local_rank: int, world: int) -> None:
     dA, dB = hA.to(dev), hB.to(dev)
     dC = torch.empty((N, M), dtype=torch.float64, device=dev)
     oz1 = args.scheme == "oz1"
+    if args.karatsuba:
+        ozk.check(ozk.ozk_stage_set_karatsuba(True), "ozk_stage_set_karatsuba")
     ws_bytes = ozk.ozk_dgemm_oz1_workspace_bytes(M, N, K) if oz1 else ozk.ozk_dgemm_workspace_bytes(M, N, K, L)
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
     ozk.check(ozk.ozk_set_workspace(ws.data_ptr(), ws.numel()), "ozk_set_workspace")
@@ -413,6 +417,8 @@ def run_ozk(args, rank: int, local_rank: int, world: int) -> None:
     # both limb-GEMM kernels skip the 13^2 term of modulus 169: executed = required = 4L - 1 products
     pair = ((N + 127) // 128 * 128) % 256 == 0 and os.environ.get("OZK_GEMM_PAIR", "1") != "0"
     executed = 4 * L - 1 if ozk.ozk_get_moduli(L)[0] == 169 else 4 * L
+    if args.karatsuba and pair:
+        executed -= sum(1 for l in range(L) if l == 11 or l >= 13)      # three products for the Karatsuba moduli
     fp4_flops_exec = 2.0 * executed * M * N * K
     fp4_flops_req = 2.0 * (4 * L - 1) * M * N * K        # the 13^2 term of modulus 169 is not required
     achieved = fp4_flops_exec / (gemm_ms * 1e-3) / 1e12
@@ -449,7 +455,7 @@ def run_ozk(args, rank: int, local_rank: int, world: int) -> None:
             "vs_baseline": (value / world / PAPER_TOTAL_TFLOPS[n]) if (n in PAPER_TOTAL_TFLOPS and L == 19 and args.max_bits == 53) else None,
             "dtype": "fp4_e2m1 (fp32 accumulate, integer CRT)", "data": "synthetic",
             "config": {"workload": workload_name(n, L, args.phi, shape), "l2": "inputs (%.2f + %.2f GiB) %s" % (M * K * 8 / 2 ** 30, K * N * 8 / 2 ** 30, "larger than L2" if (M * K + K * N) * 8 > (126 << 20) else "fit L2: not a valid timing size"),
-                       "parallelism": "replicas" if world > 1 else "single GPU", "moduli": L,
+                       "parallelism": "replicas" if world > 1 else "single GPU", "moduli": L, "karatsuba": bool(args.karatsuba),
                        "integer_bits": ozk.ozk_capacity_bits_ext(K, L, args.max_bits)},
             "clocks": clocks, "e2e": e2e, "gpu_launches": (KERNELS_PER_STEP + 2 * (k_ranges - 1)) * args.steps, "roofline": roofline, "stages": stages}
 

@@ -193,7 +193,8 @@ ozk_status ozk_stage_preprocess(int64_t M, int64_t N, int64_t K,
 
 /* Decodes limb plane (modulus index l, limb 0|1) of operand 'A' or 'B' from the workspace
  * into doubled-E2M1 integers (int8, values in S): out[r + k*rows], r < rows (M for 'A',
- * N for 'B'), k < K.  Valid after ozk_stage_preprocess / ozk_dgemm on the same sizes. */
+ * N for 'B'), k < K.  Valid after ozk_stage_preprocess / ozk_dgemm on the same sizes.
+ * limb = 2 reads the sum-limb plane of a Karatsuba modulus (variant on, see ozk_stage_set_karatsuba). */
 ozk_status ozk_stage_read_planes(char operand, int64_t M, int64_t N, int64_t K, int num_moduli,
                                  int l, int limb, int8_t* out, void* stream);
 
@@ -245,6 +246,16 @@ ozk_status ozk_row_shifts_noalloc(int64_t M, int64_t K, const double* A, int64_t
  * timed loop need not synchronise between its calls.  No call since then -> OZK_ERR_INVALID_ARG. */
 ozk_status ozk_stage_timing_enable(int enable);
 ozk_status ozk_stage_timing_read(float* ms3);
+
+/* Variant switch (process-wide, off by default): partial Karatsuba for the moduli whose residue classes all
+ * have a limb pair (c0, c1) with c0 + c1 again a doubled E2M1 value: 83, 73, 71, 67, 61, 59, 53 among the
+ * first 19 (Section 5.1, last paragraph; Section 6.4).  When on, the encoder writes a third plane of sum limbs
+ * for those moduli and the CTA-pair limb GEMM forms a0 b0, a1 b1 and (a0 + a1)(b0 + b1) instead of the four
+ * products (68 instead of 75 products at 19 moduli); the residues, hence C, are the same bit for bit.  Sum
+ * limbs reach 12, so a limb-GEMM launch covers at most 65536 values of k (144 K <= 2^24, Lemma 3).  The
+ * workspace grows by the sum-limb planes: query ozk_dgemm_workspace_bytes after switching.  The paper found
+ * the variant slower under kernel fusion; so does this build (measurements in profiles/). */
+ozk_status ozk_stage_set_karatsuba(int enable);
 
 /* Measurement aid: while stage timing is enabled, the thread that issues the tensor-core
  * instructions of the limb GEMM's first CTA pair counts its clocks (clock64): clk3[0] the whole

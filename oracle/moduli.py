@@ -69,6 +69,34 @@ def limb_pair_table(m: int) -> list[tuple[int, int]]:
     return table
 
 
+def limb_pair_table_karatsuba(m: int):
+    """Section 5.1, last paragraph: a limb pair per residue class whose sum c0 + c1 is itself a doubled E2M1
+    value, so that Karatsuba's third product (a0 + a1)(b0 + b1) can be formed from one more limb plane.  Returns
+    None when some class of m has no such pair.  Among the valid pairs: smallest max(|c0|, |c1|), then |c0 + c1|,
+    then (c1, c0)."""
+    table = []
+    for rho in range(m):
+        best = None
+        for v, pairs in TWO_LIMB_PAIRS.items():
+            if (v - rho) % m:
+                continue
+            for (c0, c1) in pairs:
+                if c0 + c1 not in S:
+                    continue
+                key = (max(abs(c0), abs(c1)), abs(c0 + c1), c1, c0)
+                if best is None or key < best[0]:
+                    best = (key, (c0, c1))
+        if best is None:
+            return None
+        table.append(best[1])
+    return table
+
+
+def karatsuba_moduli(moduli) -> list[int]:
+    """The moduli of the list that admit the Karatsuba form (the paper names 83, 73, 71, 67, 61, 59, 53 among its 19)."""
+    return [m for m in moduli if limb_pair_table_karatsuba(m) is not None]
+
+
 def product(moduli) -> int:
     P = 1
     for m in moduli:

@@ -16,8 +16,8 @@ from dataclasses import dataclass, field
 
 import numpy as np
 
-from .base13 import BASE
-from .moduli import capacity_bits, crt_weights, limb_pair_table, select_moduli
+from .base13 import BASE, S
+from .moduli import capacity_bits, crt_weights, limb_pair_table, limb_pair_table_karatsuba, select_moduli
 
 
 # ----------------------------------------------------------------------------
@@ -99,6 +99,26 @@ def residue_product(At: np.ndarray, Bt: np.ndarray, m: int) -> np.ndarray:
     D1 = np.rint(a0 @ b1 + a1 @ b0).astype(np.int64)
     D2 = np.rint(a1 @ b1).astype(np.int64)
     return np.mod(D0 + BASE * D1 + BASE * BASE * D2, m).astype(np.int64)
+
+
+def residue_product_karatsuba(At: np.ndarray, Bt: np.ndarray, m: int) -> np.ndarray:
+    """The same residue from three limb products (Section 5.1, last paragraph): with limb pairs whose sums
+    a_s = a0 + a1, b_s = b0 + b1 are doubled E2M1 values again,
+        a0 b1 + a1 b0 = a_s b_s - a0 b0 - a1 b1,
+    so r = (D0 + 13 (Ds - D0 - D2) + 169 D2) mod m with D0 = a0 b0, D2 = a1 b1, Ds = a_s b_s summed over k.
+    Only for the moduli moduli.karatsuba_moduli admits."""
+    table = limb_pair_table_karatsuba(m)
+    if table is None:
+        raise ValueError(f"modulus {m} has residue classes without a Karatsuba limb pair")
+    table = np.array(table, dtype=np.int64)
+    ra, rb = np.mod(At, m), np.mod(Bt, m)
+    a0, a1, b0, b1 = table[ra, 0], table[ra, 1], table[rb, 0], table[rb, 1]
+    a_s, b_s = a0 + a1, b0 + b1
+    assert np.isin(a_s, S).all() and np.isin(b_s, S).all()
+    D0 = a0 @ b0                                            # int64 matrix products: |sum| <= 144 K
+    D2 = a1 @ b1
+    Ds = a_s @ b_s
+    return np.mod(D0 + BASE * (Ds - D0 - D2) + BASE * BASE * D2, m).astype(np.int64)
 
 
 # ----------------------------------------------------------------------------

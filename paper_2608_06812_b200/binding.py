@@ -55,6 +55,7 @@ SIGNATURES = {
     "ozk_row_shifts_noalloc": (c_int, [c_int64, c_int64, c_void_p, c_int64, c_int, c_void_p, c_void_p]),
     "ozk_stage_timing_enable": (c_int, [c_int]),
     "ozk_stage_gemm_cycles": (c_int, [c_void_p]),
+    "ozk_stage_set_karatsuba": (c_int, [c_int]),
     "ozk_stage_timing_read": (c_int, [c_void_p]),
     "ozk_stage_mma_probe": (c_int, [c_void_p, c_void_p, c_int64, c_int, c_void_p, c_void_p]),
 }
@@ -176,6 +177,10 @@ def ozk_stage_timing_read() -> tuple[float, float, float]:
     ms = (ctypes.c_float * 3)()
     check(lib().ozk_stage_timing_read(ms), "ozk_stage_timing_read")
     return float(ms[0]), float(ms[1]), float(ms[2])
+
+
+def ozk_stage_set_karatsuba(enable: bool) -> int:
+    return lib().ozk_stage_set_karatsuba(1 if enable else 0)
 
 
 def ozk_stage_gemm_cycles() -> tuple[int, int, int]:

@@ -28,6 +28,7 @@ struct StageTiming {
   cudaEvent_t ev[kTimingRing][4];
 };
 StageTiming g_timing;
+bool g_karatsuba = false;
 
 void mark(int i, cudaStream_t st) {
   if (g_timing.enabled) cudaEventRecord(g_timing.ev[g_timing.calls % kTimingRing][i], st);
@@ -46,6 +47,7 @@ bool make_geometry_impl(int64_t M, int64_t N, int64_t K, int L, Geometry* g, int
   g->Np = round_up(N > 0 ? N : 1, kTileRows);
   g->Kp = round_up(K > 0 ? K : 1, kTileKNibbles);
   g->c_bits = host_capacity_bits(K, L, max_bits);
+  g->karatsuba = (g_karatsuba && karatsuba_count(L) > 0) ? 1 : 0;
   size_t off = 0;
   g->off_status = off;
   off += align_up(sizeof(StatusBlock), 1024);
@@ -64,13 +66,13 @@ bool make_geometry_impl(int64_t M, int64_t N, int64_t K, int L, Geometry* g, int
   g->plane_bytes_a = (size_t)g->Mp * g->pitch;
   g->plane_bytes_b = (size_t)g->Np * g->pitch;
   g->off_planes_a = off;
-  off += 2 * (size_t)L * g->plane_bytes_a;
+  off += (size_t)planes_per_operand(L, g->karatsuba) * g->plane_bytes_a;
   g->off_planes_b = off;
-  off += 2 * (size_t)L * g->plane_bytes_b;
+  off += (size_t)planes_per_operand(L, g->karatsuba) * g->plane_bytes_b;
   g->off_res = off;
   off += (size_t)L * (size_t)g->Mp * (size_t)g->Np;
   g->off_res_chunk = 0;
-  if (K > kChunkK) {  // k ranges beyond the first leave their residues here before they are added in
+  if (K > (g->karatsuba ? kChunkKKaratsuba : kChunkK)) {  // k ranges beyond the first leave their residues here before they are added in
     g->off_res_chunk = off;
     off += (size_t)L * (size_t)g->Mp * (size_t)g->Np;
   }
@@ -89,7 +91,7 @@ ozk_status check_common(int64_t M, int64_t N, int64_t K, int L, Geometry* g, int
 
 ozk_status run_preprocess(const Geometry& g, const ModulusTable& mt, const double* A, int64_t lda, const double* B,
                           int64_t ldb, int64_t* At_out, int64_t* Bt_out, cudaStream_t st) {
-  if (launch_build_lut(mt, g_ws.ptr + g.off_lut, st) != cudaSuccess) return OZK_ERR_CUDA;
+  if (launch_build_lut(mt, g_ws.ptr + g.off_lut, g.karatsuba, st) != cudaSuccess) return OZK_ERR_CUDA;
   if (launch_scan_and_shifts(g, A, lda, B, ldb, g_ws.ptr, st) != cudaSuccess) return OZK_ERR_CUDA;
   if (launch_encode(g, mt, A, lda, B, ldb, g_ws.ptr, At_out, Bt_out, st) != cudaSuccess) return OZK_ERR_CUDA;
   return OZK_OK;
@@ -135,16 +137,18 @@ bool device_is_sm100() {
 // Limb GEMM over all of K: one launch per k range of at most kChunkK (the FP32 accumulators stay exact
 // integers inside a range, Lemma 3 with |limb| <= 8); the residues of later ranges are added modulo m.
 ozk_status gemm_residues_chunked(const Geometry& g, const ModulusTable& mt, uint8_t* ws, cudaStream_t st) {
-  if (g.Kp <= kChunkK) return gemm_residues(g, mt, ws, st);
+  const int64_t chunk = g.karatsuba ? kChunkKKaratsuba : kChunkK;
+  if (g.Kp <= chunk) return gemm_residues(g, mt, ws, st);
   if (!g.off_res_chunk) return OZK_ERR_WORKSPACE;
-  for (int64_t k0 = 0; k0 < g.Kp; k0 += kChunkK) {
-    const int64_t klen = g.Kp - k0 < kChunkK ? g.Kp - k0 : kChunkK;
+  for (int64_t k0 = 0; k0 < g.Kp; k0 += chunk) {
+    const int64_t klen = g.Kp - k0 < chunk ? g.Kp - k0 : chunk;
     const ozk_status rc = gemm_residues(g, mt, ws, st, k0, klen, k0 == 0 ? nullptr : ws + g.off_res_chunk);
     if (rc != OZK_OK) return rc;
     if (k0 > 0 && launch_add_residues(g, mt, ws + g.off_res, ws + g.off_res_chunk, st) != cudaSuccess) return OZK_ERR_CUDA;
   }
   return OZK_OK;
 }
+bool karatsuba_enabled() { return g_karatsuba; }
 bool stage_timing_enabled() { return g_timing.enabled; }
 uint8_t* workspace_ptr() { return g_ws.ptr; }
 size_t workspace_bytes() { return g_ws.bytes; }
@@ -246,10 +250,11 @@ ozk_status ozk_stage_read_planes(char operand, int64_t M, int64_t N, int64_t K, 
   Geometry g;
   ozk_status rc = check_common(M, N, K, num_moduli, &g);
   if (rc != OZK_OK) return rc;
-  if (!out || l < 0 || l >= num_moduli || (limb != 0 && limb != 1) || (operand != 'A' && operand != 'B'))
-    return OZK_ERR_INVALID_ARG;
+  if (!out || l < 0 || l >= num_moduli || limb < 0 || limb > 2 || (operand != 'A' && operand != 'B')) return OZK_ERR_INVALID_ARG;
+  if (limb == 2 && !(g.karatsuba && karatsuba_modulus(l))) return OZK_ERR_INVALID_ARG;  // sum-limb planes exist in the Karatsuba variant only
   const bool a = operand == 'A';
-  const uint8_t* plane = g_ws.ptr + (a ? g.off_planes_a : g.off_planes_b) + (size_t)(2 * l + limb) * (a ? g.plane_bytes_a : g.plane_bytes_b);
+  const int index = limb < 2 ? 2 * l + limb : 2 * num_moduli + karatsuba_rank(l);
+  const uint8_t* plane = g_ws.ptr + (a ? g.off_planes_a : g.off_planes_b) + (size_t)index * (a ? g.plane_bytes_a : g.plane_bytes_b);
   return launch_decode_plane(plane, a ? M : N, K, g.pitch, out, static_cast<cudaStream_t>(stream)) == cudaSuccess ? OZK_OK
                                                                                                                 : OZK_ERR_CUDA;
 }
@@ -351,6 +356,11 @@ ozk_status ozk_stage_timing_read(float* ms3) {
   }
   for (int i = 0; i < 3; ++i) ms3[i] = (float)(sum[i] / n);
   g_timing.calls = 0;
+  return OZK_OK;
+}
+
+ozk_status ozk_stage_set_karatsuba(int enable) {
+  g_karatsuba = enable != 0;
   return OZK_OK;
 }
 

@@ -19,11 +19,13 @@ constexpr int kCrtWords = 6;         // 192-bit integers cover sum r_l w_l for a
 //                      E2M1 codes of a limb pair (c0, c1), c0 + 13 c1 = residue (mod m), as code(c0) | code(c1) << 4 for
 //                      elements at even k and code(c1) | code(c0) << 4 for elements at odd k
 //   B fragments        of the encoder's mma.sync (kEncTiles tiles of two moduli, 32 lanes, two registers)
+//   sum-limb tables    indexed by an even-k limb-pair byte: the code of c0 + c1 in the low nibble / in the high nibble
 constexpr int kLimbTabStride = 176;  // >= 169, a multiple of 16
 constexpr int kEncTiles = (kMaxModuli + 1) / 2;
 constexpr size_t kLimbTabBytes = (size_t)kMaxModuli * 2 * kLimbTabStride;
 constexpr size_t kEncFragBytes = (size_t)kEncTiles * 32 * 2 * sizeof(uint32_t);
-constexpr size_t kEncTableBytes = kLimbTabBytes + kEncFragBytes;
+constexpr size_t kEncSumTabBytes = 2 * 256;   // limb-pair byte -> E2M1 code of c0 + c1 (low nibble / high nibble): Karatsuba variant
+constexpr size_t kEncTableBytes = kLimbTabBytes + kEncFragBytes + kEncSumTabBytes;
 constexpr int64_t kChunkK = OZK_CHUNK_K;  // longest k range of one limb-GEMM launch: 128 K <= 2^24 keeps FP32 sums exact (|limb| <= 8)
 constexpr int64_t kMaxK = OZK_MAX_K;      // 16 ranges; the grid limits of the O(N^2) kernels lie beyond it
 
@@ -44,6 +46,7 @@ struct Geometry {
   int64_t Mp, Np, Kp;      // padded to 128 / 128 / 256
   int L;
   int c_bits;
+  int karatsuba;           // partial Karatsuba variant (Section 5.1, last paragraph): sum-limb planes after the 2 L regular ones
   // byte offsets into the workspace
   size_t off_status, off_lut, off_amax_a, off_amax_b, off_s, off_t, off_planes_a, off_planes_b, off_res;
   size_t off_res_chunk;                  // second set of residue matrices, present when K > kChunkK (else 0)
@@ -53,6 +56,18 @@ struct Geometry {
 };
 
 static inline int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
+
+// Partial Karatsuba (Section 5.1, last paragraph): moduli all of whose residue classes have a limb pair (c0, c1)
+// whose sum c0 + c1 is again in S, so that a0 b0, a1 b1 and (a0 + a1)(b0 + b1) replace the four products.  In the
+// modulus list these are 83 (index 11) and everything from 73 (index 13) on: the paper's seven among the first 19.
+// An exhaustive search (host side, at table build) checks this rule against the list in use.
+__host__ __device__ constexpr bool karatsuba_modulus(int l) { return l == 11 || l >= 13; }
+__host__ __device__ constexpr int karatsuba_rank(int l) { return l <= 11 ? 0 : l - 12; }   // Karatsuba moduli before index l
+__host__ __device__ constexpr int karatsuba_count(int L) { return L <= 11 ? 0 : (L <= 13 ? 1 : L - 12); }
+// Longest k range of one limb-GEMM launch with the variant on: sum limbs reach 12, 144 K <= 2^24 (Lemma 3)
+constexpr int64_t kChunkKKaratsuba = 65536;
+// Planes per operand: two per modulus, plus one sum-limb plane per Karatsuba modulus when the variant is on
+static inline int planes_per_operand(int L, int karatsuba) { return 2 * L + (karatsuba ? karatsuba_count(L) : 0); }
 
 // ---- per-modulus constants handed to kernels by value --------------------------------
 struct ModulusTable {
@@ -105,7 +120,8 @@ bool host_build_modulus_table(int L, ModulusTable* t);
 bool host_build_crt_table(int L, CrtTable* t);
 
 // kernels' launchers (each returns cudaError_t of the launch)
-cudaError_t launch_build_lut(const ModulusTable& mt, uint8_t* lut, cudaStream_t st);
+cudaError_t launch_build_lut(const ModulusTable& mt, uint8_t* lut, int karatsuba, cudaStream_t st);
+bool karatsuba_enabled();   // process-wide switch of the variant (ozk_api.cu)
 cudaError_t launch_scan_operand(const Geometry& g, int which, const double* X, int64_t ldx, uint8_t* ws, cudaStream_t st);
 cudaError_t launch_encode_operand(const Geometry& g, const ModulusTable& mt, int which, const double* X, int64_t ldx,
                                   uint8_t* ws, int64_t* int_out, cudaStream_t st);

@@ -49,6 +49,8 @@ struct GemmCore {
   unsigned int* wave_counter;  // optional: producers of all CTAs meet here before every wave of items
   int fast_combine;    // K <= 17476: D1 + 13 D2 stays below 2^24 and may be formed in FP32 before the release
   int count_cycles;    // measurement aid: the issuing thread of pair 0 records where its clocks went (status block)
+  int karatsuba;       // CTA-pair kernel: moduli with karatsuba_modulus(l) run three products with sum-limb planes
+  int sum_plane_base;  // plane index of the first sum-limb plane (2 L)
   StatusBlock* status;
   uint32_t scale_word;  // four copies of the UE8M0 scale byte
 };
@@ -126,9 +128,13 @@ __device__ __forceinline__ void decode_item(const GemmCore& p, int item, int& l,
 // multiply-add per element, u = D1 + 13 D2 (|u| <= 128 K + 13 * 64 K < 2^24 for K <= 17476); the
 // conversions, the rest of the weighted sum and the reduction mod m run after the release and
 // overlap the next tile's main loop.  Returns t = D0 + 13 D1 + 169 D2 + offset (non-negative).
-template <bool kFast, bool kZeroTop>
-__device__ __forceinline__ void drain_and_release(uint32_t base, int W, bool top, uint32_t offset, uint32_t release_bar,
+// mode: 0 = modulus 169 (no 13^2 accumulator), 1 = the regular three accumulators [D0 | D1 | D2],
+//       2 = Karatsuba accumulators [a0 b0 | (a0 + a1)(b0 + b1) | a1 b1]: t = D0 + 13 (Ds - D0 - D2) + 169 D2
+//           = D0 + 13 (Ds - D0 + 12 D2), the inner sum below 976 K < 2^24 for K <= 17152.
+template <bool kFast, bool kZeroTop, bool kKara = false>
+__device__ __forceinline__ void drain_and_release(uint32_t base, int W, int mode, uint32_t offset, uint32_t release_bar,
                                                   bool release_remote, int lane, uint32_t (&t)[64]) {
+  const bool top = mode != 0;
   uint32_t u[kFast ? 64 : 1];
 #pragma unroll
   for (int c = 0; c < 2; ++c) {
@@ -139,9 +145,15 @@ __device__ __forceinline__ void drain_and_release(uint32_t base, int W, bool top
       // D0 goes straight into t (raw FP32 bits until after the release): one wait covers all three loads
       tmem_ld_32x32(base + 0 * W + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&t[c * 32]));
       tmem_wait_ld();
+      if (kKara && mode == 2) {
 #pragma unroll
-      for (int e = 0; e < 32; ++e)
-        u[c * 32 + e] = top ? __float_as_uint(fmaf(__uint_as_float(d2[e]), 13.0f, __uint_as_float(d1[e]))) : d1[e];
+        for (int e = 0; e < 32; ++e)
+          u[c * 32 + e] = __float_as_uint(fmaf(__uint_as_float(d2[e]), 12.0f, __uint_as_float(d1[e]) - __uint_as_float(t[c * 32 + e])));
+      } else {
+#pragma unroll
+        for (int e = 0; e < 32; ++e)
+          u[c * 32 + e] = top ? __float_as_uint(fmaf(__uint_as_float(d2[e]), 13.0f, __uint_as_float(d1[e]))) : d1[e];
+      }
     } else {
       uint32_t d0[32];
       tmem_ld_32x32(base + 0 * W + c * 32, d0);
@@ -151,7 +163,8 @@ __device__ __forceinline__ void drain_and_release(uint32_t base, int W, bool top
         const int a0 = __float2int_rn(__uint_as_float(d0[e]));
         const int a1 = __float2int_rn(__uint_as_float(d1[e]));
         const int a2 = top ? __float2int_rn(__uint_as_float(d2[e])) : 0;
-        t[c * 32 + e] = (uint32_t)(a0 + 13 * a1 + 169 * a2) + offset;  // non-negative, < 2^32
+        const int cross = (kKara && mode == 2) ? a1 - a0 - a2 : a1;
+        t[c * 32 + e] = (uint32_t)(a0 + 13 * cross + 169 * a2) + offset;  // non-negative, < 2^32
       }
     }
   }
@@ -220,7 +233,7 @@ struct ResidueEpilogue {
     const uint32_t m = (uint32_t)ep.m[l], recip = ep.recip[l], offset = ep.offset[l];
     const bool top = !(core.skip_top_first && l == 0);
     uint32_t t[64];
-    drain_and_release<kFast, false>(base, W, top, offset, release_bar, false, lane, t);
+    drain_and_release<kFast, false>(base, W, top ? 1 : 0, offset, release_bar, false, lane, t);
     const int64_t j = (int64_t)tp * kTileRows + quad * 32 + lane;
     uint4* dst = reinterpret_cast<uint4*>(ep.res + (size_t)l * ep.res_stride + (size_t)j * (size_t)ep.res_ld +
                                           (size_t)tq * W + half * 64);
@@ -535,7 +548,7 @@ constexpr int kPairStageBytes = 3 * kPTileBytes;  // p0, p1 and this CTA's half 
 constexpr int kPairThreads = 64 + 32 * 8;
 constexpr int kPairZeroBytes = 64 * kTileKBytes;  // this CTA's half of a 128-row all-zero column-side tile
 
-template <bool kFast>
+template <bool kFast, bool kKara>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
 residue_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_q,
                          const __grid_constant__ CUtensorMap map_qh, const __grid_constant__ GemmCore p,
@@ -605,6 +618,7 @@ residue_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
           const long long target = 2 * min((wave + 1) * (long long)npairs, (long long)total_items);
           if (!wave_barrier(p.wave_counter, (unsigned int)target, sh, p.status)) break;
         }
+        const bool kara = kKara && karatsuba_modulus(l);
         for (int kb = 0; kb < p.kblocks; ++kb) {
           if (!wait_bounded(smem_u32(&sh->empty[stage]), phase ^ 1u, sh, p.status, 0x300 + stage)) {
             ok = false;
@@ -619,15 +633,30 @@ residue_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
           // should stay; the row-side tiles are shared only within the current wave and may leave first
           tma_load_3d_pair_hint(dst + 0 * kPTileBytes, &map_p, leader_full, x, prow, 2 * l + 0, pol_keep);
           tma_load_3d_pair_hint(dst + 1 * kPTileBytes, &map_p, leader_full, x, prow, 2 * l + 1, pol_keep);
-          if (p.skip_top_first && l == 0) {
-            // m = 169 needs p0 q0, p0 q1, p1 q0 only: three 128-column instructions, for which this CTA
-            // supplies rows [64 rank, 64 rank + 64) of q0 and of q1 instead of all of one of them
-            tma_load_3d_pair(dst + 2 * kPTileBytes, &map_qh, leader_full, x, tq * W + 64 * (int)rank, 0);
-            tma_load_3d_pair(dst + 2 * kPTileBytes + kPTileBytes / 2, &map_qh, leader_full, x, tq * W + 64 * (int)rank, 1);
+          if ((p.skip_top_first && l == 0) || kara) {
+            // m = 169 needs p0 q0, p0 q1, p1 q0 only, a Karatsuba modulus p0 q0, p1 q1 here (and ps qs from the next
+            // stage): 128-column instructions, for which this CTA supplies rows [64 rank, 64 rank + 64) of q0 and of
+            // q1 instead of all of one of them
+            tma_load_3d_pair(dst + 2 * kPTileBytes, &map_qh, leader_full, x, tq * W + 64 * (int)rank, 2 * l + 0);
+            tma_load_3d_pair(dst + 2 * kPTileBytes + kPTileBytes / 2, &map_qh, leader_full, x, tq * W + 64 * (int)rank, 2 * l + 1);
           } else {
             tma_load_3d_pair_hint(dst + 2 * kPTileBytes, &map_q, leader_full, x, tq * W, 2 * l + (int)rank, pol_stream);
           }
           if (++stage == kPairStages) stage = 0, phase ^= 1u;
+          if (kara) {
+            // second stage of the k block: the sum-limb tiles ps (this CTA's 128 rows) and qs (its 64 rows)
+            if (!wait_bounded(smem_u32(&sh->empty[stage]), phase ^ 1u, sh, p.status, 0x300 + stage)) {
+              ok = false;
+              break;
+            }
+            const uint32_t leader_full2 = map_to_cta(smem_u32(&sh->full[stage]), 0);
+            const uint32_t dst2 = smem_u32(tiles + stage * kPairStageBytes);
+            if (rank == 0) mbar_arrive_expect_tx(smem_u32(&sh->full[stage]), 2 * (kPTileBytes + kPTileBytes / 2));
+            const int sp = p.sum_plane_base + karatsuba_rank(l);
+            tma_load_3d_pair_hint(dst2, &map_p, leader_full2, x, prow, sp, pol_keep);
+            tma_load_3d_pair(dst2 + 2 * kPTileBytes, &map_qh, leader_full2, x, tq * W + 64 * (int)rank, sp);
+            if (++stage == kPairStages) stage = 0, phase ^= 1u;
+          }
         }
       }
     }
@@ -645,6 +674,7 @@ residue_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
         int l, tp, tq;
         decode_item(p, item, l, tp, tq);
         const bool three = p.skip_top_first && l == 0;
+        const bool kara = kKara && karatsuba_modulus(l);
         if (count) clk_a = clock64();
         if (!wait_bounded(smem_u32(&sh->tmem_empty), acc_phase ^ 1u, sh, p.status, 0x400)) break;
         if (count) clk_empty += clock64() - clk_a;
@@ -658,7 +688,31 @@ residue_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
           if (count) clk_full += clock64() - clk_a;
           tc_fence_after();
           const uint32_t base = smem_u32(tiles + stage * kPairStageBytes);
-          if (three) {
+          if (kara) {
+            // Karatsuba: a0 b0 and a1 b1 from this stage, (a0 + a1)(b0 + b1) from the next one
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+              const uint32_t first = (kb == 0 && ks == 0) ? 0u : 1u;
+              mma_mxf4_pair(tmem + 0, smem_desc_sw128(base + 0 * kPTileBytes + ks * 32),
+                            smem_desc_sw128(base + 2 * kPTileBytes + ks * 32), idesc_mxf4_pair(W), sf, sf, first);
+              mma_mxf4_pair(tmem + 2 * W, smem_desc_sw128(base + 1 * kPTileBytes + ks * 32),
+                            smem_desc_sw128(base + 2 * kPTileBytes + kPTileBytes / 2 + ks * 32), idesc_mxf4_pair(W), sf, sf, first);
+            }
+            mma_commit_pair(smem_u32(&sh->empty[stage]), (uint16_t)3);
+            if (++stage == kPairStages) stage = 0, phase ^= 1u;
+            if (count) clk_a = clock64();
+            if (!wait_bounded(smem_u32(&sh->full[stage]), phase, sh, p.status, 0x410 + stage)) {
+              ok = false;
+              break;
+            }
+            if (count) clk_full += clock64() - clk_a;
+            tc_fence_after();
+            const uint32_t base2 = smem_u32(tiles + stage * kPairStageBytes);
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)
+              mma_mxf4_pair(tmem + W, smem_desc_sw128(base2 + ks * 32), smem_desc_sw128(base2 + 2 * kPTileBytes + ks * 32),
+                            idesc_mxf4_pair(W), sf, sf, (kb == 0 && ks == 0) ? 0u : 1u);
+          } else if (three) {
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks) {
               const uint32_t first = (kb == 0 && ks == 0) ? 0u : 1u;
@@ -714,7 +768,8 @@ residue_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
       tc_fence_after();
       const uint32_t m = (uint32_t)ep.m[l], recip = ep.recip[l], offset = ep.offset[l];
       uint32_t t[64];
-      drain_and_release<kFast, false>(base, W, !(p.skip_top_first && l == 0), offset, leader_empty, true, lane, t);
+      const int mode = (p.skip_top_first && l == 0) ? 0 : ((kKara && karatsuba_modulus(l)) ? 2 : 1);
+      drain_and_release<kFast, false, kKara>(base, W, mode, offset, leader_empty, true, lane, t);
       const int64_t j = (int64_t)(2 * tp + (int)rank) * kTileRows + quad * 32 + lane;
       uint4* dst = reinterpret_cast<uint4*>(ep.res + (size_t)l * ep.res_stride + (size_t)j * (size_t)ep.res_ld +
                                             (size_t)tq * W + half * 64);
@@ -927,12 +982,14 @@ ozk_status launch_limb_gemm(const CUtensorMap& map_p, const CUtensorMap& map_q, 
 ozk_status gemm_residues(const Geometry& g, const ModulusTable& mt, uint8_t* ws, cudaStream_t st, int64_t k0, int64_t klen,
                          uint8_t* res) {
   if (klen <= 0) klen = g.Kp - k0;
-  if (k0 < 0 || k0 % kTileKNibbles || klen % kTileKNibbles || k0 + klen > g.Kp || klen > kChunkK) return OZK_ERR_INVALID_ARG;
+  if (k0 < 0 || k0 % kTileKNibbles || klen % kTileKNibbles || k0 + klen > g.Kp || klen > (g.karatsuba ? kChunkKKaratsuba : kChunkK))
+    return OZK_ERR_INVALID_ARG;
   const uint8_t* planes_b = ws + g.off_planes_b + k0 / 2;
   const uint8_t* planes_a = ws + g.off_planes_a + k0 / 2;
   CUtensorMap map_p, map_q;
-  if (!make_plane_map(&map_p, planes_b, klen / 2, g.Np, 2 * g.L, g.plane_bytes_b, kTileRows, g.pitch)) return OZK_ERR_CUDA;
-  if (!make_plane_map(&map_q, planes_a, klen / 2, g.Mp, 2 * g.L, g.plane_bytes_a, 128, g.pitch)) return OZK_ERR_CUDA;
+  const int planes = planes_per_operand(g.L, g.karatsuba);
+  if (!make_plane_map(&map_p, planes_b, klen / 2, g.Np, planes, g.plane_bytes_b, kTileRows, g.pitch)) return OZK_ERR_CUDA;
+  if (!make_plane_map(&map_q, planes_a, klen / 2, g.Mp, planes, g.plane_bytes_a, 128, g.pitch)) return OZK_ERR_CUDA;
   GemmCore core;
   core.L = g.L;
   core.tiles_p = (int)(g.Np / kTileRows);
@@ -941,8 +998,11 @@ ozk_status gemm_residues(const Geometry& g, const ModulusTable& mt, uint8_t* ws,
   core.group = 16;
   core.skip_top_first = (mt.m[0] == 169) ? 1 : 0;  // 13^2 a1 b1 vanishes mod 169 (Section 5.1)
   core.q_groups = 0;
-  core.fast_combine = (g.K <= 17476 || klen <= 17408) ? 1 : 0;  // 128 K + 13 * 64 K = 960 K < 2^24
+  // one FP32 multiply-add before the release needs 128 K + 13 * 64 K = 960 K < 2^24 (Karatsuba: 976 K)
+  core.fast_combine = (g.karatsuba ? klen <= 17152 : (g.K <= 17476 || klen <= 17408)) ? 1 : 0;
   core.count_cycles = 0;
+  core.karatsuba = 0;  // the single-CTA kernel runs the four products on the same planes
+  core.sum_plane_base = 0;
   core.wave_counter = nullptr;
   core.status = reinterpret_cast<StatusBlock*>(ws + g.off_status);
   core.scale_word = 0x80808080u;  // UE8M0 byte 0x80 = 2: both operands doubled, accumulators hold integers
@@ -964,15 +1024,19 @@ ozk_status gemm_residues(const Geometry& g, const ModulusTable& mt, uint8_t* ws,
     pc.skip_top_first = (mt.m[0] == 169 && three_product_enabled()) ? 1 : 0;  // 13^2 a1 b1 vanishes mod 169 (Section 5.1)
     pc.count_cycles = stage_timing_enabled() ? 1 : 0;
     CUtensorMap map_qh;  // 64-row boxes of the A-side planes, for the three-product form of m = 169
-    if (!make_plane_map(&map_qh, planes_a, klen / 2, g.Mp, 2 * g.L, g.plane_bytes_a, 64, g.pitch)) return OZK_ERR_CUDA;
+    if (!make_plane_map(&map_qh, planes_a, klen / 2, g.Mp, planes, g.plane_bytes_a, 64, g.pitch)) return OZK_ERR_CUDA;
+    pc.karatsuba = g.karatsuba;
+    pc.sum_plane_base = 2 * g.L;
     pc.wave_counter = reinterpret_cast<unsigned int*>(ws + g.off_status + 512);
     const size_t smem = (size_t)kPairStages * kPairStageBytes + kPairZeroBytes + sizeof(GemmShared) + 1024;
     static std::atomic<bool> attr_set[kMaxDevices];
     const int dev = current_device_ordinal();
     if (dev < 0) return OZK_ERR_CUDA;
     if (!attr_set[dev].load(std::memory_order_acquire)) {
-      if (cudaFuncSetAttribute(residue_gemm_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
-          cudaFuncSetAttribute(residue_gemm_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      if (cudaFuncSetAttribute(residue_gemm_pair_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+          cudaFuncSetAttribute(residue_gemm_pair_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+          cudaFuncSetAttribute(residue_gemm_pair_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+          cudaFuncSetAttribute(residue_gemm_pair_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return OZK_ERR_CUDA;
       attr_set[dev].store(true, std::memory_order_release);
     }
@@ -991,8 +1055,13 @@ ozk_status gemm_residues(const Geometry& g, const ModulusTable& mt, uint8_t* ws,
     attr[0].val.cooperative = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    const cudaError_t e = pc.fast_combine ? cudaLaunchKernelEx(&cfg, residue_gemm_pair_kernel<true>, map_p, map_q, map_qh, pc, ep)
-                                          : cudaLaunchKernelEx(&cfg, residue_gemm_pair_kernel<false>, map_p, map_q, map_qh, pc, ep);
+    cudaError_t e;
+    if (pc.karatsuba)
+      e = pc.fast_combine ? cudaLaunchKernelEx(&cfg, residue_gemm_pair_kernel<true, true>, map_p, map_q, map_qh, pc, ep)
+                          : cudaLaunchKernelEx(&cfg, residue_gemm_pair_kernel<false, true>, map_p, map_q, map_qh, pc, ep);
+    else
+      e = pc.fast_combine ? cudaLaunchKernelEx(&cfg, residue_gemm_pair_kernel<true, false>, map_p, map_q, map_qh, pc, ep)
+                          : cudaLaunchKernelEx(&cfg, residue_gemm_pair_kernel<false, false>, map_p, map_q, map_qh, pc, ep);
     if (e == cudaSuccess) return OZK_OK;
     (void)cudaGetLastError();  // the cooperative launch was refused: fall through to the single-CTA kernel
   }
@@ -1021,6 +1090,8 @@ ozk_status gemm_int8(const uint8_t* planes_a, const uint8_t* planes_b, int64_t M
   core.wave_counter = nullptr;
   core.fast_combine = 0;
   core.count_cycles = 0;
+  core.karatsuba = 0;
+  core.sum_plane_base = 0;
   core.status = status;
   core.scale_word = 0x80808080u;
   Int32Epilogue::Params ep;
@@ -1050,6 +1121,8 @@ ozk_status gemm_oz1_passes(const uint8_t* planes_a, const uint8_t* planes_b, int
   core.wave_counter = nullptr;
   core.fast_combine = 0;
   core.count_cycles = 0;
+  core.karatsuba = 0;
+  core.sum_plane_base = 0;
   core.status = status;
   core.scale_word = 0x80808080u;
   Int64BlockEpilogue::Params ep;

@@ -86,6 +86,7 @@ bool make_host_layout(int64_t M, int64_t N, int64_t K, int L, HostLayout* h) {
   if (h->cblocks < 1) h->cblocks = 1;
   if (h->rblocks > kMaxBlocks || h->cblocks > kMaxBlocks) return false;
   if (!make_geometry(h->mb, h->nb, K, L, &h->g)) return false;
+  h->g.karatsuba = 0;  // the host-buffer path keeps the two planes per modulus
   const Geometry& g = h->g;
   auto up = [](size_t x) { return (x + 1023) / 1024 * 1024; };
   const size_t kk = (size_t)(K > 0 ? K : 1);
@@ -187,7 +188,7 @@ ozk_status ozk_dgemm_host(int64_t M, int64_t N, int64_t K, const double* A, int6
   OZK_TRY(cudaEventRecord(p.start, st));
   OZK_TRY(cudaStreamWaitEvent(p.s_in, p.start, 0));
   OZK_TRY(cudaStreamWaitEvent(p.s_out, p.start, 0));
-  OZK_TRY(launch_build_lut(mt, ws + h.off_lut, st));
+  OZK_TRY(launch_build_lut(mt, ws + h.off_lut, 0, st));
   auto rows_of = [&](int r) { const int64_t i0 = (int64_t)r * h.mb; return M - i0 < h.mb ? M - i0 : h.mb; };
   auto cols_of = [&](int b) { const int64_t j0 = (int64_t)b * h.nb; return N - j0 < h.nb ? N - j0 : h.nb; };
   int out_index = 0;

@@ -25,9 +25,23 @@ __device__ __constant__ int8_t kDoubledE2M1[8] = {0, 1, 2, 3, 4, 6, 8, 12};
 // The tables are indexed by t = (residue + 2^62) mod m, the value the encoder's contraction yields.
 // Block l < L writes the two byte tables of modulus l; block L writes the B fragments of the encoder's MMA.
 // ------------------------------------------------------------------------------------
-__global__ void build_lut_kernel(ModulusTable mt, uint8_t* __restrict__ tables) {
+__global__ void build_lut_kernel(ModulusTable mt, uint8_t* __restrict__ tables, int karatsuba) {
   const int l = blockIdx.x;
   if (l == mt.L) {
+    // sum-limb tables of the Karatsuba variant: the limb-pair byte of an even-k element (code(c0) | code(c1) << 4)
+    // gives the code of c0 + c1, in the low nibble (first table) and in the high nibble (second table)
+    {
+      uint8_t* sum_tab = tables + kLimbTabBytes + kEncFragBytes;
+      const int x = threadIdx.x;  // 256 threads
+      const int i0 = x & 15, i1 = x >> 4;
+      const int c0 = kDoubledE2M1[i0 & 7] * ((i0 & 8) ? -1 : 1), c1 = kDoubledE2M1[i1 & 7] * ((i1 & 8) ? -1 : 1);
+      const int sum = c0 + c1;
+      int code = 0;  // pairs whose sum is not in S never occur in a Karatsuba table
+      for (int i = 0; i < 16; ++i)
+        if (i != 8 && kDoubledE2M1[i & 7] * ((i & 8) ? -1 : 1) == sum) code = i;
+      sum_tab[x] = (uint8_t)code;
+      sum_tab[256 + x] = (uint8_t)(code << 4);
+    }
     // B fragments (m16n8k32, u8 x u8): tile T holds the moduli 2 T and 2 T + 1.  Column n of a tile belongs to
     // lane n / 2 of every quad and to modulus 2 T + n % 2: it is non-zero only in the k slots of that lane (bytes 0..3
     // of its element in slots 4 q .. 4 q + 3, bytes 4..7 in slots 16 + 4 q ..), where it holds 2^(8 p) mod m.
@@ -60,7 +74,12 @@ __global__ void build_lut_kernel(ModulusTable mt, uint8_t* __restrict__ tables) 
       const int c0 = kDoubledE2M1[i0 & 7] * ((i0 & 8) ? -1 : 1);
       const int c1 = kDoubledE2M1[i1 & 7] * ((i1 & 8) ? -1 : 1);
       const int a0 = abs(c0), a1 = abs(c1);
-      if (max(a0, a1) <= 8) {  // every class of every modulus has a pair with |c| <= 8 (keeps 128 K <= 2^24)
+      bool admissible = max(a0, a1) <= 8;  // every class of every modulus has a pair with |c| <= 8 (keeps 128 K <= 2^24)
+      if (karatsuba && karatsuba_modulus(l)) {  // the sum limb must be representable as well (Section 5.1, last paragraph)
+        const int sa = abs(c0 + c1);
+        admissible = admissible && (sa <= 4 || sa == 6 || sa == 8 || sa == 12);
+      }
+      if (admissible) {
         // fewest negative limbs first (sign changes in the operand streams cost power on the tensor pipe:
         // a few per cent of the limb GEMM's time under the power cap), then smallest magnitudes
         const int key = 2000 * ((c0 < 0) + (c1 < 0)) + max(a0, a1) * 64 + (a0 + a1);
@@ -221,10 +240,11 @@ bool enc_moduli_match(const ModulusTable& mt) {
 struct EncTables {
   uint8_t limb[kMaxModuli][2][kLimbTabStride];
   uint2 frag[kEncTiles][32];
+  uint8_t sum[2][256];
 };
-static_assert(sizeof(EncTables) == kLimbTabBytes + kEncFragBytes, "shared copy mirrors the workspace layout");
+static_assert(sizeof(EncTables) == kEncTableBytes, "shared copy mirrors the workspace layout");
 __device__ __forceinline__ void load_tables(const uint8_t* __restrict__ tables, int L, EncTables* tab) {
-  const int limb_vec = L * 2 * kLimbTabStride / 16, frag_vec = (int)(kEncFragBytes / 16);
+  const int limb_vec = L * 2 * kLimbTabStride / 16, frag_vec = (int)((kEncFragBytes + kEncSumTabBytes) / 16);
   const uint4* src = reinterpret_cast<const uint4*>(tables);
   const uint4* src_frag = reinterpret_cast<const uint4*>(tables + kLimbTabBytes);
   uint4* dst = reinterpret_cast<uint4*>(tab->limb);
@@ -235,6 +255,7 @@ __device__ __forceinline__ void load_tables(const uint8_t* __restrict__ tables, 
 
 // Plane words of the thread's eight elements for every modulus, stored at dst + plane * plane_bytes.
 // Warp-collective (all 32 lanes must call it).
+template <bool kKaratsuba>
 __device__ __forceinline__ void encode_planes(const Shifted8& v, int L, const EncTables& tab, uint8_t* dst, size_t plane_bytes) {
   const int lane = threadIdx.x & 31;
 #pragma unroll
@@ -263,6 +284,20 @@ __device__ __forceinline__ void encode_planes(const Shifted8& v, int L, const En
       // even table: code(c0) | code(c1) << 4, odd table: code(c1) | code(c0) << 4
       *reinterpret_cast<uint32_t*>(dst + (size_t)(2 * l) * plane_bytes) = (xa & 0x0F0F0F0Fu) | (xb & 0xF0F0F0F0u);
       *reinterpret_cast<uint32_t*>(dst + (size_t)(2 * l + 1) * plane_bytes) = ((xa >> 4) & 0x0F0F0F0Fu) | ((xb << 4) & 0xF0F0F0F0u);
+      if constexpr (kKaratsuba) {
+        if (karatsuba_modulus(l)) {
+          // sum-limb plane: code(c0 + c1) from the pair byte (odd-k bytes carry the nibbles swapped: swap them back)
+          uint32_t sa[4], sb[4];
+#pragma unroll
+          for (int h = 0; h < 4; ++h) {
+            sa[h] = tab.sum[0][ea[h]];
+            sb[h] = tab.sum[1][((eb[h] << 4) | (eb[h] >> 4)) & 0xFFu];
+          }
+          const uint32_t ya = __byte_perm(__byte_perm(sa[0], sa[1], 0x0040), __byte_perm(sa[2], sa[3], 0x0040), 0x5410);
+          const uint32_t yb = __byte_perm(__byte_perm(sb[0], sb[1], 0x0040), __byte_perm(sb[2], sb[3], 0x0040), 0x5410);
+          *reinterpret_cast<uint32_t*>(dst + (size_t)(2 * L + karatsuba_rank(l)) * plane_bytes) = ya | yb;
+        }
+      }
     }
   }
 }
@@ -272,6 +307,7 @@ __device__ __forceinline__ void encode_planes(const Shifted8& v, int L, const En
 // Block = 256 threads = 2048 consecutive k of one column; thread = 8 consecutive k (a warp = 256 k: whole warps
 // lie inside or outside the padded K, which is a multiple of 256).
 // ------------------------------------------------------------------------------------
+template <bool kKaratsuba>
 __global__ void __launch_bounds__(256) encode_cols_kernel(const double* __restrict__ B, int64_t ldb, int64_t N, int64_t K,
                                                           int64_t Kp, int L, const uint8_t* __restrict__ tables,
                                                           const int32_t* __restrict__ shifts, uint8_t* __restrict__ planes,
@@ -310,7 +346,7 @@ __global__ void __launch_bounds__(256) encode_cols_kernel(const double* __restri
     }
     Shifted8 v;
     shift8(a, v);
-    encode_planes(v, L, tab, planes + (size_t)j * pitch + (size_t)(k / 2), plane_bytes);
+    encode_planes<kKaratsuba>(v, L, tab, planes + (size_t)j * pitch + (size_t)(k / 2), plane_bytes);
   }
 }
 
@@ -327,6 +363,7 @@ constexpr int kRowTileK = 128;
 constexpr int kGroupStride = 9;                                         // doubles per group of 8 k (8 used)
 constexpr int kRowStride = (kRowTileK / 8) * kGroupStride + 1;          // doubles per row: 145, odd
 
+template <bool kKaratsuba>
 __global__ void __launch_bounds__(256) encode_rows_kernel(const double* __restrict__ A, int64_t lda, int64_t M, int64_t K,
                                                           int64_t Kp, int L, const uint8_t* __restrict__ tables,
                                                           const int32_t* __restrict__ shifts, uint8_t* __restrict__ planes,
@@ -366,7 +403,7 @@ __global__ void __launch_bounds__(256) encode_rows_kernel(const double* __restri
     }
     Shifted8 v;
     shift8(a, v);
-    encode_planes(v, L, tab, planes + (size_t)i * pitch + (size_t)(k0 / 2) + 4 * g, plane_bytes);
+    encode_planes<kKaratsuba>(v, L, tab, planes + (size_t)i * pitch + (size_t)(k0 / 2) + 4 * g, plane_bytes);
   }
 }
 
@@ -384,8 +421,8 @@ __global__ void decode_plane_kernel(const uint8_t* __restrict__ plane, int64_t r
 
 }  // namespace
 
-cudaError_t launch_build_lut(const ModulusTable& mt, uint8_t* lut, cudaStream_t st) {
-  build_lut_kernel<<<mt.L + 1, 256, 0, st>>>(mt, lut);
+cudaError_t launch_build_lut(const ModulusTable& mt, uint8_t* lut, int karatsuba, cudaStream_t st) {
+  build_lut_kernel<<<mt.L + 1, 256, 0, st>>>(mt, lut, karatsuba);
   return cudaGetLastError();
 }
 
@@ -433,11 +470,13 @@ cudaError_t launch_encode_operand(const Geometry& g, const ModulusTable& mt, int
   const int reps = 4;
   if (which == 0) {
     dim3 grid((unsigned)(g.Mp / kRowTile), (unsigned)((g.Kp / kRowTileK + reps - 1) / reps));
-    encode_rows_kernel<<<grid, 256, 0, st>>>(X, ldx, g.M, g.K, g.Kp, mt.L, tables, reinterpret_cast<const int32_t*>(ws + g.off_s),
+    auto* kernel = g.karatsuba ? encode_rows_kernel<true> : encode_rows_kernel<false>;
+    kernel<<<grid, 256, 0, st>>>(X, ldx, g.M, g.K, g.Kp, mt.L, tables, reinterpret_cast<const int32_t*>(ws + g.off_s),
                                              ws + g.off_planes_a, g.plane_bytes_a, g.pitch, int_out, reps);
   } else {
     dim3 grid((unsigned)g.Np, (unsigned)(((g.Kp + 2047) / 2048 + reps - 1) / reps));
-    encode_cols_kernel<<<grid, 256, 0, st>>>(X, ldx, g.N, g.K, g.Kp, mt.L, tables, reinterpret_cast<const int32_t*>(ws + g.off_t),
+    auto* kernel = g.karatsuba ? encode_cols_kernel<true> : encode_cols_kernel<false>;
+    kernel<<<grid, 256, 0, st>>>(X, ldx, g.N, g.K, g.Kp, mt.L, tables, reinterpret_cast<const int32_t*>(ws + g.off_t),
                                              ws + g.off_planes_b, g.plane_bytes_b, g.pitch, int_out, reps);
   }
   return cudaGetLastError();

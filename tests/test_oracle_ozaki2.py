@@ -10,7 +10,7 @@ from fractions import Fraction
 import numpy as np
 import pytest
 
-from oracle import exact, moduli, ozaki2
+from oracle import base13, exact, moduli, ozaki2
 from paper_2608_06812_b200 import inputs
 
 GOLD = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "paper_constants.json")))
@@ -314,3 +314,30 @@ def test_limb_products_through_float64_are_exact_at_the_headline_k():
             got = ozaki2.residue_product(At, Bt, m)
             want = np.array([[sum(int(At[i, k]) * int(Bt[k, j]) for k in range(K)) % m for j in range(2)] for i in range(3)])
             assert np.array_equal(np.asarray(got, dtype=np.int64), want), (m, kind)
+
+
+def test_karatsuba_moduli_are_the_papers_seven():
+    """Section 5.1, last paragraph: among the 19 moduli exactly 83, 73, 71, 67, 61, 59, 53 have, in every residue
+    class, a limb pair whose sum is representable too (68 products instead of 75)."""
+    mods = moduli.select_moduli(19)
+    assert moduli.karatsuba_moduli(mods) == [83, 73, 71, 67, 61, 59, 53]
+    assert 4 * 19 - 1 - len(moduli.karatsuba_moduli(mods)) == 68
+    # the continuation of the list (47 ... 11) admits it as well; 79 and everything above 83 does not
+    assert moduli.karatsuba_moduli(moduli.select_moduli(27)) == [83, 73, 71, 67, 61, 59, 53, 47, 43, 41, 31, 29, 19, 17, 11]
+    for m in (83, 53, 11):
+        for rho, (c0, c1) in enumerate(moduli.limb_pair_table_karatsuba(m)):
+            assert c0 in base13.S and c1 in base13.S and c0 + c1 in base13.S and (c0 + 13 * c1 - rho) % m == 0
+            assert max(abs(c0), abs(c1)) <= 8                          # sum limbs reach 12, the limbs themselves 8
+
+
+def test_karatsuba_residue_product_equals_the_four_product_form():
+    rng = np.random.default_rng(8)
+    At = rng.integers(-2 ** 52, 2 ** 52, size=(5, 300), dtype=np.int64)
+    Bt = rng.integers(-2 ** 52, 2 ** 52, size=(300, 4), dtype=np.int64)
+    for m in (83, 73, 71, 67, 61, 59, 53, 11):
+        got = ozaki2.residue_product_karatsuba(At, Bt, m)
+        assert np.array_equal(got, ozaki2.residue_product(At, Bt, m))
+        want = np.array([[sum(int(At[i, k]) * int(Bt[k, j]) for k in range(300)) % m for j in range(4)] for i in range(5)])
+        assert np.array_equal(got, want)
+    with pytest.raises(ValueError):
+        ozaki2.residue_product_karatsuba(At, Bt, 79)
