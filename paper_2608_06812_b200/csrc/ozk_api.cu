@@ -48,6 +48,8 @@ bool make_geometry_impl(int64_t M, int64_t N, int64_t K, int L, Geometry* g, int
   g->Kp = round_up(K > 0 ? K : 1, kTileKNibbles);
   g->c_bits = host_capacity_bits(K, L, max_bits);
   g->karatsuba = (g_karatsuba && karatsuba_count(L) > 0) ? 1 : 0;
+  // short K on CTA pairs: two-accumulator form with gamma planes on the A side
+  g->gamma = (!g->karatsuba && gamma_form_enabled() && K > 0 && K <= kGammaMaxK && g->Np % 256 == 0) ? 1 : 0;
   size_t off = 0;
   g->off_status = off;
   off += align_up(sizeof(StatusBlock), 1024);
@@ -66,7 +68,7 @@ bool make_geometry_impl(int64_t M, int64_t N, int64_t K, int L, Geometry* g, int
   g->plane_bytes_a = (size_t)g->Mp * g->pitch;
   g->plane_bytes_b = (size_t)g->Np * g->pitch;
   g->off_planes_a = off;
-  off += (size_t)planes_per_operand(L, g->karatsuba) * g->plane_bytes_a;
+  off += (size_t)planes_of_a(L, g->karatsuba, g->gamma) * g->plane_bytes_a;
   g->off_planes_b = off;
   off += (size_t)planes_per_operand(L, g->karatsuba) * g->plane_bytes_b;
   g->off_res = off;
@@ -149,6 +151,14 @@ ozk_status gemm_residues_chunked(const Geometry& g, const ModulusTable& mt, uint
   return OZK_OK;
 }
 bool karatsuba_enabled() { return g_karatsuba; }
+bool gamma_form_enabled() {
+  static int v = -1;
+  if (v < 0) {
+    const char* e = getenv("OZK_GEMM_GAMMA");
+    v = (e && e[0] == '0') ? 0 : 1;
+  }
+  return v == 1;
+}
 bool stage_timing_enabled() { return g_timing.enabled; }
 uint8_t* workspace_ptr() { return g_ws.ptr; }
 size_t workspace_bytes() { return g_ws.bytes; }
@@ -250,10 +260,11 @@ ozk_status ozk_stage_read_planes(char operand, int64_t M, int64_t N, int64_t K, 
   Geometry g;
   ozk_status rc = check_common(M, N, K, num_moduli, &g);
   if (rc != OZK_OK) return rc;
-  if (!out || l < 0 || l >= num_moduli || limb < 0 || limb > 2 || (operand != 'A' && operand != 'B')) return OZK_ERR_INVALID_ARG;
+  if (!out || l < 0 || l >= num_moduli || limb < 0 || limb > 4 || (operand != 'A' && operand != 'B')) return OZK_ERR_INVALID_ARG;
   if (limb == 2 && !(g.karatsuba && karatsuba_modulus(l))) return OZK_ERR_INVALID_ARG;  // sum-limb planes exist in the Karatsuba variant only
   const bool a = operand == 'A';
-  const int index = limb < 2 ? 2 * l + limb : 2 * num_moduli + karatsuba_rank(l);
+  if (limb >= 3 && !(a && g.gamma)) return OZK_ERR_INVALID_ARG;                          // gamma planes: A side, short K
+  const int index = limb < 2 ? 2 * l + limb : (limb == 2 ? 2 * num_moduli + karatsuba_rank(l) : 2 * num_moduli + 2 * l + (limb - 3));
   const uint8_t* plane = g_ws.ptr + (a ? g.off_planes_a : g.off_planes_b) + (size_t)index * (a ? g.plane_bytes_a : g.plane_bytes_b);
   return launch_decode_plane(plane, a ? M : N, K, g.pitch, out, static_cast<cudaStream_t>(stream)) == cudaSuccess ? OZK_OK
                                                                                                                 : OZK_ERR_CUDA;

@@ -20,12 +20,13 @@ constexpr int kCrtWords = 6;         // 192-bit integers cover sum r_l w_l for a
 //                      elements at even k and code(c1) | code(c0) << 4 for elements at odd k
 //   B fragments        of the encoder's mma.sync (kEncTiles tiles of two moduli, 32 lanes, two registers)
 //   sum-limb tables    indexed by an even-k limb-pair byte: the code of c0 + c1 in the low nibble / in the high nibble
+//   gamma tables       like the limb-pair tables, for the residue class 13 * residue (two-accumulator form)
 constexpr int kLimbTabStride = 176;  // >= 169, a multiple of 16
 constexpr int kEncTiles = (kMaxModuli + 1) / 2;
 constexpr size_t kLimbTabBytes = (size_t)kMaxModuli * 2 * kLimbTabStride;
 constexpr size_t kEncFragBytes = (size_t)kEncTiles * 32 * 2 * sizeof(uint32_t);
 constexpr size_t kEncSumTabBytes = 2 * 256;   // limb-pair byte -> E2M1 code of c0 + c1 (low nibble / high nibble): Karatsuba variant
-constexpr size_t kEncTableBytes = kLimbTabBytes + kEncFragBytes + kEncSumTabBytes;
+constexpr size_t kEncTableBytes = kLimbTabBytes + kEncFragBytes + kEncSumTabBytes + kLimbTabBytes;   // last: gamma tables
 constexpr int64_t kChunkK = OZK_CHUNK_K;  // longest k range of one limb-GEMM launch: 128 K <= 2^24 keeps FP32 sums exact (|limb| <= 8)
 constexpr int64_t kMaxK = OZK_MAX_K;      // 16 ranges; the grid limits of the O(N^2) kernels lie beyond it
 
@@ -47,6 +48,7 @@ struct Geometry {
   int L;
   int c_bits;
   int karatsuba;           // partial Karatsuba variant (Section 5.1, last paragraph): sum-limb planes after the 2 L regular ones
+  int gamma;               // two-accumulator form for short K: the A side also carries the limb planes of 13 a mod m (after its 2 L planes)
   // byte offsets into the workspace
   size_t off_status, off_lut, off_amax_a, off_amax_b, off_s, off_t, off_planes_a, off_planes_b, off_res;
   size_t off_res_chunk;                  // second set of residue matrices, present when K > kChunkK (else 0)
@@ -68,6 +70,14 @@ __host__ __device__ constexpr int karatsuba_count(int L) { return L <= 11 ? 0 : 
 constexpr int64_t kChunkKKaratsuba = 65536;
 // Planes per operand: two per modulus, plus one sum-limb plane per Karatsuba modulus when the variant is on
 static inline int planes_per_operand(int L, int karatsuba) { return 2 * L + (karatsuba ? karatsuba_count(L) : 0); }
+// Two-accumulator form of the residue product (used for short K, where the turn-around between tiles weighs most):
+//   a b = a0 beta + a1 gamma (mod m),  beta = b mod m,  gamma = 13 b mod m,  each in two limbs, so that
+//   D_lo = a0 beta0 + a1 gamma0,  D_hi = a0 beta1 + a1 gamma1,  r = (D_lo + 13 D_hi) mod m
+// needs two accumulators of W columns instead of three; with W = 120 two sets fit tensor memory and the read-back of one
+// tile overlaps the products of the next.  The A-matrix side carries beta (its regular planes) and gamma (2 L more).
+constexpr int kGammaTileW = 120;
+constexpr int64_t kGammaMaxK = 768;    // longest K that takes this form: measured faster up to here, slower from 1024 on (more operand traffic)
+static inline int planes_of_a(int L, int karatsuba, int gamma) { return planes_per_operand(L, karatsuba) + (gamma ? 2 * L : 0); }
 
 // ---- per-modulus constants handed to kernels by value --------------------------------
 struct ModulusTable {
@@ -122,6 +132,7 @@ bool host_build_crt_table(int L, CrtTable* t);
 // kernels' launchers (each returns cudaError_t of the launch)
 cudaError_t launch_build_lut(const ModulusTable& mt, uint8_t* lut, int karatsuba, cudaStream_t st);
 bool karatsuba_enabled();   // process-wide switch of the variant (ozk_api.cu)
+bool gamma_form_enabled();  // two-accumulator form for short K (on unless OZK_GEMM_GAMMA=0: a measurement aid)
 cudaError_t launch_scan_operand(const Geometry& g, int which, const double* X, int64_t ldx, uint8_t* ws, cudaStream_t st);
 cudaError_t launch_encode_operand(const Geometry& g, const ModulusTable& mt, int which, const double* X, int64_t ldx,
                                   uint8_t* ws, int64_t* int_out, cudaStream_t st);

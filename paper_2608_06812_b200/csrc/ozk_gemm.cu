@@ -67,15 +67,15 @@ struct __align__(8) GemmShared {
 
 // Bounded wait on an mbarrier phase.  Returns false after the time limit or when another role
 // of this CTA has already given up.
-__device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, GemmShared* sh, StatusBlock* status, int where) {
+__device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, volatile int* abort, StatusBlock* status, int where) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_timer_ns();
   for (uint32_t it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 63u) == 0u) {
-      if (sh->abort) return false;
+      if (*abort) return false;
       if (global_timer_ns() - t0 > kWaitLimitNs) {
-        sh->abort = 1;
+        *abort = 1;
         atomicMin(&status->code, (int)OZK_ERR_DEVICE_TIMEOUT);
         atomicExch(&status->where, where);
         return false;
@@ -90,7 +90,7 @@ __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, Gemm
 // done so.  It keeps the CTAs of a wave within one tile of each other, so that tiles requested by
 // several CTAs are still in L2 when the last of them asks.  Needs all CTAs resident (persistent
 // grid, cooperative launch).  Returns false on expiry.
-__device__ __forceinline__ bool wave_barrier(unsigned int* counter, unsigned int target, GemmShared* sh, StatusBlock* status) {
+__device__ __forceinline__ bool wave_barrier(unsigned int* counter, unsigned int target, volatile int* abort, StatusBlock* status) {
   atomicAdd(counter, 1u);
   const uint64_t t0 = global_timer_ns();
   for (uint32_t it = 0;; ++it) {
@@ -99,9 +99,9 @@ __device__ __forceinline__ bool wave_barrier(unsigned int* counter, unsigned int
     if (v >= target) return true;
     __nanosleep(64);
     if ((it & 63u) == 63u) {
-      if (sh->abort) return false;
+      if (*abort) return false;
       if (global_timer_ns() - t0 > kWaitLimitNs) {
-        sh->abort = 1;
+        *abort = 1;
         atomicMin(&status->code, (int)OZK_ERR_DEVICE_TIMEOUT);
         atomicExch(&status->where, 0x700);
         return false;
@@ -411,10 +411,10 @@ limb_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constan
         if (p.wave_counter) {
           const long long wave = item / (int)gridDim.x;
           const long long target = min((wave + 1) * (long long)gridDim.x, (long long)total_items);
-          if (!wave_barrier(p.wave_counter, (unsigned int)target, sh, p.status)) break;
+          if (!wave_barrier(p.wave_counter, (unsigned int)target, &sh->abort, p.status)) break;
         }
         for (int kb = 0; kb < p.kblocks; ++kb) {
-          if (!wait_bounded(smem_u32(&sh->empty[stage]), phase ^ 1u, sh, p.status, 0x000 + stage)) {
+          if (!wait_bounded(smem_u32(&sh->empty[stage]), phase ^ 1u, &sh->abort, p.status, 0x000 + stage)) {
             ok = false;
             break;
           }
@@ -455,10 +455,10 @@ limb_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constan
         int l, tp, tq;
         decode_item(p, item, l, tp, tq);
         const bool skip_top = p.skip_top_first && l == 0;
-        if (!wait_bounded(smem_u32(&sh->tmem_empty), acc_phase ^ 1u, sh, p.status, 0x100)) break;
+        if (!wait_bounded(smem_u32(&sh->tmem_empty), acc_phase ^ 1u, &sh->abort, p.status, 0x100)) break;
         tc_fence_after();
         for (int kb = 0; kb < p.kblocks; ++kb) {
-          if (!wait_bounded(smem_u32(&sh->full[stage]), phase, sh, p.status, 0x110 + stage)) {
+          if (!wait_bounded(smem_u32(&sh->full[stage]), phase, &sh->abort, p.status, 0x110 + stage)) {
             ok = false;
             break;
           }
@@ -512,7 +512,7 @@ limb_gemm_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constan
       int l, tp, tq;
       decode_item(p, item, l, tp, tq);
       // the outcome must be warp-uniform: the TMEM loads below are warp-collective
-      if (!__all_sync(0xFFFFFFFFu, wait_bounded(smem_u32(&sh->tmem_full), acc_phase, sh, p.status, 0x200 + warp))) break;
+      if (!__all_sync(0xFFFFFFFFu, wait_bounded(smem_u32(&sh->tmem_full), acc_phase, &sh->abort, p.status, 0x200 + warp))) break;
       tc_fence_after();
       Epi::template run<W>(ep, p, tmem, warp - 2, lane, l, tp, tq, smem_u32(&sh->tmem_empty));
       acc_phase ^= 1u;
@@ -616,11 +616,11 @@ residue_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
         if (p.wave_counter) {  // both CTAs of every pair take part: 2 * npairs arrivals per wave
           const long long wave = item / npairs;
           const long long target = 2 * min((wave + 1) * (long long)npairs, (long long)total_items);
-          if (!wave_barrier(p.wave_counter, (unsigned int)target, sh, p.status)) break;
+          if (!wave_barrier(p.wave_counter, (unsigned int)target, &sh->abort, p.status)) break;
         }
         const bool kara = kKara && karatsuba_modulus(l);
         for (int kb = 0; kb < p.kblocks; ++kb) {
-          if (!wait_bounded(smem_u32(&sh->empty[stage]), phase ^ 1u, sh, p.status, 0x300 + stage)) {
+          if (!wait_bounded(smem_u32(&sh->empty[stage]), phase ^ 1u, &sh->abort, p.status, 0x300 + stage)) {
             ok = false;
             break;
           }
@@ -645,7 +645,7 @@ residue_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
           if (++stage == kPairStages) stage = 0, phase ^= 1u;
           if (kara) {
             // second stage of the k block: the sum-limb tiles ps (this CTA's 128 rows) and qs (its 64 rows)
-            if (!wait_bounded(smem_u32(&sh->empty[stage]), phase ^ 1u, sh, p.status, 0x300 + stage)) {
+            if (!wait_bounded(smem_u32(&sh->empty[stage]), phase ^ 1u, &sh->abort, p.status, 0x300 + stage)) {
               ok = false;
               break;
             }
@@ -676,12 +676,12 @@ residue_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
         const bool three = p.skip_top_first && l == 0;
         const bool kara = kKara && karatsuba_modulus(l);
         if (count) clk_a = clock64();
-        if (!wait_bounded(smem_u32(&sh->tmem_empty), acc_phase ^ 1u, sh, p.status, 0x400)) break;
+        if (!wait_bounded(smem_u32(&sh->tmem_empty), acc_phase ^ 1u, &sh->abort, p.status, 0x400)) break;
         if (count) clk_empty += clock64() - clk_a;
         tc_fence_after();
         for (int kb = 0; kb < p.kblocks; ++kb) {
           if (count) clk_a = clock64();
-          if (!wait_bounded(smem_u32(&sh->full[stage]), phase, sh, p.status, 0x410 + stage)) {
+          if (!wait_bounded(smem_u32(&sh->full[stage]), phase, &sh->abort, p.status, 0x410 + stage)) {
             ok = false;
             break;
           }
@@ -701,7 +701,7 @@ residue_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
             mma_commit_pair(smem_u32(&sh->empty[stage]), (uint16_t)3);
             if (++stage == kPairStages) stage = 0, phase ^= 1u;
             if (count) clk_a = clock64();
-            if (!wait_bounded(smem_u32(&sh->full[stage]), phase, sh, p.status, 0x410 + stage)) {
+            if (!wait_bounded(smem_u32(&sh->full[stage]), phase, &sh->abort, p.status, 0x410 + stage)) {
               ok = false;
               break;
             }
@@ -764,7 +764,7 @@ residue_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
     for (int item = pair; item < total_items; item += npairs) {
       int l, tp, tq;
       decode_item(p, item, l, tp, tq);
-      if (!__all_sync(0xFFFFFFFFu, wait_bounded(smem_u32(&sh->tmem_full), acc_phase, sh, p.status, 0x500 + warp))) break;
+      if (!__all_sync(0xFFFFFFFFu, wait_bounded(smem_u32(&sh->tmem_full), acc_phase, &sh->abort, p.status, 0x500 + warp))) break;
       tc_fence_after();
       const uint32_t m = (uint32_t)ep.m[l], recip = ep.recip[l], offset = ep.offset[l];
       uint32_t t[64];
@@ -775,6 +775,230 @@ residue_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
                                             (size_t)tq * W + half * 64);
       reduce_and_store(t, m, recip, dst);
       acc_phase ^= 1u;
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  cluster_arrive();  // neither CTA leaves while the other may still signal its barriers
+  cluster_wait();
+  tc_fence_after();
+  if (warp == 1) {
+    __syncwarp();
+    tmem_dealloc_pair(tmem, kTmemCols);
+  }
+}
+
+// ------------------------------------------------------------------------------------
+// DGEMM path for short K on CTA pairs: the two-accumulator form (see kGammaTileW in ozk_common.cuh).
+//   ab = p0 beta + p1 gamma (mod m):  D_lo = p0 beta0 + p1 gamma0,  D_hi = p0 beta1 + p1 gamma1,  r = (D_lo + 13 D_hi) mod m
+// p0, p1 are the B-matrix limbs (TMEM lanes), beta = the A-matrix residue and gamma = 13 * it, two limbs each, stacked
+// along the TMEM columns: per K step two N = 240 instructions, p0 x [beta0 ; beta1] and p1 x [gamma0 ; gamma1], both
+// into the same 240 columns.  A 256 x 120 tile needs 240 columns, so two accumulator sets fit tensor memory beside the
+// scale-factor columns: the epilogue drains one set while the tensor core fills the other, which hides the turn-around
+// of about 4 k clocks per tile that the three-accumulator kernel above pays (a third of a tile's time at K = 1024).
+// Price: the A side carries four planes per modulus, and a stage holds 62 KiB (three stages).
+// Each CTA loads its own p0, p1 rows, and of the stacked column-side operands the leader keeps beta0 and gamma0, its peer
+// beta1 and gamma1 (120 rows each).
+// ------------------------------------------------------------------------------------
+constexpr int kGW = kGammaTileW;
+constexpr int kGQBytes = kGW * kTileKBytes;                      // one 120-row tile of a column-side plane
+constexpr int kGStageBytes = 2 * kPTileBytes + 2 * kGQBytes;     // p0, p1, this CTA's halves of [beta0 ; beta1] and [gamma0 ; gamma1]
+constexpr int kGStages = 3;
+struct __align__(8) GammaShared {
+  uint64_t full[kGStages];
+  uint64_t empty[kGStages];
+  uint64_t tmem_full[2];   // per accumulator set
+  uint64_t tmem_empty[2];
+  uint64_t drained;
+  uint32_t tmem_base;
+  volatile int abort;
+};
+constexpr size_t kGammaSmemBytes = (size_t)kGStages * kGStageBytes + sizeof(GammaShared) + 1024;
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
+residue_gemm_gamma_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_q,
+                          const __grid_constant__ GemmCore p, const __grid_constant__ ResidueParams ep, int64_t rows_padded) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  GammaShared* sh = reinterpret_cast<GammaShared*>(tiles + kGStages * kGStageBytes);
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+  const int total_items = p.L * p.tiles_p * p.tiles_q;  // tiles_p: 256-wide column tiles, tiles_q: 120-wide row tiles
+
+  if (threadIdx.x == 0) {
+    prefetch_tensormap(&map_p);
+    prefetch_tensormap(&map_q);
+    for (int s = 0; s < kGStages; ++s) {
+      mbar_init(smem_u32(&sh->full[s]), 1);   // used in the leader only
+      mbar_init(smem_u32(&sh->empty[s]), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(smem_u32(&sh->tmem_full[a]), 1);
+      mbar_init(smem_u32(&sh->tmem_empty[a]), 16);  // 8 epilogue warps of each CTA; used in the leader only
+    }
+    mbar_init(smem_u32(&sh->drained), 1);
+    sh->abort = 0;
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(smem_u32(&sh->tmem_base), kTmemCols);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = sh->tmem_base;
+  if (warp >= 2) {
+    const uint32_t quad = (uint32_t)(warp & 3), half = (uint32_t)((warp - 2) >> 2);
+    if (half == 0) {  // constant UE8M0 scale bytes
+      tmem_st_32x8_const(tmem + ((quad * 32u) << 16) + kScaleCol, p.scale_word);
+      tmem_st_32x8_const(tmem + ((quad * 32u) << 16) + kScaleCol + 8, p.scale_word);
+    }
+    tmem_wait_st();
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_arrive();  // the peer's barriers are initialised before anything is sent to them
+  cluster_wait();
+  tc_fence_after();
+
+  if (warp == 0) {
+    // ------------------------------ TMA producer (both CTAs) ------------------------------
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      const uint64_t pol_keep = l2_policy_evict_last(), pol_stream = l2_policy_evict_first();
+      for (int item = pair; item < total_items && ok; item += npairs) {
+        int l, tp, tq;
+        decode_item(p, item, l, tp, tq);
+        if (p.wave_counter) {  // both CTAs of every pair take part: 2 * npairs arrivals per wave
+          const long long wave = item / npairs;
+          const long long target = 2 * min((wave + 1) * (long long)npairs, (long long)total_items);
+          if (!wave_barrier(p.wave_counter, (unsigned int)target, &sh->abort, p.status)) break;
+        }
+        for (int kb = 0; kb < p.kblocks; ++kb) {
+          if (!wait_bounded(smem_u32(&sh->empty[stage]), phase ^ 1u, &sh->abort, p.status, 0x600 + stage)) {
+            ok = false;
+            break;
+          }
+          const uint32_t leader_full = map_to_cta(smem_u32(&sh->full[stage]), 0);
+          const uint32_t dst = smem_u32(tiles + stage * kGStageBytes);
+          if (rank == 0) mbar_arrive_expect_tx(smem_u32(&sh->full[stage]), 2 * kGStageBytes);
+          const int x = kb * kTileKBytes;
+          const int prow = (2 * tp + (int)rank) * kTileRows;
+          tma_load_3d_pair_hint(dst + 0 * kPTileBytes, &map_p, leader_full, x, prow, 2 * l + 0, pol_keep);
+          tma_load_3d_pair_hint(dst + 1 * kPTileBytes, &map_p, leader_full, x, prow, 2 * l + 1, pol_keep);
+          tma_load_3d_pair_hint(dst + 2 * kPTileBytes, &map_q, leader_full, x, tq * kGW, 2 * l + (int)rank, pol_stream);
+          tma_load_3d_pair_hint(dst + 2 * kPTileBytes + kGQBytes, &map_q, leader_full, x, tq * kGW, p.sum_plane_base + 2 * l + (int)rank,
+                                pol_stream);
+          if (++stage == kGStages) stage = 0, phase ^= 1u;
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer (leader only) ------------------------------
+    if (lane == 0 && rank == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      const uint32_t sf = tmem + kScaleCol;
+      constexpr uint32_t kIdesc = idesc_mxf4_pair(2 * kGW);
+      bool ok = true;
+      const bool count = p.count_cycles != 0;
+      long long clk_start = count ? clock64() : 0, clk_empty = 0, clk_full = 0, clk_a = 0;
+      int n = 0;
+      for (int item = pair; item < total_items && ok; item += npairs, ++n) {
+        const int set = n & 1;
+        const uint32_t set_phase = (uint32_t)((n >> 1) & 1);
+        const uint32_t acc = tmem + (uint32_t)(set * 2 * kGW);
+        if (count) clk_a = clock64();
+        if (!wait_bounded(smem_u32(&sh->tmem_empty[set]), set_phase ^ 1u, &sh->abort, p.status, 0x700 + set)) break;
+        if (count) clk_empty += clock64() - clk_a;
+        tc_fence_after();
+        for (int kb = 0; kb < p.kblocks; ++kb) {
+          if (count) clk_a = clock64();
+          if (!wait_bounded(smem_u32(&sh->full[stage]), phase, &sh->abort, p.status, 0x710 + stage)) {
+            ok = false;
+            break;
+          }
+          if (count) clk_full += clock64() - clk_a;
+          tc_fence_after();
+          const uint32_t base = smem_u32(tiles + stage * kGStageBytes);
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks) {
+            mma_mxf4_pair(acc, smem_desc_sw128(base + 0 * kPTileBytes + ks * 32), smem_desc_sw128(base + 2 * kPTileBytes + ks * 32), kIdesc,
+                          sf, sf, (kb == 0 && ks == 0) ? 0u : 1u);
+            mma_mxf4_pair(acc, smem_desc_sw128(base + 1 * kPTileBytes + ks * 32),
+                          smem_desc_sw128(base + 2 * kPTileBytes + kGQBytes + ks * 32), kIdesc, sf, sf, 1u);
+          }
+          mma_commit_pair(smem_u32(&sh->empty[stage]), (uint16_t)3);
+          if (++stage == kGStages) stage = 0, phase ^= 1u;
+        }
+        if (!ok) break;
+        mma_commit_pair(smem_u32(&sh->tmem_full[set]), (uint16_t)3);
+      }
+      if (count && blockIdx.x == 0) {
+        p.status->mma_clk_total = clock64() - clk_start;
+        p.status->mma_clk_wait_tmem = clk_empty;
+        p.status->mma_clk_wait_operands = clk_full;
+      }
+      if (sh->abort) {
+        mma_commit_pair(smem_u32(&sh->drained), (uint16_t)1);
+        const uint64_t t0 = global_timer_ns();
+        while (!mbar_try_wait(smem_u32(&sh->drained), 0u) && global_timer_ns() - t0 < kWaitLimitNs) {
+        }
+      }
+    }
+  } else {
+    // ------------------------------ epilogue (both CTAs) ----------------------------------
+    // warp (quadrant q, half h): lanes 32 q .., columns [0, 64) or [64, 120) of both accumulators, 8 at a time
+    const uint32_t quad = (uint32_t)(warp & 3), half = (uint32_t)((warp - 2) >> 2);
+    const int col0 = half ? 64 : 0, chunks = half ? 7 : 8;
+    const uint32_t lane_base = tmem + ((quad * 32u) << 16) + (uint32_t)col0;
+    int n = 0;
+    for (int item = pair; item < total_items; item += npairs, ++n) {
+      int l, tp, tq;
+      decode_item(p, item, l, tp, tq);
+      const int set = n & 1;
+      const uint32_t set_phase = (uint32_t)((n >> 1) & 1);
+      const uint32_t leader_empty = map_to_cta(smem_u32(&sh->tmem_empty[set]), 0);
+      if (!__all_sync(0xFFFFFFFFu, wait_bounded(smem_u32(&sh->tmem_full[set]), set_phase, &sh->abort, p.status, 0x800 + warp))) break;
+      tc_fence_after();
+      const uint32_t base = lane_base + (uint32_t)(set * 2 * kGW);
+      uint32_t lo[8][8], hi[8][8];
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        if (c < chunks) {
+          tmem_ld_32x8(base + 8 * c, lo[c]);
+          tmem_ld_32x8(base + kGW + 8 * c, hi[c]);
+        }
+      }
+      tmem_wait_ld();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(leader_empty);
+      const uint32_t m = (uint32_t)ep.m[l], recip = ep.recip[l], offset = ep.offset[l];
+      const int64_t j = (int64_t)(2 * tp + (int)rank) * kTileRows + quad * 32 + lane;
+      const int64_t i0 = (int64_t)tq * kGW + col0;
+      uint8_t* dst = ep.res + (size_t)l * ep.res_stride + (size_t)j * (size_t)ep.res_ld + (size_t)i0;
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        if (c < chunks && i0 + 8 * c < rows_padded) {   // the last row tile may reach past the padded rows
+          uint32_t w[2] = {0u, 0u};
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            const uint32_t x = (uint32_t)(__float2int_rn(__uint_as_float(lo[c][e])) + 13 * __float2int_rn(__uint_as_float(hi[c][e]))) + offset;
+            uint32_t r = x - __umulhi(x, recip) * m;  // in [0, 2m)
+            r = min(r, r - m);
+            w[e >> 2] |= r << (8 * (e & 3));
+          }
+          *reinterpret_cast<uint2*>(dst + 8 * c) = make_uint2(w[0], w[1]);
+        }
+      }
     }
   }
 
@@ -1015,6 +1239,45 @@ ozk_status gemm_residues(const Geometry& g, const ModulusTable& mt, uint8_t* ws,
   ep.res = res ? res : ws + g.off_res;
   ep.res_ld = g.Mp;
   ep.res_stride = (size_t)g.Mp * (size_t)g.Np;
+  if (g.gamma && g.Np % 256 == 0 && pair_kernel_enabled()) {
+    // short K: the two-accumulator kernel on CTA pairs (the A side holds beta planes 0 .. 2L-1 and gamma planes 2L .. 4L-1).
+    // Cooperative launch like the pair kernel below, which also serves as its fallback (on the beta planes).
+    GemmCore gc = core;
+    gc.tiles_p = (int)(g.Np / 256);
+    gc.tiles_q = (int)((g.Mp + kGW - 1) / kGW);
+    gc.group = 8;
+    gc.skip_top_first = 0;
+    gc.count_cycles = stage_timing_enabled() ? 1 : 0;
+    gc.sum_plane_base = 2 * g.L;
+    gc.wave_counter = reinterpret_cast<unsigned int*>(ws + g.off_status + 512);
+    CUtensorMap map_q120;
+    if (!make_plane_map(&map_q120, planes_a, klen / 2, g.Mp, planes_of_a(g.L, 0, 1), g.plane_bytes_a, kGW, g.pitch)) return OZK_ERR_CUDA;
+    static std::atomic<bool> attr_set[kMaxDevices];
+    const int dev = current_device_ordinal();
+    if (dev < 0) return OZK_ERR_CUDA;
+    if (!attr_set[dev].load(std::memory_order_acquire)) {
+      if (cudaFuncSetAttribute(residue_gemm_gamma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGammaSmemBytes) != cudaSuccess)
+        return OZK_ERR_CUDA;
+      attr_set[dev].store(true, std::memory_order_release);
+    }
+    const int max_pairs = device_sm_count() / 2;
+    if (max_pairs < 1) return OZK_ERR_CUDA;
+    const long long items = (long long)gc.L * gc.tiles_p * gc.tiles_q;
+    const int pairs = (int)(items < max_pairs ? items : max_pairs);
+    if (cudaMemsetAsync(gc.wave_counter, 0, 4, st) != cudaSuccess) return OZK_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(2 * pairs), 1, 1);
+    cfg.blockDim = dim3(kPairThreads, 1, 1);
+    cfg.dynamicSmemBytes = kGammaSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, residue_gemm_gamma_kernel, map_p, map_q120, gc, ep, (int64_t)g.Mp) == cudaSuccess) return OZK_OK;
+    (void)cudaGetLastError();  // refused: the kernels below run on the beta planes
+  }
   if (g.Np % 256 == 0 && pair_kernel_enabled()) {
     // CTA-pair kernel.  Its producers meet at a global counter before every wave of items, which needs
     // all CTAs resident: the launch is cooperative, and when that is refused the single-CTA kernel runs.

@@ -87,6 +87,7 @@ bool make_host_layout(int64_t M, int64_t N, int64_t K, int L, HostLayout* h) {
   if (h->rblocks > kMaxBlocks || h->cblocks > kMaxBlocks) return false;
   if (!make_geometry(h->mb, h->nb, K, L, &h->g)) return false;
   h->g.karatsuba = 0;  // the host-buffer path keeps the two planes per modulus
+  h->g.gamma = 0;
   const Geometry& g = h->g;
   auto up = [](size_t x) { return (x + 1023) / 1024 * 1024; };
   const size_t kk = (size_t)(K > 0 ? K : 1);

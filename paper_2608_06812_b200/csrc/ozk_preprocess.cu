@@ -84,19 +84,23 @@ __global__ void build_lut_kernel(ModulusTable mt, uint8_t* __restrict__ tables, 
         // a few per cent of the limb GEMM's time under the power cap), then smallest magnitudes
         const int key = 2000 * ((c0 < 0) + (c1 < 0)) + max(a0, a1) * 64 + (a0 + a1);
         const int rho = ((c0 + 13 * c1) % m + m) % m;
-        const int idx = (rho + mt.off62[l]) % m;  // the tables are indexed by the shifted residue
-        atomicMin(&best[idx], (unsigned int)key * 256u + (unsigned int)threadIdx.x);
+        atomicMin(&best[rho], (unsigned int)key * 256u + (unsigned int)threadIdx.x);
       }
     }
   }
   __syncthreads();
+  // the tables are indexed by the shifted residue idx = (rho + 2^62) mod m; the gamma tables hold the pair of 13 rho
   uint8_t* even = tables + (size_t)l * 2 * kLimbTabStride;
   uint8_t* odd = even + kLimbTabStride;
+  uint8_t* even_g = tables + kLimbTabBytes + kEncFragBytes + kEncSumTabBytes + (size_t)l * 2 * kLimbTabStride;
+  uint8_t* odd_g = even_g + kLimbTabStride;
   for (int idx = threadIdx.x; idx < kLimbTabStride; idx += blockDim.x) {
-    const unsigned int pair = idx < m ? best[idx] & 0xFFu : 0u;
-    const unsigned int i0 = pair & 15u, i1 = pair >> 4;
-    even[idx] = (uint8_t)(i0 | (i1 << 4));
-    odd[idx] = (uint8_t)(i1 | (i0 << 4));
+    const int rho = idx < m ? (idx - mt.off62[l] + m) % m : 0;
+    const unsigned int pair = idx < m ? best[rho] & 0xFFu : 0u, pair_g = idx < m ? best[(13 * rho) % m] & 0xFFu : 0u;
+    even[idx] = (uint8_t)((pair & 15u) | ((pair >> 4) << 4));
+    odd[idx] = (uint8_t)((pair >> 4) | ((pair & 15u) << 4));
+    even_g[idx] = (uint8_t)((pair_g & 15u) | ((pair_g >> 4) << 4));
+    odd_g[idx] = (uint8_t)((pair_g >> 4) | ((pair_g & 15u) << 4));
   }
 }
 
@@ -241,8 +245,10 @@ struct EncTables {
   uint8_t limb[kMaxModuli][2][kLimbTabStride];
   uint2 frag[kEncTiles][32];
   uint8_t sum[2][256];
+  uint8_t limb_gamma[kMaxModuli][2][kLimbTabStride];   // copied only by the kernels that write gamma planes
 };
 static_assert(sizeof(EncTables) == kEncTableBytes, "shared copy mirrors the workspace layout");
+template <bool kGamma>
 __device__ __forceinline__ void load_tables(const uint8_t* __restrict__ tables, int L, EncTables* tab) {
   const int limb_vec = L * 2 * kLimbTabStride / 16, frag_vec = (int)((kEncFragBytes + kEncSumTabBytes) / 16);
   const uint4* src = reinterpret_cast<const uint4*>(tables);
@@ -251,11 +257,17 @@ __device__ __forceinline__ void load_tables(const uint8_t* __restrict__ tables, 
   uint4* dst_frag = reinterpret_cast<uint4*>(tab->frag);
   for (int i = threadIdx.x; i < limb_vec; i += blockDim.x) dst[i] = src[i];
   for (int i = threadIdx.x; i < frag_vec; i += blockDim.x) dst_frag[i] = src_frag[i];
+  if constexpr (kGamma) {
+    const uint4* src_g = reinterpret_cast<const uint4*>(tables + kLimbTabBytes + kEncFragBytes + kEncSumTabBytes);
+    uint4* dst_g = reinterpret_cast<uint4*>(tab->limb_gamma);
+    for (int i = threadIdx.x; i < limb_vec; i += blockDim.x) dst_g[i] = src_g[i];
+  }
 }
 
 // Plane words of the thread's eight elements for every modulus, stored at dst + plane * plane_bytes.
 // Warp-collective (all 32 lanes must call it).
-template <bool kKaratsuba>
+// kGamma: also the two planes of 13 a mod m per modulus, at plane index 2 L + 2 l + limb (two-accumulator form, A side).
+template <bool kKaratsuba, bool kGamma>
 __device__ __forceinline__ void encode_planes(const Shifted8& v, int L, const EncTables& tab, uint8_t* dst, size_t plane_bytes) {
   const int lane = threadIdx.x & 31;
 #pragma unroll
@@ -273,11 +285,23 @@ __device__ __forceinline__ void encode_planes(const Shifted8& v, int L, const En
       const uint8_t* even = tab.limb[l][0];
       const uint8_t* odd = tab.limb[l][1];
       uint32_t ea[4], eb[4];  // table bytes of the elements at even / odd k
+      uint32_t ga[kGamma ? 4 : 1], gb[kGamma ? 4 : 1];
 #pragma unroll
       for (int h = 0; h < 4; ++h) {
         const uint32_t t0 = (uint32_t)d[h][mm], t1 = (uint32_t)d[h][2 + mm];
-        ea[h] = even[t0 - __umulhi(t0, recip1) * m];
-        eb[h] = odd[t1 - __umulhi(t1, recip1) * m];
+        const uint32_t r0 = t0 - __umulhi(t0, recip1) * m, r1 = t1 - __umulhi(t1, recip1) * m;
+        ea[h] = even[r0];
+        eb[h] = odd[r1];
+        if constexpr (kGamma) {
+          ga[h] = tab.limb_gamma[l][0][r0];
+          gb[h] = tab.limb_gamma[l][1][r1];
+        }
+      }
+      if constexpr (kGamma) {
+        const uint32_t ya = __byte_perm(__byte_perm(ga[0], ga[1], 0x0040), __byte_perm(ga[2], ga[3], 0x0040), 0x5410);
+        const uint32_t yb = __byte_perm(__byte_perm(gb[0], gb[1], 0x0040), __byte_perm(gb[2], gb[3], 0x0040), 0x5410);
+        *reinterpret_cast<uint32_t*>(dst + (size_t)(2 * L + 2 * l) * plane_bytes) = (ya & 0x0F0F0F0Fu) | (yb & 0xF0F0F0F0u);
+        *reinterpret_cast<uint32_t*>(dst + (size_t)(2 * L + 2 * l + 1) * plane_bytes) = ((ya >> 4) & 0x0F0F0F0Fu) | ((yb << 4) & 0xF0F0F0F0u);
       }
       const uint32_t xa = __byte_perm(__byte_perm(ea[0], ea[1], 0x0040), __byte_perm(ea[2], ea[3], 0x0040), 0x5410);
       const uint32_t xb = __byte_perm(__byte_perm(eb[0], eb[1], 0x0040), __byte_perm(eb[2], eb[3], 0x0040), 0x5410);
@@ -313,7 +337,7 @@ __global__ void __launch_bounds__(256) encode_cols_kernel(const double* __restri
                                                           const int32_t* __restrict__ shifts, uint8_t* __restrict__ planes,
                                                           size_t plane_bytes, size_t pitch, int64_t* __restrict__ int_out, int reps) {
   __shared__ __align__(16) EncTables tab;
-  load_tables(tables, L, &tab);  // copied once per block and reused for `reps` chunks of 2048 k
+  load_tables<false>(tables, L, &tab);  // copied once per block and reused for `reps` chunks of 2048 k
   __syncthreads();
   const int64_t j = blockIdx.x;
   for (int rep = 0; rep < reps; ++rep) {
@@ -346,7 +370,7 @@ __global__ void __launch_bounds__(256) encode_cols_kernel(const double* __restri
     }
     Shifted8 v;
     shift8(a, v);
-    encode_planes<kKaratsuba>(v, L, tab, planes + (size_t)j * pitch + (size_t)(k / 2), plane_bytes);
+    encode_planes<kKaratsuba, false>(v, L, tab, planes + (size_t)j * pitch + (size_t)(k / 2), plane_bytes);
   }
 }
 
@@ -363,7 +387,7 @@ constexpr int kRowTileK = 128;
 constexpr int kGroupStride = 9;                                         // doubles per group of 8 k (8 used)
 constexpr int kRowStride = (kRowTileK / 8) * kGroupStride + 1;          // doubles per row: 145, odd
 
-template <bool kKaratsuba>
+template <bool kKaratsuba, bool kGamma>
 __global__ void __launch_bounds__(256) encode_rows_kernel(const double* __restrict__ A, int64_t lda, int64_t M, int64_t K,
                                                           int64_t Kp, int L, const uint8_t* __restrict__ tables,
                                                           const int32_t* __restrict__ shifts, uint8_t* __restrict__ planes,
@@ -372,7 +396,7 @@ __global__ void __launch_bounds__(256) encode_rows_kernel(const double* __restri
   __shared__ double in_s[kRowTile * kRowStride];
   const int t = threadIdx.x;
   const int64_t i0 = (int64_t)blockIdx.x * kRowTile;
-  load_tables(tables, L, &tab);  // copied once per block and reused for `reps` tiles along k
+  load_tables<kGamma>(tables, L, &tab);  // copied once per block and reused for `reps` tiles along k
   const int r = t >> 4, g = t & 15;  // encode role: row r, k group g
   const int64_t i = i0 + r;
   const ScalePair sc = make_scale(shifts[i]);  // shifts has Mp entries; padded rows hold 0
@@ -403,7 +427,7 @@ __global__ void __launch_bounds__(256) encode_rows_kernel(const double* __restri
     }
     Shifted8 v;
     shift8(a, v);
-    encode_planes<kKaratsuba>(v, L, tab, planes + (size_t)i * pitch + (size_t)(k0 / 2) + 4 * g, plane_bytes);
+    encode_planes<kKaratsuba, kGamma>(v, L, tab, planes + (size_t)i * pitch + (size_t)(k0 / 2) + 4 * g, plane_bytes);
   }
 }
 
@@ -470,7 +494,7 @@ cudaError_t launch_encode_operand(const Geometry& g, const ModulusTable& mt, int
   const int reps = 4;
   if (which == 0) {
     dim3 grid((unsigned)(g.Mp / kRowTile), (unsigned)((g.Kp / kRowTileK + reps - 1) / reps));
-    auto* kernel = g.karatsuba ? encode_rows_kernel<true> : encode_rows_kernel<false>;
+    auto* kernel = g.karatsuba ? encode_rows_kernel<true, false> : (g.gamma ? encode_rows_kernel<false, true> : encode_rows_kernel<false, false>);
     kernel<<<grid, 256, 0, st>>>(X, ldx, g.M, g.K, g.Kp, mt.L, tables, reinterpret_cast<const int32_t*>(ws + g.off_s),
                                              ws + g.off_planes_a, g.plane_bytes_a, g.pitch, int_out, reps);
   } else {

@@ -68,6 +68,19 @@ def test_k_beyond_one_limb_gemm_range_bit_exact(shape):
     assert gu.bits_equal(gu.dgemm(A, B, 19), ozaki2.dgemm(A, B, 19).C)
 
 
+@pytest.mark.parametrize("shape,L", [((384, 512, 700), 19), ((1000, 256, 64), 19), ((130, 768, 768), 27), ((2048, 1024, 512), 19),
+                                     ((121, 256, 1), 12), ((600, 512, 769), 19)])
+def test_short_k_two_accumulator_form_bit_exact(shape, L):
+    """K up to 768 with a column count that pads to a multiple of 256 runs the two-accumulator limb GEMM (row tiles of
+    120, the last one ragged, gamma planes on the A side); K = 769 is the first size on the three-accumulator kernel."""
+    M, N, K = shape
+    A = inputs.lognormal_matrix(M, K, 1.0, seed=50)
+    B = inputs.lognormal_matrix(K, N, 1.0, seed=51)
+    A[0, :] = np.abs(A[0, :])
+    B[:, 0] = np.abs(B[:, 0])
+    assert gu.bits_equal(gu.dgemm(A, B, L), ozaki2.dgemm(A, B, L).C)
+
+
 def test_more_than_65535_columns():
     """N beyond the y-dimension limit of a CUDA grid: the O(N^2) kernels loop over the columns.  Small integers
     make C the exact integer product, so the whole matrix is checked against an int64 product."""

@@ -63,6 +63,24 @@ def test_preprocess_matches_oracle(shape, L, phi):
             assert np.all((c0 + 13 * c1 - X) % mods[l] == 0)
 
 
+def test_gamma_planes_of_the_two_accumulator_form():
+    """Short K on CTA pairs (column count a multiple of 256): the A side also carries the limb planes of 13 a mod m
+    (planes 3 and 4 of ozk_stage_read_planes), with which a b = a0 beta + a1 gamma needs two accumulators only."""
+    M, N, K, L = 130, 256, 300, 19
+    A = inputs.lognormal_matrix(M, K, 1.0, seed=0)
+    B = inputs.lognormal_matrix(K, N, 1.0, seed=1)
+    s, t, At, Bt = run_preprocess(A, B, L)
+    mods = moduli.select_moduli(L)
+    for l in (0, 1, 7, 18):
+        g0 = read_plane("A", M, N, K, L, l, 3)
+        g1 = read_plane("A", M, N, K, L, l, 4)
+        assert np.isin(g0, base13.S).all() and np.isin(g1, base13.S).all()
+        assert max(np.abs(g0).max(), np.abs(g1).max()) <= 8
+        assert np.all((g0 + 13 * g1 - 13 * At) % mods[l] == 0)
+    out = torch.zeros((K, N), dtype=torch.int8, device="cuda")
+    assert ozk.ozk_stage_read_planes("B", M, N, K, L, 0, 3, out.data_ptr(), gu.stream()) == ozk.OZK_ERR_INVALID_ARG
+
+
 def test_subnormal_and_extreme_rows():
     A = np.array([[2.0 ** -1074, 3 * 2.0 ** -1074, 0.0, -(2.0 ** -1070)],
                   [1.7e308, -1e300, 1e-300, 5e307],
