@@ -72,7 +72,10 @@ const char* ozk_version(void);
 /* Bytes of device workspace ozk_dgemm(M,N,K,...,num_moduli) needs: status block, limb-pair
  * tables, shifts s (rows of A) and t (columns of B), 2*num_moduli E2M1 limb planes per
  * operand padded to 128 rows x 256 k, and num_moduli residue matrices of one byte per
- * element of the padded C.  Returns 0 on invalid arguments. */
+ * element of the padded C.  For 0 < K <= 768 with N padding to a multiple of 256 the A side
+ * holds two more planes per modulus (the limbs of 13 a mod m, see the two-accumulator form
+ * under ozk_stage_residue_gemm); with the Karatsuba variant on, one sum-limb plane per Karatsuba
+ * modulus and operand.  Returns 0 on invalid arguments. */
 size_t ozk_dgemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int num_moduli);
 
 /* Bytes of device workspace ozk_igemm_i8(M,N,K,...) needs (3 limb planes per operand). */
@@ -194,13 +197,23 @@ ozk_status ozk_stage_preprocess(int64_t M, int64_t N, int64_t K,
 /* Decodes limb plane (modulus index l, limb 0|1) of operand 'A' or 'B' from the workspace
  * into doubled-E2M1 integers (int8, values in S): out[r + k*rows], r < rows (M for 'A',
  * N for 'B'), k < K.  Valid after ozk_stage_preprocess / ozk_dgemm on the same sizes.
- * limb = 2 reads the sum-limb plane of a Karatsuba modulus (variant on, see ozk_stage_set_karatsuba). */
+ * limb = 2 reads the sum-limb plane of a Karatsuba modulus (variant on, see ozk_stage_set_karatsuba).
+ * limb = 3 | 4 (operand 'A' only, sizes that take the two-accumulator form) reads limb 0 | 1 of
+ * (13 a) mod m_l, the planes that form multiplies by the high limbs of B. */
 ozk_status ozk_stage_read_planes(char operand, int64_t M, int64_t N, int64_t K, int num_moduli,
                                  int l, int limb, int8_t* out, void* stream);
 
 /* Stage 2 (Section 5.1, Section 6.4): the limb GEMM with residue composition, on the
  * planes in the workspace.  residues_out (optional, device): num_moduli matrices of
- * M x N bytes, column-major with ld = M, r_l = (A~ B~) mod m_l in [0, m_l). */
+ * M x N bytes, column-major with ld = M, r_l = (A~ B~) mod m_l in [0, m_l).
+ * Two forms of the same residues (bit for bit).  Regular: b = b0 + 13 b1, a = a0 + 13 a1,
+ * three accumulators a0 b0, a0 b1 + a1 b0, a1 b1 per tile of C.  Two-accumulator form, taken
+ * for 0 < K <= 768 when N pads to a multiple of 256: a b = b0 beta + b1 gamma (mod m) with
+ * beta = a mod m and gamma = 13 a mod m, both as limb pairs, so that only the accumulators
+ * b0 beta_0 + b1 gamma_0 and b0 beta_1 + b1 gamma_1 exist and two tiles of C fit tensor memory
+ * at once: the read-back of one overlaps the products of the next (faster at short K, slower
+ * from K = 1024 on because the A side moves twice the planes).  OZK_GEMM_GAMMA=0 in the
+ * environment keeps the regular form at every K (measurement aid, read once per process). */
 ozk_status ozk_stage_residue_gemm(int64_t M, int64_t N, int64_t K, int num_moduli,
                                   uint8_t* residues_out, void* stream);
 
