@@ -72,7 +72,7 @@ const char* ozk_version(void);
 /* Bytes of device workspace ozk_dgemm(M,N,K,...,num_moduli) needs: status block, limb-pair
  * tables, shifts s (rows of A) and t (columns of B), 2*num_moduli E2M1 limb planes per
  * operand padded to 128 rows x 256 k, and num_moduli residue matrices of one byte per
- * element of the padded C.  For 0 < K <= 768 with N padding to a multiple of 256 the A side
+ * element of the padded C.  For 0 < K <= 1792 with N padding to a multiple of 256 the A side
  * holds two more planes per modulus (the limbs of 13 a mod m, see the two-accumulator form
  * under ozk_stage_residue_gemm); with the Karatsuba variant on, one sum-limb plane per Karatsuba
  * modulus and operand.  Returns 0 on invalid arguments. */
@@ -208,11 +208,11 @@ ozk_status ozk_stage_read_planes(char operand, int64_t M, int64_t N, int64_t K, 
  * M x N bytes, column-major with ld = M, r_l = (A~ B~) mod m_l in [0, m_l).
  * Two forms of the same residues (bit for bit).  Regular: b = b0 + 13 b1, a = a0 + 13 a1,
  * three accumulators a0 b0, a0 b1 + a1 b0, a1 b1 per tile of C.  Two-accumulator form, taken
- * for 0 < K <= 768 when N pads to a multiple of 256: a b = b0 beta + b1 gamma (mod m) with
+ * for 0 < K <= 1792 when N pads to a multiple of 256: a b = b0 beta + b1 gamma (mod m) with
  * beta = a mod m and gamma = 13 a mod m, both as limb pairs, so that only the accumulators
  * b0 beta_0 + b1 gamma_0 and b0 beta_1 + b1 gamma_1 exist and two tiles of C fit tensor memory
- * at once: the read-back of one overlaps the products of the next (faster at short K, slower
- * from K = 1024 on because the A side moves twice the planes).  OZK_GEMM_GAMMA=0 in the
+ * at once: the read-back of one overlaps the products of the next (faster at short K, level
+ * with the regular form at K = 2048 and slower beyond, because the A side moves twice the planes).  OZK_GEMM_GAMMA=0 in the
  * environment keeps the regular form at every K (measurement aid, read once per process). */
 ozk_status ozk_stage_residue_gemm(int64_t M, int64_t N, int64_t K, int num_moduli,
                                   uint8_t* residues_out, void* stream);

@@ -76,7 +76,7 @@ static inline int planes_per_operand(int L, int karatsuba) { return 2 * L + (kar
 // needs two accumulators of W columns instead of three; with W = 120 two sets fit tensor memory and the read-back of one
 // tile overlaps the products of the next.  The A-matrix side carries beta (its regular planes) and gamma (2 L more).
 constexpr int kGammaTileW = 120;
-constexpr int64_t kGammaMaxK = 768;    // longest K that takes this form: measured faster up to here, slower from 1024 on (more operand traffic)
+constexpr int64_t kGammaMaxK = 1792;   // longest K that takes this form: measured faster up to here, level at 2048, slower beyond (more operand traffic)
 static inline int planes_of_a(int L, int karatsuba, int gamma) { return planes_per_operand(L, karatsuba) + (gamma ? 2 * L : 0); }
 
 // ---- per-modulus constants handed to kernels by value --------------------------------

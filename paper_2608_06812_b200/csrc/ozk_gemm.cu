@@ -110,6 +110,36 @@ __device__ __forceinline__ bool wave_barrier(unsigned int* counter, unsigned int
   }
 }
 
+// The same counter used for pacing only, in the two-accumulator kernel whose tiles are short: a producer announces each
+// item and goes on as soon as the counter has reached `target`, which the caller sets to the arrivals of the wave before
+// the previous one.  `seen` is the newest value this producer knows; wave_counter_probe() reads the counter without
+// waiting for the answer (it is looked at one item later), so that in step no producer ever polls.
+__device__ __forceinline__ unsigned int wave_counter_probe(const unsigned int* counter) {
+  unsigned int v;
+  asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
+  return v;
+}
+__device__ __forceinline__ bool wave_barrier_lagged(unsigned int* counter, unsigned int target, unsigned int& seen, volatile int* abort,
+                                                    StatusBlock* status) {
+  atomicAdd(counter, 1u);
+  if (seen >= target) return true;
+  const uint64_t t0 = global_timer_ns();
+  for (uint32_t it = 0;; ++it) {
+    seen = wave_counter_probe(counter);
+    if (seen >= target) return true;
+    __nanosleep(64);
+    if ((it & 63u) == 63u) {
+      if (*abort) return false;
+      if (global_timer_ns() - t0 > kWaitLimitNs) {
+        *abort = 1;
+        atomicMin(&status->code, (int)OZK_ERR_DEVICE_TIMEOUT);
+        atomicExch(&status->where, 0x701);
+        return false;
+      }
+    }
+  }
+}
+
 __device__ __forceinline__ void decode_item(const GemmCore& p, int item, int& l, int& tp, int& tq) {
   const int per_group = p.tiles_p * p.tiles_q;
   l = item / per_group;
@@ -121,6 +151,39 @@ __device__ __forceinline__ void decode_item(const GemmCore& p, int item, int& l,
   tq = rem / gsize;
   tp = g * p.group + (rem - tq * gsize);
 }
+
+// Walks the items item, item + step, ... of one CTA pair in the order of decode_item without a division per item.
+struct ItemCursor {
+  int l, g, rem;           // modulus, band of column tiles, position inside the band (tq * gsize + column tile of the band)
+  int gsize, band_items;   // column tiles and items of this band
+  uint32_t inv_gsize;      // ceil(2^32 / gsize): rem / gsize by one multiply-high (rem < 2^29)
+  __device__ __forceinline__ void set_band(const GemmCore& p) {
+    gsize = min(p.group, p.tiles_p - g * p.group);
+    band_items = gsize * p.tiles_q;
+    inv_gsize = gsize > 1 ? 0xFFFFFFFFu / (uint32_t)gsize + 1u : 0u;
+  }
+  __device__ __forceinline__ void init(const GemmCore& p, int item) {
+    const int per_group = p.tiles_p * p.tiles_q;
+    l = item / per_group;
+    const int t = item - l * per_group;
+    const int band = p.group * p.tiles_q;
+    g = t / band;
+    rem = t - g * band;
+    set_band(p);
+  }
+  __device__ __forceinline__ void advance(const GemmCore& p, int step) {
+    rem += step;
+    while (rem >= band_items) {
+      rem -= band_items;
+      if (++g * p.group >= p.tiles_p) g = 0, ++l;
+      set_band(p);
+    }
+  }
+  __device__ __forceinline__ void tile(const GemmCore& p, int& tp, int& tq) const {
+    tq = gsize > 1 ? (int)__umulhi((uint32_t)rem, inv_gsize) : rem;
+    tp = g * p.group + (rem - tq * gsize);
+  }
+};
 
 
 // Drains the three accumulators of 64 columns (lanes of this warp's quadrant) and hands tensor memory
@@ -802,6 +865,7 @@ residue_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
 // beta1 and gamma1 (120 rows each).
 // ------------------------------------------------------------------------------------
 constexpr int kGW = kGammaTileW;
+static_assert(14 * 128 * kGammaMaxK < (1 << 22), "the epilogue holds D_lo + 13 D_hi plus an offset above 2^22 in 23 bits");
 constexpr int kGQBytes = kGW * kTileKBytes;                      // one 120-row tile of a column-side plane
 constexpr int kGStageBytes = 2 * kPTileBytes + 2 * kGQBytes;     // p0, p1, this CTA's halves of [beta0 ; beta1] and [gamma0 ; gamma1]
 constexpr int kGStages = 3;
@@ -810,18 +874,21 @@ struct __align__(8) GammaShared {
   uint64_t empty[kGStages];
   uint64_t tmem_full[2];   // per accumulator set
   uint64_t tmem_empty[2];
+  uint64_t staged[2];      // per output buffer: the 8 epilogue warps have written their residues
   uint64_t drained;
   uint32_t tmem_base;
   volatile int abort;
 };
-constexpr size_t kGammaSmemBytes = (size_t)kGStages * kGStageBytes + sizeof(GammaShared) + 1024;
+constexpr int kGOutBytes = kTileRows * kGW;  // residues of one CTA's 128 columns x 120 rows, one byte each
+constexpr size_t kGammaSmemBytes = (size_t)kGStages * kGStageBytes + 2 * kGOutBytes + sizeof(GammaShared) + 1024;
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
 residue_gemm_gamma_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_q,
                           const __grid_constant__ GemmCore p, const __grid_constant__ ResidueParams ep, int64_t rows_padded) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  GammaShared* sh = reinterpret_cast<GammaShared*>(tiles + kGStages * kGStageBytes);
+  uint8_t* out_stage = tiles + kGStages * kGStageBytes;  // two buffers of kGOutBytes
+  GammaShared* sh = reinterpret_cast<GammaShared*>(out_stage + 2 * kGOutBytes);
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
@@ -838,6 +905,7 @@ residue_gemm_gamma_kernel(const __grid_constant__ CUtensorMap map_p, const __gri
     for (int a = 0; a < 2; ++a) {
       mbar_init(smem_u32(&sh->tmem_full[a]), 1);
       mbar_init(smem_u32(&sh->tmem_empty[a]), 16);  // 8 epilogue warps of each CTA; used in the leader only
+      mbar_init(smem_u32(&sh->staged[a]), 8);
     }
     mbar_init(smem_u32(&sh->drained), 1);
     sh->abort = 0;
@@ -873,13 +941,22 @@ residue_gemm_gamma_kernel(const __grid_constant__ CUtensorMap map_p, const __gri
       uint32_t phase = 0;
       bool ok = true;
       const uint64_t pol_keep = l2_policy_evict_last(), pol_stream = l2_policy_evict_first();
-      for (int item = pair; item < total_items && ok; item += npairs) {
-        int l, tp, tq;
-        decode_item(p, item, l, tp, tq);
-        if (p.wave_counter) {  // both CTAs of every pair take part: 2 * npairs arrivals per wave
-          const long long wave = item / npairs;
-          const long long target = 2 * min((wave + 1) * (long long)npairs, (long long)total_items);
-          if (!wave_barrier(p.wave_counter, (unsigned int)target, &sh->abort, p.status)) break;
+      unsigned int seen = 0, probe = 0;  // the wave counter as last known, and as read during the previous item
+      ItemCursor cur;
+      cur.init(p, pair);
+      int wave = 0;
+      for (int item = pair; item < total_items && ok; item += npairs, ++wave, cur.advance(p, npairs)) {
+        const int l = cur.l;
+        int tp, tq;
+        cur.tile(p, tp, tq);
+        if (p.wave_counter) {
+          // Both CTAs of every pair announce each item (2 * npairs arrivals per wave) and wait for the arrivals of the
+          // wave before the previous one: the pairs stay within three tiles of each other (the planes of a modulus stay in L2
+          // at these K), and no round trip to the counter is paid per tile.
+          if (probe > seen) seen = probe;
+          const long long target = wave >= 2 ? 2 * min((long long)(wave - 1) * npairs, (long long)total_items) : 0;
+          if (!wave_barrier_lagged(p.wave_counter, (unsigned int)target, seen, &sh->abort, p.status)) break;
+          probe = wave_counter_probe(p.wave_counter);
         }
         for (int kb = 0; kb < p.kblocks; ++kb) {
           if (!wait_bounded(smem_u32(&sh->empty[stage]), phase ^ 1u, &sh->abort, p.status, 0x600 + stage)) {
@@ -891,11 +968,8 @@ residue_gemm_gamma_kernel(const __grid_constant__ CUtensorMap map_p, const __gri
           if (rank == 0) mbar_arrive_expect_tx(smem_u32(&sh->full[stage]), 2 * kGStageBytes);
           const int x = kb * kTileKBytes;
           const int prow = (2 * tp + (int)rank) * kTileRows;
-          tma_load_3d_pair_hint(dst + 0 * kPTileBytes, &map_p, leader_full, x, prow, 2 * l + 0, pol_keep);
-          tma_load_3d_pair_hint(dst + 1 * kPTileBytes, &map_p, leader_full, x, prow, 2 * l + 1, pol_keep);
-          tma_load_3d_pair_hint(dst + 2 * kPTileBytes, &map_q, leader_full, x, tq * kGW, 2 * l + (int)rank, pol_stream);
-          tma_load_3d_pair_hint(dst + 2 * kPTileBytes + kGQBytes, &map_q, leader_full, x, tq * kGW, p.sum_plane_base + 2 * l + (int)rank,
-                                pol_stream);
+          tma_load_3d_pair_hint(dst, &map_p, leader_full, x, prow, 2 * l, pol_keep);                           // p0, p1
+          tma_load_4d_pair_hint(dst + 2 * kPTileBytes, &map_q, leader_full, x, tq * kGW, 2 * l + (int)rank, 0, pol_stream);  // beta, gamma
           if (++stage == kGStages) stage = 0, phase ^= 1u;
         }
       }
@@ -907,6 +981,7 @@ residue_gemm_gamma_kernel(const __grid_constant__ CUtensorMap map_p, const __gri
       uint32_t phase = 0;
       const uint32_t sf = tmem + kScaleCol;
       constexpr uint32_t kIdesc = idesc_mxf4_pair(2 * kGW);
+
       bool ok = true;
       const bool count = p.count_cycles != 0;
       long long clk_start = count ? clock64() : 0, clk_empty = 0, clk_full = 0, clk_a = 0;
@@ -955,18 +1030,38 @@ residue_gemm_gamma_kernel(const __grid_constant__ CUtensorMap map_p, const __gri
     }
   } else {
     // ------------------------------ epilogue (both CTAs) ----------------------------------
-    // warp (quadrant q, half h): lanes 32 q .., columns [0, 64) or [64, 120) of both accumulators, 8 at a time
+    // warp (quadrant q, half h): lanes 32 q .., columns [0, 64) or [64, 120) of both accumulators, 8 at a time.
+    // The residues cross shared memory so that they leave as whole rows: a thread's 64 or 56 bytes (column j of C, rows
+    // col0 ..) go into row quad * 32 + lane of an output buffer (120-byte pitch: the 8-byte writes of a warp fall on 16
+    // distinct bank pairs), and each warp writes 16 of the 128 rows to memory, 30 lanes x 4 bytes = one 120-byte run of a
+    // residue column per instruction (stored from the registers, a warp's store would touch 32 lines with 8 bytes each).
+    // Two buffers: the rows of the previous tile are written out between the arithmetic of the current one, two rows
+    // per chunk, so the store queue never holds the warp up.
     const uint32_t quad = (uint32_t)(warp & 3), half = (uint32_t)((warp - 2) >> 2);
     const int col0 = half ? 64 : 0, chunks = half ? 7 : 8;
     const uint32_t lane_base = tmem + ((quad * 32u) << 16) + (uint32_t)col0;
+    const int row0 = (warp - 2) * 16;  // the rows of an output buffer this warp writes to memory
+    const uint32_t out_base = smem_u32(out_stage);
+    const uint32_t out_mine = (quad * 32u + (uint32_t)lane) * (uint32_t)kGW + (uint32_t)col0;
+    const uint32_t out_rows = (uint32_t)(row0 * kGW + 4 * lane);
+    constexpr uint32_t kInsert[4] = {0x3214u, 0x3240u, 0x3410u, 0x4210u};
+    const float kOneTiny = __uint_as_float(1u), kThirteenTiny = __uint_as_float(13u);  // 2^-149 and 13 * 2^-149
+    uint8_t* prev_dst = nullptr;  // where this warp's rows of the previous tile go; null: nothing pending (or beyond the rows)
+    bool ok = true;
     int n = 0;
-    for (int item = pair; item < total_items; item += npairs, ++n) {
-      int l, tp, tq;
-      decode_item(p, item, l, tp, tq);
+    ItemCursor cur;
+    cur.init(p, pair);
+    for (int item = pair; item < total_items; item += npairs, ++n, cur.advance(p, npairs)) {
+      const int l = cur.l;
+      int tp, tq;
+      cur.tile(p, tp, tq);
       const int set = n & 1;
       const uint32_t set_phase = (uint32_t)((n >> 1) & 1);
       const uint32_t leader_empty = map_to_cta(smem_u32(&sh->tmem_empty[set]), 0);
-      if (!__all_sync(0xFFFFFFFFu, wait_bounded(smem_u32(&sh->tmem_full[set]), set_phase, &sh->abort, p.status, 0x800 + warp))) break;
+      if (!__all_sync(0xFFFFFFFFu, wait_bounded(smem_u32(&sh->tmem_full[set]), set_phase, &sh->abort, p.status, 0x800 + warp))) {
+        ok = false;
+        break;
+      }
       tc_fence_after();
       const uint32_t base = lane_base + (uint32_t)(set * 2 * kGW);
       uint32_t lo[8][8], hi[8][8];
@@ -981,22 +1076,55 @@ residue_gemm_gamma_kernel(const __grid_constant__ CUtensorMap map_p, const __gri
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(leader_empty);
-      const uint32_t m = (uint32_t)ep.m[l], recip = ep.recip[l], offset = ep.offset[l];
-      const int64_t j = (int64_t)(2 * tp + (int)rank) * kTileRows + quad * 32 + lane;
-      const int64_t i0 = (int64_t)tq * kGW + col0;
-      uint8_t* dst = ep.res + (size_t)l * ep.res_stride + (size_t)j * (size_t)ep.res_ld + (size_t)i0;
+      // every warp has put the previous tile into the other buffer, and has finished reading this one (the tile before that)
+      if (n > 0 && !__all_sync(0xFFFFFFFFu, wait_bounded(smem_u32(&sh->staged[set ^ 1]), (uint32_t)(((n - 1) >> 1) & 1), &sh->abort,
+                                                          p.status, 0x900 + warp))) {
+        ok = false;
+        break;
+      }
+      // |D_lo + 13 D_hi| <= 14 * 128 K < 2^22 for K <= kGammaMaxK; offset: the multiple of m just above 2^22
+      const uint32_t m = (uint32_t)ep.m[l], recip1 = ep.recip[l] + 1u;
+      const float offset_tiny = __uint_as_float(m * ((1u << 22) / m + 1u));  // as a subnormal: bit pattern = integer
+      const uint32_t out_cur = out_base + (uint32_t)(set * kGOutBytes), out_prev = out_base + (uint32_t)((set ^ 1) * kGOutBytes);
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
-        if (c < chunks && i0 + 8 * c < rows_padded) {   // the last row tile may reach past the padded rows
+        if (c < chunks) {
           uint32_t w[2] = {0u, 0u};
 #pragma unroll
           for (int e = 0; e < 8; ++e) {
-            const uint32_t x = (uint32_t)(__float2int_rn(__uint_as_float(lo[c][e])) + 13 * __float2int_rn(__uint_as_float(hi[c][e]))) + offset;
-            uint32_t r = x - __umulhi(x, recip) * m;  // in [0, 2m)
-            r = min(r, r - m);
-            w[e >> 2] |= r << (8 * (e & 3));
+            // y = D_lo + 13 D_hi + offset < 2^23, formed as y * 2^-149: the bit pattern of that subnormal is the integer
+            // y itself (both multiply-adds are exact), so no conversion is needed
+            const uint32_t y = __float_as_uint(fmaf(__uint_as_float(hi[c][e]), kThirteenTiny, fmaf(__uint_as_float(lo[c][e]), kOneTiny, offset_tiny)));
+            const uint32_t r = y - __umulhi(y, recip1) * m;  // exact for y < 2^24: recip1 = floor(2^32 / m) + 1
+            w[e >> 2] = e & 3 ? __byte_perm(w[e >> 2], r, kInsert[e & 3]) : r;
           }
-          *reinterpret_cast<uint2*>(dst + 8 * c) = make_uint2(w[0], w[1]);
+          asm volatile("st.shared.v2.u32 [%0], {%1, %2};" ::"r"(out_cur + out_mine + 8u * c), "r"(w[0]), "r"(w[1]) : "memory");
+        }
+        if (prev_dst) {  // rows 2 c and 2 c + 1 of the previous tile
+          uint32_t v0, v1;
+          asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v0) : "r"(out_prev + out_rows + (uint32_t)(2 * c * kGW)) : "memory");
+          asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v1) : "r"(out_prev + out_rows + (uint32_t)((2 * c + 1) * kGW)) : "memory");
+          *reinterpret_cast<uint32_t*>(prev_dst + (size_t)(2 * c) * (size_t)ep.res_ld) = v0;
+          *reinterpret_cast<uint32_t*>(prev_dst + (size_t)(2 * c + 1) * (size_t)ep.res_ld) = v1;
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&sh->staged[set]));
+      const int64_t i = (int64_t)tq * kGW + 4 * lane;  // the last row tile may reach past the padded rows
+      prev_dst = (lane < kGW / 4 && i < rows_padded)
+                     ? ep.res + (size_t)l * ep.res_stride + (size_t)((int64_t)(2 * tp + (int)rank) * kTileRows + row0) * (size_t)ep.res_ld + (size_t)i
+                     : nullptr;
+    }
+    if (ok && n > 0) {  // the rows of the last tile
+      const int set = (n - 1) & 1;
+      if (__all_sync(0xFFFFFFFFu, wait_bounded(smem_u32(&sh->staged[set]), (uint32_t)(((n - 1) >> 1) & 1), &sh->abort, p.status, 0x900 + warp)) &&
+          prev_dst) {
+        const uint32_t src = out_base + (uint32_t)(set * kGOutBytes) + out_rows;
+#pragma unroll
+        for (int r = 0; r < 16; ++r) {
+          uint32_t v;
+          asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(src + (uint32_t)(r * kGW)) : "memory");
+          *reinterpret_cast<uint32_t*>(prev_dst + (size_t)r * (size_t)ep.res_ld) = v;
         }
       }
     }
@@ -1134,17 +1262,30 @@ EncodeTiledFn encode_tiled_fn() {
 // Planes of one operand as a (bytes along K, rows, plane) byte tensor; box = 128 bytes x box_rows.
 // Rows of a box that fall outside the tensor are filled with zero bytes (E2M1 code 0 = value 0).
 bool make_plane_map(CUtensorMap* map, const void* base, int64_t k_bytes, int64_t rows, int64_t planes, size_t plane_bytes,
-                    int box_rows, size_t pitch = 0) {
+                    int box_rows, size_t pitch = 0, int box_planes = 1) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return false;
   cuuint64_t dims[3] = {(cuuint64_t)k_bytes, (cuuint64_t)rows, (cuuint64_t)planes};
   cuuint64_t strides[2] = {(cuuint64_t)(pitch ? pitch : (size_t)k_bytes), (cuuint64_t)plane_bytes};
-  cuuint32_t box[3] = {(cuuint32_t)kTileKBytes, (cuuint32_t)box_rows, 1};
+  cuuint32_t box[3] = {(cuuint32_t)kTileKBytes, (cuuint32_t)box_rows, (cuuint32_t)box_planes};
   cuuint32_t estr[3] = {1, 1, 1};
   const int rank = planes > 0 ? 3 : 2;
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, rank, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// A-side planes of the two-accumulator form as a (bytes along K, rows, plane, kind) tensor: kind 0 = the 2 L limb planes
+// of beta, kind 1 = those of gamma, which follow them.  A box takes 120 rows of one plane of both kinds.
+bool make_gamma_q_map(CUtensorMap* map, const void* base, int64_t k_bytes, int64_t rows, int L, size_t plane_bytes, size_t pitch) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  cuuint64_t dims[4] = {(cuuint64_t)k_bytes, (cuuint64_t)rows, (cuuint64_t)(2 * L), 2};
+  cuuint64_t strides[3] = {(cuuint64_t)pitch, (cuuint64_t)plane_bytes, (cuuint64_t)plane_bytes * (cuuint64_t)(2 * L)};
+  cuuint32_t box[4] = {(cuuint32_t)kTileKBytes, (cuuint32_t)kGammaTileW, 1, 2};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 // cudaFuncSetAttribute acts on the current device only: remember per device ordinal where it has been done.
@@ -1250,8 +1391,9 @@ ozk_status gemm_residues(const Geometry& g, const ModulusTable& mt, uint8_t* ws,
     gc.count_cycles = stage_timing_enabled() ? 1 : 0;
     gc.sum_plane_base = 2 * g.L;
     gc.wave_counter = reinterpret_cast<unsigned int*>(ws + g.off_status + 512);
-    CUtensorMap map_q120;
-    if (!make_plane_map(&map_q120, planes_a, klen / 2, g.Mp, planes_of_a(g.L, 0, 1), g.plane_bytes_a, kGW, g.pitch)) return OZK_ERR_CUDA;
+    CUtensorMap map_p2, map_q120;  // one copy brings p0 and p1, another this CTA's limb of beta and of gamma
+    if (!make_plane_map(&map_p2, planes_b, klen / 2, g.Np, planes, g.plane_bytes_b, kTileRows, g.pitch, 2)) return OZK_ERR_CUDA;
+    if (!make_gamma_q_map(&map_q120, planes_a, klen / 2, g.Mp, g.L, g.plane_bytes_a, g.pitch)) return OZK_ERR_CUDA;
     static std::atomic<bool> attr_set[kMaxDevices];
     const int dev = current_device_ordinal();
     if (dev < 0) return OZK_ERR_CUDA;
@@ -1264,7 +1406,7 @@ ozk_status gemm_residues(const Geometry& g, const ModulusTable& mt, uint8_t* ws,
     if (max_pairs < 1) return OZK_ERR_CUDA;
     const long long items = (long long)gc.L * gc.tiles_p * gc.tiles_q;
     const int pairs = (int)(items < max_pairs ? items : max_pairs);
-    if (cudaMemsetAsync(gc.wave_counter, 0, 4, st) != cudaSuccess) return OZK_ERR_CUDA;
+    if (gc.wave_counter && cudaMemsetAsync(gc.wave_counter, 0, 4, st) != cudaSuccess) return OZK_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(2 * pairs), 1, 1);
     cfg.blockDim = dim3(kPairThreads, 1, 1);
@@ -1275,7 +1417,7 @@ ozk_status gemm_residues(const Geometry& g, const ModulusTable& mt, uint8_t* ws,
     attr[0].val.cooperative = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, residue_gemm_gamma_kernel, map_p, map_q120, gc, ep, (int64_t)g.Mp) == cudaSuccess) return OZK_OK;
+    if (cudaLaunchKernelEx(&cfg, residue_gemm_gamma_kernel, map_p2, map_q120, gc, ep, (int64_t)g.Mp) == cudaSuccess) return OZK_OK;
     (void)cudaGetLastError();  // refused: the kernels below run on the beta planes
   }
   if (g.Np % 256 == 0 && pair_kernel_enabled()) {

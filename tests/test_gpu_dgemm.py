@@ -69,10 +69,12 @@ def test_k_beyond_one_limb_gemm_range_bit_exact(shape):
 
 
 @pytest.mark.parametrize("shape,L", [((384, 512, 700), 19), ((1000, 256, 64), 19), ((130, 768, 768), 27), ((2048, 1024, 512), 19),
-                                     ((121, 256, 1), 12), ((600, 512, 769), 19)])
+                                     ((121, 256, 1), 12), ((600, 512, 1024), 19), ((250, 256, 1792), 19), ((250, 256, 1793), 19),
+                                     ((9000, 512, 300), 16)])
 def test_short_k_two_accumulator_form_bit_exact(shape, L):
-    """K up to 768 with a column count that pads to a multiple of 256 runs the two-accumulator limb GEMM (row tiles of
-    120, the last one ragged, gamma planes on the A side); K = 769 is the first size on the three-accumulator kernel."""
+    """K up to 1792 with a column count that pads to a multiple of 256 runs the two-accumulator limb GEMM (row tiles of
+    120, the last one ragged, gamma planes on the A side, residues staged through shared memory, more tiles than CTA
+    pairs in the 9000-row case); K = 1793 is the first size on the three-accumulator kernel."""
     M, N, K = shape
     A = inputs.lognormal_matrix(M, K, 1.0, seed=50)
     B = inputs.lognormal_matrix(K, N, 1.0, seed=51)

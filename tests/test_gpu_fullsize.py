@@ -92,24 +92,26 @@ def x_words_by_stages(n, L, dA, dB):
 
 def freivalds_on_device(n, L, A, B, dX):
     """The same identity with the 192-bit words left on the device (dX[j, i, 6], int32): x v = At (Bt v) modulo two
-    31-bit primes.  At, Bt come from the CPU oracle; torch int64 arithmetic on the GPU is test infrastructure."""
-    c = moduli.capacity_bits(n, L)
+    31-bit primes.  At, Bt come from the CPU oracle; torch int64 arithmetic on the GPU is test infrastructure.
+    A is M x K, B is K x N (n is the square size of the callers above and is not used for the extents)."""
+    (M, K), N = A.shape, B.shape[1]
+    c = moduli.capacity_bits(K, L)
     dAt = torch.from_numpy(ozaki2.to_integers(A, ozaki2.shared_shifts(A, 1, c), 1)).cuda()     # [i, k]
     dBt = torch.from_numpy(ozaki2.to_integers(B, ozaki2.shared_shifts(B, 0, c), 0)).cuda()     # [k, j]
     gen = torch.Generator(device="cuda")
     gen.manual_seed(99)
     step = 512
     for q in (2147483647, 2147483629):
-        v = torch.randint(0, q, (n,), dtype=torch.int64, device="cuda", generator=gen)
-        Bv = torch.zeros(n, dtype=torch.int64, device="cuda")
-        for j0 in range(0, n, step):                          # every product is reduced (< 2^31) before the sum
+        v = torch.randint(0, q, (N,), dtype=torch.int64, device="cuda", generator=gen)
+        Bv = torch.zeros(K, dtype=torch.int64, device="cuda")
+        for j0 in range(0, N, step):                          # every product is reduced (< 2^31) before the sum
             Bv = (Bv + ((dBt[:, j0:j0 + step] % q) * v[None, j0:j0 + step] % q).sum(dim=1)) % q
-        right = torch.zeros(n, dtype=torch.int64, device="cuda")
-        for k0 in range(0, n, step):
+        right = torch.zeros(M, dtype=torch.int64, device="cuda")
+        for k0 in range(0, K, step):
             right = (right + ((dAt[:, k0:k0 + step] % q) * Bv[None, k0:k0 + step] % q).sum(dim=1)) % q
         pw = [pow(2, 32 * k, q) for k in range(6)]
-        left = torch.zeros(n, dtype=torch.int64, device="cuda")
-        for j0 in range(0, n, step):
+        left = torch.zeros(M, dtype=torch.int64, device="cuda")
+        for j0 in range(0, N, step):
             W = dX[j0:j0 + step].to(torch.int64) & 0xFFFFFFFF                                   # [j, i, 6]
             xm = torch.zeros(W.shape[:2], dtype=torch.int64, device="cuda")
             for k in range(6):
@@ -204,3 +206,32 @@ def test_config5_16384_headline_configuration():
     Cs = dC[torch.from_numpy(jj).cuda(), torch.from_numpy(ii).cuda()].cpu().numpy()
     want = np.array([ozaki2.round_scaled_to_double(words_to_int(Xs[k]), int(s_ref[ii[k]]) + int(t_ref[jj[k]])) for k in range(ii.size)])
     assert gu.bits_equal(Cs, want)
+
+
+@pytest.mark.parametrize("M,N,K", [(8192, 8192, 1024), (16384, 4096, 512)])
+def test_short_k_whole_matrix(M, N, K):
+    """Short K at full width (the two-accumulator limb GEMM: row tiles of 120 with a ragged last one, many more tiles
+    than CTA pairs, residues staged through shared memory): every reconstructed integer by the Freivalds identity,
+    a 128 x 128 block plus scattered rows and columns of C against the oracle bit for bit, staged calls = ozk_dgemm."""
+    L = 19
+    A = inputs.lognormal_matrix(M, K, 1.0, seed=0)
+    B = inputs.lognormal_matrix(K, N, 1.0, seed=1)
+    dA = torch.from_numpy(np.ascontiguousarray(A.T)).cuda()
+    dB = torch.from_numpy(np.ascontiguousarray(B.T)).cuda()
+    gu.ensure_workspace(ozk.ozk_dgemm_workspace_bytes(M, N, K, L))
+    dC = torch.empty((N, M), dtype=torch.float64, device="cuda")
+    ozk.check(ozk.ozk_dgemm(M, N, K, dA.data_ptr(), M, dB.data_ptr(), K, dC.data_ptr(), M, L, gu.stream()), "ozk_dgemm")
+    ozk.check(ozk.ozk_get_async_status(gu.stream()), "status")
+    rng = np.random.default_rng(8)
+    rows = np.concatenate([np.arange(128), np.sort(rng.choice(np.arange(128, M), 40, replace=False)), np.arange(M - 24, M)])
+    cols = np.concatenate([np.arange(128), np.sort(rng.choice(np.arange(128, N), 40, replace=False)), np.arange(N - 24, N)])
+    check_samples(A, B, dC, L, rows, cols)
+    dX = torch.empty((N, M, 6), dtype=torch.int32, device="cuda")
+    dC2 = torch.empty((N, M), dtype=torch.float64, device="cuda")
+    ozk.check(ozk.ozk_stage_preprocess(M, N, K, dA.data_ptr(), M, dB.data_ptr(), K, L, None, None, None, None, gu.stream()),
+              "ozk_stage_preprocess")
+    ozk.check(ozk.ozk_stage_residue_gemm(M, N, K, L, None, gu.stream()), "ozk_stage_residue_gemm")
+    ozk.check(ozk.ozk_stage_crt(M, N, K, L, None, None, None, dC2.data_ptr(), M, dX.data_ptr(), gu.stream()), "ozk_stage_crt")
+    ozk.check(ozk.ozk_get_async_status(gu.stream()), "status")
+    assert torch.equal(dC2.view(torch.int64), dC.view(torch.int64))
+    freivalds_on_device(0, L, A, B, dX)

@@ -21,11 +21,11 @@ def karatsuba_on():
 
 
 def test_workspace_grows_by_the_sum_limb_planes():
-    on = ozk.ozk_dgemm_workspace_bytes(1024, 1024, 1024, 19)
+    on = ozk.ozk_dgemm_workspace_bytes(1024, 1024, 2048, 19)            # K beyond the two-accumulator form, which has planes of its own
     ozk.ozk_stage_set_karatsuba(False)
-    off = ozk.ozk_dgemm_workspace_bytes(1024, 1024, 1024, 19)
+    off = ozk.ozk_dgemm_workspace_bytes(1024, 1024, 2048, 19)
     ozk.ozk_stage_set_karatsuba(True)
-    assert on - off == 7 * 2 * 1024 * 512                               # seven more planes of 1024 x 1024 nibbles per operand
+    assert on - off == 7 * 2 * 1024 * 1024                              # seven more planes of 1024 x 2048 nibbles per operand
     assert ozk.ozk_dgemm_workspace_bytes(64, 64, 64, 11) == (ozk.ozk_stage_set_karatsuba(False), ozk.ozk_dgemm_workspace_bytes(64, 64, 64, 11),
                                                              ozk.ozk_stage_set_karatsuba(True))[1]   # no Karatsuba modulus among the first 11
 
