@@ -199,6 +199,25 @@ __device__ __forceinline__ void drain_and_release(uint32_t base, int W, int mode
                                                   bool release_remote, int lane, uint32_t (&t)[64]) {
   const bool top = mode != 0;
   uint32_t u[kFast ? 64 : 1];
+  if constexpr (kFast && !kKara) {
+    // 16 columns of each accumulator at a time; the loads of the next chunk are in flight while this chunk's
+    // multiply-adds run (a wait covers every load issued before it, so it sits between the two)
+    uint32_t d1[2][16], d2[2][16];
+    auto issue = [&](int c) {
+      tmem_ld_32x16(base + 1 * W + c * 16, d1[c & 1]);
+      if (top) tmem_ld_32x16(base + 2 * W + c * 16, d2[c & 1]);
+      tmem_ld_32x16(base + 0 * W + c * 16, *reinterpret_cast<uint32_t(*)[16]>(&t[c * 16]));  // raw FP32 bits until after the release
+    };
+    issue(0);
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      tmem_wait_ld();
+      if (c < 3) issue(c + 1);
+#pragma unroll
+      for (int e = 0; e < 16; ++e)
+        u[c * 16 + e] = top ? __float_as_uint(fmaf(__uint_as_float(d2[c & 1][e]), 13.0f, __uint_as_float(d1[c & 1][e]))) : d1[c & 1][e];
+    }
+  } else
 #pragma unroll
   for (int c = 0; c < 2; ++c) {
     uint32_t d1[32], d2[32];
