@@ -188,6 +188,30 @@ __global__ void finalize_shifts_kernel(const unsigned long long* __restrict__ am
   shifts[i] = s;
 }
 
+// The same for both operands in one launch: the maxima of A's rows and of B's columns lie back to back (Mp, then Np
+// entries).
+__global__ void finalize_shifts_pair_kernel(const unsigned long long* __restrict__ amax, int64_t m, int64_t m_pad, int64_t n, int64_t n_pad,
+                                            int c_bits, int32_t* __restrict__ shifts_a, int32_t* __restrict__ shifts_b,
+                                            StatusBlock* __restrict__ status) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= m_pad + n_pad) return;
+  const bool live = i < m_pad ? i < m : i - m_pad < n;
+  int32_t s = 0;
+  if (live) {
+    const unsigned long long b = amax[i];
+    if (b != 0) {
+      const int E = (int)(b >> 52);
+      if (E == 0x7FF) {
+        atomicMin(&status->code, (int)OZK_ERR_NONFINITE);
+      } else {
+        const int e = E ? E - 1023 : (63 - __clzll((long long)b)) - 1074;
+        s = c_bits - 1 - e;
+      }
+    }
+  }
+  if (i < m_pad) shifts_a[i] = s; else shifts_b[i - m_pad] = s;
+}
+
 // ------------------------------------------------------------------------------------
 // Residues and limb codes of eight consecutive-k integers per thread, all moduli (Section 5.1), with the
 // residue contraction on the tensor cores.
@@ -479,11 +503,29 @@ cudaError_t launch_scan_operand(const Geometry& g, int which, const double* X, i
   return cudaGetLastError();
 }
 
+// Both operands: one clearing of the two (adjacent) arrays of maxima, the two scans, one kernel for all shifts.
 cudaError_t launch_scan_and_shifts(const Geometry& g, const double* A, int64_t lda, const double* B, int64_t ldb,
                                    uint8_t* ws, cudaStream_t st) {
-  cudaError_t e = launch_scan_operand(g, 0, A, lda, ws, st);
+  auto* status = reinterpret_cast<StatusBlock*>(ws + g.off_status);
+  auto* amax_a = reinterpret_cast<unsigned long long*>(ws + g.off_amax_a);
+  auto* amax_b = reinterpret_cast<unsigned long long*>(ws + g.off_amax_b);
+  if (g.off_amax_b != g.off_amax_a + (size_t)g.Mp * sizeof(unsigned long long)) {  // not laid out back to back: one operand at a time
+    cudaError_t e = launch_scan_operand(g, 0, A, lda, ws, st);
+    if (e != cudaSuccess) return e;
+    return launch_scan_operand(g, 1, B, ldb, ws, st);
+  }
+  cudaError_t e = cudaMemsetAsync(amax_a, 0, (size_t)(g.Mp + g.Np) * sizeof(unsigned long long), st);
   if (e != cudaSuccess) return e;
-  return launch_scan_operand(g, 1, B, ldb, ws, st);
+  if (g.K > 0) {
+    const int kslab_a = 64, kslab_b = 8192;
+    scan_rows_kernel<<<dim3((unsigned)((g.M + 255) / 256), (unsigned)((g.K + kslab_a - 1) / kslab_a)), 256, 0, st>>>(A, lda, g.M, g.K, kslab_a,
+                                                                                                                  amax_a);
+    scan_cols_kernel<<<dim3((unsigned)g.N, (unsigned)((g.K + kslab_b - 1) / kslab_b)), 256, 0, st>>>(B, ldb, g.K, kslab_b, amax_b);
+  }
+  finalize_shifts_pair_kernel<<<(unsigned)((g.Mp + g.Np + 255) / 256), 256, 0, st>>>(amax_a, g.M, g.Mp, g.N, g.Np, g.c_bits,
+                                                                                     reinterpret_cast<int32_t*>(ws + g.off_s),
+                                                                                     reinterpret_cast<int32_t*>(ws + g.off_t), status);
+  return cudaGetLastError();
 }
 
 // Limb planes of A (which = 0, rows of A) or of B (which = 1, columns of B).
@@ -491,7 +533,11 @@ cudaError_t launch_encode_operand(const Geometry& g, const ModulusTable& mt, int
                                   uint8_t* ws, int64_t* int_out, cudaStream_t st) {
   const uint8_t* tables = ws + g.off_lut;
   if (!enc_moduli_match(mt)) return cudaErrorInvalidValue;  // the kernels carry the modulus list as constants
-  const int reps = 4;
+  // tiles along k per block: four when there is enough work for several waves of blocks, fewer for small operands
+  const int64_t k_units = which == 0 ? g.Kp / kRowTileK : (g.Kp + 2047) / 2048;
+  const int64_t row_units = which == 0 ? g.Mp / kRowTile : g.Np;
+  int reps = 4;
+  while (reps > 1 && row_units * ((k_units + reps - 1) / reps) < 6 * (int64_t)device_sm_count()) reps >>= 1;
   if (which == 0) {
     dim3 grid((unsigned)(g.Mp / kRowTile), (unsigned)((g.Kp / kRowTileK + reps - 1) / reps));
     auto* kernel = g.karatsuba ? encode_rows_kernel<true, false> : (g.gamma ? encode_rows_kernel<false, true> : encode_rows_kernel<false, false>);
