@@ -38,7 +38,7 @@ SM_COUNT = 148
 # kernel source it was taken from; a capture of other source is not reported
 TRAFFIC_FILE = os.path.join(ROOT, "profiles", "limb_gemm_dram_traffic.json")
 GEMM_SOURCES = ["paper_2608_06812_b200/csrc/ozk_gemm.cu", "paper_2608_06812_b200/csrc/ozk_ptx.cuh"]
-KERNELS_PER_STEP = 9   # lut, scan_rows, scan_cols, 2 x finalize, encode_rows, encode_cols, limb GEMM, CRT
+KERNELS_PER_STEP = 8   # lut, scan_rows, scan_cols, shifts of both operands, encode_rows, encode_cols, limb GEMM, CRT
 
 
 def parse_args():
@@ -417,6 +417,10 @@ def run_ozk(args, rank: int, local_rank: int, world: int) -> None:
     # both limb-GEMM kernels skip the 13^2 term of modulus 169: executed = required = 4L - 1 products
     pair = ((N + 127) // 128 * 128) % 256 == 0 and os.environ.get("OZK_GEMM_PAIR", "1") != "0"
     executed = 4 * L - 1 if ozk.ozk_get_moduli(L)[0] == 169 else 4 * L
+    # K up to 1792 takes the two-accumulator kernel (b0 beta + b1 gamma: four products for every modulus)
+    gamma = pair and not args.karatsuba and 0 < K <= 1792 and os.environ.get("OZK_GEMM_GAMMA", "1") != "0"
+    if gamma:
+        executed = 4 * L
     if args.karatsuba and pair:
         executed -= sum(1 for l in range(L) if l == 11 or l >= 13)      # three products for the Karatsuba moduli
     fp4_flops_exec = 2.0 * executed * M * N * K
@@ -436,7 +440,8 @@ def run_ozk(args, rank: int, local_rank: int, world: int) -> None:
                      "sm_mhz": clocks["sm_mhz"], "gemm_ms_x_sm_mhz": gemm_ms * clocks["sm_mhz"],
                      "issue_thread": {"clocks": clk_total, "waiting_for_tensor_memory": clk_tmem, "waiting_for_operands": clk_operands,
                                       "issuing_frac": (1.0 - (clk_tmem + clk_operands) / clk_total) if clk_total > 0 else None}}
-    roofline = {"bound": "tensor", "kernel": "residue_gemm_pair_kernel" if pair else "limb_gemm_kernel", "achieved": achieved,
+    roofline = {"bound": "tensor", "kernel": "residue_gemm_gamma_kernel" if gamma else ("residue_gemm_pair_kernel" if pair else "limb_gemm_kernel"),
+                "achieved": achieved,
                 "peak": NOMINAL_FP4_TFLOPS, "unit": "TFLOP/s", "frac": achieved / NOMINAL_FP4_TFLOPS, "traffic": traffic,
                 "traffic_source": traffic_note,
                 "peak_source": "nominal dense FP4 of B200 (no FP4 peak is measured on this pool; the measured BF16 proxies follow)",
