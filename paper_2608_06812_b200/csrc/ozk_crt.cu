@@ -190,7 +190,8 @@ __device__ __forceinline__ double reconstruct_lean(const unsigned long long (&ac
   const uint32_t h3 = ct.halfP[3];
   bool over = x3 > h3;
   if (x3 == h3) {
-    uint32_t u0, u1, u2, u3, bw;
+    [[maybe_unused]] uint32_t u0, u1, u2, u3;  // only the borrow is wanted
+    uint32_t bw;
     asm("sub.cc.u32 %0, %5, %9;\n\tsubc.cc.u32 %1, %6, %10;\n\tsubc.cc.u32 %2, %7, %11;\n\tsubc.cc.u32 %3, %8, %12;\n\tsubc.u32 %4, 0, 0;"
         : "=r"(u0), "=r"(u1), "=r"(u2), "=r"(u3), "=r"(bw)
         : "r"(ct.halfP[0]), "r"(ct.halfP[1]), "r"(ct.halfP[2]), "r"(h3), "r"(x0), "r"(x1), "r"(x2), "r"(x3));
@@ -268,7 +269,8 @@ __device__ __forceinline__ double reconstruct_lean5(const unsigned long long (&a
       "subc.u32 %4, %9, %14;"
       : "=r"(e0), "=r"(e1), "=r"(e2), "=r"(e3), "=r"(e4)
       : "r"(P0), "r"(P1), "r"(P2), "r"(P3), "r"(P4), "r"(x0), "r"(x1), "r"(x2), "r"(x3), "r"(x4));
-  uint32_t u0, u1, u2, u3, u4, over;  // halfP - x borrows exactly when x > P/2
+  [[maybe_unused]] uint32_t u0, u1, u2, u3, u4;
+  uint32_t over;  // halfP - x borrows exactly when x > P/2
   asm("sub.cc.u32 %0, %6, %11;\n\t"
       "subc.cc.u32 %1, %7, %12;\n\t"
       "subc.cc.u32 %2, %8, %13;\n\t"
@@ -395,9 +397,6 @@ __device__ __forceinline__ unsigned long long mad_wide(uint32_t a, uint32_t b, u
 }
 __device__ __forceinline__ void sts64(uint32_t addr, unsigned long long v) {
   asm volatile("st.shared.u64 [%0], %1;" ::"r"(addr), "l"(v) : "memory");
-}
-__device__ __forceinline__ void lds128x4(uint32_t addr, uint32_t (&w)[4]) {
-  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(addr) : "memory");
 }
 __device__ __forceinline__ void lds128(uint32_t addr, unsigned long long& a, unsigned long long& b) {
   asm volatile("ld.shared.v2.u64 {%0, %1}, [%2];" : "=l"(a), "=l"(b) : "r"(addr) : "memory");

@@ -83,6 +83,16 @@ def test_short_k_two_accumulator_form_bit_exact(shape, L):
     assert gu.bits_equal(gu.dgemm(A, B, L), ozaki2.dgemm(A, B, L).C)
 
 
+@pytest.mark.parametrize("L", list(range(2, 28)))
+def test_every_moduli_count_on_cta_pairs(L):
+    """256 columns put the product on CTA pairs: K = 200 on the two-accumulator kernel, K = 1900 on the three-accumulator
+    one, for every moduli count the library accepts (the small shapes elsewhere run the single-CTA kernel)."""
+    for K, seed in ((200, 60), (1900, 62)):
+        A = inputs.lognormal_matrix(136, K, 0.5, seed=seed)
+        B = inputs.lognormal_matrix(K, 256, 0.5, seed=seed + 1)
+        assert gu.bits_equal(gu.dgemm(A, B, L), ozaki2.dgemm(A, B, L).C), f"K = {K}"
+
+
 def test_more_than_65535_columns():
     """N beyond the y-dimension limit of a CUDA grid: the O(N^2) kernels loop over the columns.  Small integers
     make C the exact integer product, so the whole matrix is checked against an int64 product."""
