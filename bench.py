@@ -436,7 +436,10 @@ def run_ozk(args, rank: int, local_rank: int, world: int) -> None:
         mac_per_clk_sm = fp4_flops_exec / 2.0 / k_ranges / (SM_COUNT * gemm_ms / k_ranges * 1e-3 * clocks["sm_mhz"] * 1e6)
         nominal_mac = NOMINAL_FP4_TFLOPS * 1e12 / 2.0 / (SM_COUNT * clocks["sm_max_mhz"] * 1e6)
         clk_total, clk_tmem, clk_operands = gemm_cycles
+        # 16384 multiply-adds per SM and clock is what the tensor pipe does when ncu shows it 100 % active (calibrated on a
+        # capture with K = 16384 tiles: 14 876 per clock at 91.3 % sm__pipe_tensor_cycles_active, see profiles/)
         per_cycle = {"mac_per_clk_per_sm": mac_per_clk_sm, "nominal_mac_per_clk_per_sm": nominal_mac, "frac": mac_per_clk_sm / nominal_mac,
+                     "pipe_mac_per_clk_per_sm": 16384, "frac_of_pipe": mac_per_clk_sm / 16384.0,
                      "sm_mhz": clocks["sm_mhz"], "gemm_ms_x_sm_mhz": gemm_ms * clocks["sm_mhz"],
                      "issue_thread": {"clocks": clk_total, "waiting_for_tensor_memory": clk_tmem, "waiting_for_operands": clk_operands,
                                       "issuing_frac": (1.0 - (clk_tmem + clk_operands) / clk_total) if clk_total > 0 else None}}
