@@ -148,16 +148,19 @@ __device__ __forceinline__ double round_scaled_fast(const uint32_t (&mag)[NW], i
 }
 
 
-// Lean reconstruction for 2^100 <= P < 2^126 (16 to 19 moduli): the weighted sum S (up to 137 bits)
+// Lean reconstruction for 2^84 <= P < 2^126 (13 to 19 moduli): the weighted sum S (up to 137 bits)
 // arrives as four 64-bit column sums acc[k] (weight 2^(32 k), no carries yet).
 //   q  = ((S >> (p_bits - 21)) * q_mul) >> 52 is the true quotient floor(S / P) or one below it.  The 32 bits
-//        of S it needs come from the two top column sums alone: the carries left out are worth less than
-//        2^98 < P / 4 and only lower the estimate, which keeps it in {floor(S / P) - 1, floor(S / P)}.
+//        of S it needs come from the top column sums alone (from bit 96 up for P >= 2^116, where what is left out is
+//        below 2^98 < P / 2^18; otherwise from bit 64 up with the carry out of the second sum, leaving out less than
+//        2^66 < P / 2^18), which only lowers the estimate and keeps it in {floor(S / P) - 1, floor(S / P)}
+//        (checked against big integers for every moduli count from 13 to 23, extreme residues included).
 //   x  = S - q P in [0, 2P) is formed column by column as acc[k] + q n_k with n = 2^128 - P (one wide
 //        multiply-add per word, then a single carry pass), modulo 2^128.
 //   The two comparisons (x >= P, x > P / 2) look at the top word first; the full comparison runs only when
 //   the top words are equal.  The rounding builds the FP64 bit pattern from the top three words directly;
-//   magnitudes below 2^96 and results outside the normal range take the general routine.
+//   a magnitude below 2^96 is moved one word up first; below 2^64, and results outside the normal range, take the
+//   general routine.
 __device__ __forceinline__ double reconstruct_lean(const unsigned long long (&acc)[4], const CrtTable& ct, int shift) {
   const uint32_t a3l = (uint32_t)acc[3], a3h = (uint32_t)(acc[3] >> 32), a2h = (uint32_t)(acc[2] >> 32);
   uint32_t t_lo, t_hi;
@@ -200,11 +203,16 @@ __device__ __forceinline__ double reconstruct_lean(const unsigned long long (&ac
   uint32_t e0, e1, e2, e3;
   asm("sub.cc.u32 %0, %4, %8;\n\tsubc.cc.u32 %1, %5, %9;\n\tsubc.cc.u32 %2, %6, %10;\n\tsubc.u32 %3, %7, %11;"
       : "=r"(e0), "=r"(e1), "=r"(e2), "=r"(e3) : "r"(P0), "r"(P1), "r"(P2), "r"(P3), "r"(x0), "r"(x1), "r"(x2), "r"(x3));
-  const uint32_t m0 = over ? e0 : x0, m1 = over ? e1 : x1, m2 = over ? e2 : x2, m3 = over ? e3 : x3;
+  uint32_t m0 = over ? e0 : x0, m1 = over ? e1 : x1, m2 = over ? e2 : x2, m3 = over ? e3 : x3;
+  int top_bit = 127 + 1022;
+  if (m3 == 0u) {  // a magnitude below 2^96 (usual with 16 or 17 moduli, or after cancellation): one word up
+    m3 = m2, m2 = m1, m1 = m0, m0 = 0u;
+    top_bit -= 32;
+  }
   const int lz = __clz(m3);
-  const int e_biased = 127 + 1022 - lz - shift;  // exponent field minus one
-  if (m3 == 0u || (unsigned)e_biased >= 2046u) {
-    const uint32_t mag[4] = {m0, m1, m2, m3};
+  const int e_biased = top_bit - lz - shift;  // exponent field minus one
+  if (m3 == 0u || (unsigned)e_biased >= 2046u) {  // below 2^64, or a result outside the normal range: general routine
+    const uint32_t mag[4] = {over ? e0 : x0, over ? e1 : x1, over ? e2 : x2, over ? e3 : x3};
     const double r = round_scaled_fast<4>(mag, shift);
     return over ? -r : r;
   }
@@ -600,7 +608,7 @@ cudaError_t launch_crt(const Geometry& g, const CrtTable& ct, const uint8_t* res
     const int64_t cap = (int64_t)device_sm_count() * (ww <= 4 ? 3 : 4);
     const unsigned grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>((units + wpb - 1) / wpb, cap));
     const int nhi = ct.L <= 16 ? 0 : ct.L <= 20 ? 1 : ct.L <= 24 ? 2 : 3;
-    const bool lean = ct.words <= 5 && ww <= 4 && ct.p_bits >= 101 && ct.p_bits <= 126;   // 16 to 19 moduli
+    const bool lean = ct.words <= 5 && ww <= 4 && ct.p_bits >= 85 && ct.p_bits <= 126;    // 13 to 19 moduli
     const bool lean5 = ct.words <= 6 && ww <= 5 && ct.p_bits >= 129 && ct.p_bits <= 158;  // 20 to 23 moduli
 #define OZK_CRT_MMA(NT, NHI, WW, NW, LEAN)                                                                           \
   crt_mma_kernel<NT, NHI, WW, NW, LEAN><<<grid, kCrtWarps(NT) * 32, 0, st>>>(ct, res, (size_t)res_ld, res_stride, s, t, g.M, g.N, rows16, C, ldc)

@@ -264,7 +264,7 @@ bool build_crt_table(int L, CrtTable* t) {
   t->inv_P = 1.0 / big_to_double(P);
   t->p_bits = big_bits(P);
   t->q_mul = 0, t->q_word = 0, t->q_bit = 0;
-  if (t->p_bits >= 100 && t->p_bits <= 160) {
+  if (t->p_bits >= 85 && t->p_bits <= 160) {
     // largest c with c P 2^28 <= 2^(52 + shift) (2^28 - 1), by bisection
     const int shift = t->p_bits - 21;
     const Big rhs = big_shl(big_from((1ull << 28) - 1), 52 + shift);

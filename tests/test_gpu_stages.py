@@ -129,7 +129,7 @@ def words_to_int(words: np.ndarray) -> int:
 
 
 @pytest.mark.parametrize("fast", [False, True])
-@pytest.mark.parametrize("L", [2, 9, 12, 14, 16, 17, 18, 19, 20, 21, 22, 23, 24, 27])
+@pytest.mark.parametrize("L", [2, 9, 12, 13, 14, 15, 16, 17, 18, 19, 20, 21, 22, 23, 24, 27])
 def test_crt_stage_matches_oracle_on_arbitrary_residues(L, fast):
     """fast=False: one element per thread, with the reconstructed integers exported; fast=True: the
     tensor-core kernel the full pipeline uses (row count a multiple of 16: one full block of 128 rows and a
