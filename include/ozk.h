@@ -75,7 +75,8 @@ const char* ozk_version(void);
  * element of the padded C.  For 0 < K <= 1792 with N padding to a multiple of 256 the A side
  * holds two more planes per modulus (the limbs of 13 a mod m, see the two-accumulator form
  * under ozk_stage_residue_gemm); with the Karatsuba variant on, one sum-limb plane per Karatsuba
- * modulus and operand.  Returns 0 on invalid arguments. */
+ * modulus and operand.  The size is therefore not monotonic in K (K = 1792 needs more than K = 2048): a caller that
+ * reuses one workspace for several shapes registers the largest of their sizes.  Returns 0 on invalid arguments. */
 size_t ozk_dgemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int num_moduli);
 
 /* Bytes of device workspace ozk_igemm_i8(M,N,K,...) needs (3 limb planes per operand). */
