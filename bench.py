@@ -477,6 +477,25 @@ def run_ozk(args, rank: int, local_rank: int, world: int) -> None:
             del x
         except Exception as exc:                          # out of memory on small boxes: context is optional
             line["native_fp64_tflops_context"] = f"unavailable: {type(exc).__name__}"
+    if not args.no_fp64_context and world == 1:
+        # the limb GEMM's own rate when the operands do not toggle (A = 0: every A-side nibble is zero), the counterpart of the
+        # paper's single-kernel rate R (Section 7.4): what the same launch does when the 1 kW power cap does not bind
+        try:
+            dZ = torch.zeros_like(dA)
+            for _ in range(2):
+                ozk.check(ozk.ozk_dgemm(M, N, K, dZ.data_ptr(), M, dB.data_ptr(), K, dC.data_ptr(), M, L, stream), "ozk_dgemm")
+            torch.cuda.synchronize()
+            ozk.ozk_stage_timing_read()
+            for _ in range(2):
+                ozk.check(ozk.ozk_dgemm(M, N, K, dZ.data_ptr(), M, dB.data_ptr(), K, dC.data_ptr(), M, L, stream), "ozk_dgemm")
+            torch.cuda.synchronize()
+            own_ms = float(ozk.ozk_stage_timing_read()[1])
+            own = fp4_flops_exec / (own_ms * 1e-3) / 1e12
+            line["roofline"]["own_kernel_constant_operands"] = {"ms_per_launch": own_ms, "tflops": own, "frac_of_nominal": own / NOMINAL_FP4_TFLOPS,
+                                                                "achieved_over_this": achieved / own}
+            del dZ
+        except Exception as exc:
+            line["roofline"]["own_kernel_constant_operands"] = f"unavailable: {type(exc).__name__}"
     if not args.no_cpu_baseline and world == 1:            # the oracle leg runs on rank 0 of a single-GPU run only
         tf, secs, sample, threads = oracle_sample_tflops(A, B, L, 512)
         line["cpu_baseline"] = {"value": tf, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample, "seconds": secs,
