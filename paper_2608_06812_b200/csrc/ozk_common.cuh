@@ -98,7 +98,7 @@ struct CrtTable {
   uint32_t w[kMaxModuli][kCrtWords];       // w_l little endian
   uint32_t P[kCrtWords];
   uint32_t halfP[kCrtWords];               // floor(P / 2)
-  uint32_t negP[4];                        // 2^128 - P (used when P < 2^128)
+  uint32_t negP[5];                        // 2^128 - P for P < 2^128 (four words), else 2^160 - P (five words)
   double inv_P;                            // 1 / P rounded to double
   int p_bits;                              // bit length of P
   // Integer quotient estimate of the carry-chain tails (P of at least 2^100, at most 2047 for floor(S / P)):

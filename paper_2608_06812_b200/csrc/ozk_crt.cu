@@ -227,48 +227,60 @@ __device__ __forceinline__ double reconstruct_lean(const unsigned long long (&ac
   return __hiloint2double((int)hi, (int)lo);
 }
 
-// The same for 2^128 <= P < 2^158 (20 to 23 moduli): S has six words and arrives as five 64-bit column sums,
-// the quotient estimate is the same multiply-high on the 32 bits of S from bit p_bits - 21 on, x has five words.
+// The same for 2^128 <= P < 2^158 (20 to 24 moduli): five 64-bit column sums, x = S - q P has five words and is formed
+// modulo 2^160 as acc[k] + q n_k with n = 2^160 - P.  The 32 bits of S for the quotient estimate come from bit 96 up
+// (the two top column sums and the high half of the third, carries from below left out: they are worth less than
+// 2^98 < P / 2^30); checked against big integers for 20 to 24 moduli.
 __device__ __forceinline__ double reconstruct_lean5(const unsigned long long (&acc)[5], const CrtTable& ct, int shift) {
-  const uint32_t a0l = (uint32_t)acc[0], a0h = (uint32_t)(acc[0] >> 32), a1l = (uint32_t)acc[1], a1h = (uint32_t)(acc[1] >> 32);
-  const uint32_t a2l = (uint32_t)acc[2], a2h = (uint32_t)(acc[2] >> 32), a3l = (uint32_t)acc[3], a3h = (uint32_t)(acc[3] >> 32);
-  const uint32_t a4l = (uint32_t)acc[4], a4h = (uint32_t)(acc[4] >> 32);
-  uint32_t S1, S2, S3, S4, S5;
-  asm("add.cc.u32 %0, %5, %6;\n\t"
-      "addc.cc.u32 %1, %7, %8;\n\t"
-      "addc.cc.u32 %2, %9, %10;\n\t"
-      "addc.cc.u32 %3, %11, %12;\n\t"
-      "addc.u32 %4, %13, 0;"
-      : "=r"(S1), "=r"(S2), "=r"(S3), "=r"(S4), "=r"(S5)
-      : "r"(a0h), "r"(a1l), "r"(a1h), "r"(a2l), "r"(a2h), "r"(a3l), "r"(a3h), "r"(a4l), "r"(a4h));
-  const uint32_t S0 = a0l;
-  const uint32_t top = ct.q_word == 4 ? __funnelshift_r(S4, S5, ct.q_bit) : __funnelshift_r(S3, S4, ct.q_bit);
+  uint32_t w3, t_lo, t_hi;  // S >> 96, approximately: w3 = word 3, t = words 4 and 5
+  asm("add.cc.u32 %0, %3, %4;\n\t"
+      "addc.cc.u32 %1, %5, %6;\n\t"
+      "addc.u32 %2, %7, 0;"
+      : "=r"(w3), "=r"(t_lo), "=r"(t_hi)
+      : "r"((uint32_t)acc[3]), "r"((uint32_t)(acc[2] >> 32)), "r"((uint32_t)acc[4]), "r"((uint32_t)(acc[3] >> 32)), "r"((uint32_t)(acc[4] >> 32)));
+  const uint32_t top = ct.q_word == 4 ? __funnelshift_r(t_lo, t_hi, ct.q_bit) : __funnelshift_r(w3, t_lo, ct.q_bit);
   const uint32_t q = __umulhi(top, ct.q_mul) >> 20;
-  const unsigned long long m0 = (unsigned long long)q * ct.P[0];
-  const unsigned long long m1 = (unsigned long long)q * ct.P[1] + (m0 >> 32);
-  const unsigned long long m2 = (unsigned long long)q * ct.P[2] + (m1 >> 32);
-  const unsigned long long m3 = (unsigned long long)q * ct.P[3] + (m2 >> 32);
-  const unsigned long long m4 = (unsigned long long)q * ct.P[4] + (m3 >> 32);
-  uint32_t x0, x1, x2, x3, x4;
-  asm("sub.cc.u32 %0, %5, %10;\n\t"
-      "subc.cc.u32 %1, %6, %11;\n\t"
-      "subc.cc.u32 %2, %7, %12;\n\t"
-      "subc.cc.u32 %3, %8, %13;\n\t"
-      "subc.u32 %4, %9, %14;"
-      : "=r"(x0), "=r"(x1), "=r"(x2), "=r"(x3), "=r"(x4)
-      : "r"(S0), "r"(S1), "r"(S2), "r"(S3), "r"(S4), "r"((uint32_t)m0), "r"((uint32_t)m1), "r"((uint32_t)m2), "r"((uint32_t)m3),
-        "r"((uint32_t)m4));
   const uint32_t P0 = ct.P[0], P1 = ct.P[1], P2 = ct.P[2], P3 = ct.P[3], P4 = ct.P[4];
-  uint32_t d0, d1, d2, d3, d4, below;  // d = x - P; below = all ones if x < P
-  asm("sub.cc.u32 %0, %6, %11;\n\t"
-      "subc.cc.u32 %1, %7, %12;\n\t"
-      "subc.cc.u32 %2, %8, %13;\n\t"
-      "subc.cc.u32 %3, %9, %14;\n\t"
-      "subc.cc.u32 %4, %10, %15;\n\t"
-      "subc.u32 %5, 0, 0;"
-      : "=r"(d0), "=r"(d1), "=r"(d2), "=r"(d3), "=r"(d4), "=r"(below)
-      : "r"(x0), "r"(x1), "r"(x2), "r"(x3), "r"(x4), "r"(P0), "r"(P1), "r"(P2), "r"(P3), "r"(P4));
-  if (!below) x0 = d0, x1 = d1, x2 = d2, x3 = d3, x4 = d4;
+  const unsigned long long c0 = acc[0] + (unsigned long long)q * ct.negP[0];
+  const unsigned long long c1 = acc[1] + (unsigned long long)q * ct.negP[1];
+  const unsigned long long c2 = acc[2] + (unsigned long long)q * ct.negP[2];
+  const unsigned long long c3 = acc[3] + (unsigned long long)q * ct.negP[3];
+  const unsigned long long c4 = acc[4] + (unsigned long long)q * ct.negP[4];
+  uint32_t x0 = (uint32_t)c0, x1, x2, x3, x4;
+  asm("add.cc.u32 %0, %4, %5;\n\t"
+      "addc.cc.u32 %1, %6, %7;\n\t"
+      "addc.cc.u32 %2, %8, %9;\n\t"
+      "addc.u32 %3, %10, %11;"
+      : "=r"(x1), "=r"(x2), "=r"(x3), "=r"(x4)
+      : "r"((uint32_t)(c0 >> 32)), "r"((uint32_t)c1), "r"((uint32_t)(c1 >> 32)), "r"((uint32_t)c2), "r"((uint32_t)(c2 >> 32)), "r"((uint32_t)c3),
+        "r"((uint32_t)(c3 >> 32)), "r"((uint32_t)c4));
+  if (x4 >= P4) {  // rarely true: x >= P needs the full comparison
+    uint32_t d0, d1, d2, d3, d4, below;
+    asm("sub.cc.u32 %0, %6, %11;\n\t"
+        "subc.cc.u32 %1, %7, %12;\n\t"
+        "subc.cc.u32 %2, %8, %13;\n\t"
+        "subc.cc.u32 %3, %9, %14;\n\t"
+        "subc.cc.u32 %4, %10, %15;\n\t"
+        "subc.u32 %5, 0, 0;"
+        : "=r"(d0), "=r"(d1), "=r"(d2), "=r"(d3), "=r"(d4), "=r"(below)
+        : "r"(x0), "r"(x1), "r"(x2), "r"(x3), "r"(x4), "r"(P0), "r"(P1), "r"(P2), "r"(P3), "r"(P4));
+    if (!below) x0 = d0, x1 = d1, x2 = d2, x3 = d3, x4 = d4;
+  }
+  const uint32_t h4 = ct.halfP[4];
+  bool over = x4 > h4;
+  if (x4 == h4) {
+    [[maybe_unused]] uint32_t u0, u1, u2, u3, u4;  // only the borrow is wanted
+    uint32_t bw;
+    asm("sub.cc.u32 %0, %6, %11;\n\t"
+        "subc.cc.u32 %1, %7, %12;\n\t"
+        "subc.cc.u32 %2, %8, %13;\n\t"
+        "subc.cc.u32 %3, %9, %14;\n\t"
+        "subc.cc.u32 %4, %10, %15;\n\t"
+        "subc.u32 %5, 0, 0;"
+        : "=r"(u0), "=r"(u1), "=r"(u2), "=r"(u3), "=r"(u4), "=r"(bw)
+        : "r"(ct.halfP[0]), "r"(ct.halfP[1]), "r"(ct.halfP[2]), "r"(ct.halfP[3]), "r"(h4), "r"(x0), "r"(x1), "r"(x2), "r"(x3), "r"(x4));
+    over = bw != 0;
+  }
   uint32_t e0, e1, e2, e3, e4;  // e = P - x
   asm("sub.cc.u32 %0, %5, %10;\n\t"
       "subc.cc.u32 %1, %6, %11;\n\t"
@@ -277,25 +289,28 @@ __device__ __forceinline__ double reconstruct_lean5(const unsigned long long (&a
       "subc.u32 %4, %9, %14;"
       : "=r"(e0), "=r"(e1), "=r"(e2), "=r"(e3), "=r"(e4)
       : "r"(P0), "r"(P1), "r"(P2), "r"(P3), "r"(P4), "r"(x0), "r"(x1), "r"(x2), "r"(x3), "r"(x4));
-  [[maybe_unused]] uint32_t u0, u1, u2, u3, u4;
-  uint32_t over;  // halfP - x borrows exactly when x > P/2
-  asm("sub.cc.u32 %0, %6, %11;\n\t"
-      "subc.cc.u32 %1, %7, %12;\n\t"
-      "subc.cc.u32 %2, %8, %13;\n\t"
-      "subc.cc.u32 %3, %9, %14;\n\t"
-      "subc.cc.u32 %4, %10, %15;\n\t"
-      "subc.u32 %5, 0, 0;"
-      : "=r"(u0), "=r"(u1), "=r"(u2), "=r"(u3), "=r"(u4), "=r"(over)
-      : "r"(ct.halfP[0]), "r"(ct.halfP[1]), "r"(ct.halfP[2]), "r"(ct.halfP[3]), "r"(ct.halfP[4]), "r"(x0), "r"(x1), "r"(x2), "r"(x3),
-        "r"(x4));
-  uint32_t mag[5];
-  mag[0] = over ? e0 : x0;
-  mag[1] = over ? e1 : x1;
-  mag[2] = over ? e2 : x2;
-  mag[3] = over ? e3 : x3;
-  mag[4] = over ? e4 : x4;
-  const double r = round_scaled_fast<5>(mag, shift);
-  return over ? -r : r;
+  uint32_t m0 = over ? e0 : x0, m1 = over ? e1 : x1, m2 = over ? e2 : x2, m3 = over ? e3 : x3, m4 = over ? e4 : x4;
+  int top_bit = 159 + 1022;
+  if (m4 == 0u) {  // a magnitude below 2^128: one word up
+    m4 = m3, m3 = m2, m2 = m1, m1 = m0, m0 = 0u;
+    top_bit -= 32;
+  }
+  const int lz = __clz(m4);
+  const int e_biased = top_bit - lz - shift;  // exponent field minus one
+  if (m4 == 0u || (unsigned)e_biased >= 2046u) {  // below 2^96, or a result outside the normal range: general routine
+    const uint32_t mag[5] = {over ? e0 : x0, over ? e1 : x1, over ? e2 : x2, over ? e3 : x3, over ? e4 : x4};
+    const double r = round_scaled_fast<5>(mag, shift);
+    return over ? -r : r;
+  }
+  const uint32_t w1 = __funnelshift_l(m3, m4, lz), w0 = __funnelshift_l(m2, m3, lz);
+  const uint32_t rest = __funnelshift_l(m1, m2, lz) | m1 | m0;
+  uint32_t lo = __funnelshift_r(w0, w1, 11), hi = w1 >> 11;
+  const uint32_t sticky = ((w0 & 0x3FFu) | rest) != 0u ? 1u : 0u;
+  const uint32_t inc = (w0 >> 10) & (sticky | lo) & 1u;
+  asm("add.cc.u32 %0, %0, %2;\n\taddc.u32 %1, %1, 0;" : "+r"(lo), "+r"(hi) : "r"(inc));
+  hi += (uint32_t)e_biased << 20;
+  if (over) hi |= 0x80000000u;
+  return __hiloint2double((int)hi, (int)lo);
 }
 
 // Tail shared by the reconstruction kernels: from the 64-bit column sums acc[k] = sum_l r_l w_l[k] (weight

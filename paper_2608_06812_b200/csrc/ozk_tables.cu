@@ -254,10 +254,11 @@ bool build_crt_table(int L, CrtTable* t) {
   Big h = big_div_small(P, 2, nullptr);
   for (int i = 0; i < kCrtWords; ++i) t->halfP[i] = h.w[i];
   {
+    const int nw = big_bits(P) <= 128 ? 4 : 5;  // 2^(32 nw) - P
     uint64_t borrow = 0;
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < 5; ++i) {
       const uint64_t d = (uint64_t)0 - P.w[i] - borrow;
-      t->negP[i] = (uint32_t)d;
+      t->negP[i] = i < nw ? (uint32_t)d : 0u;
       borrow = (d >> 32) & 1u;
     }
   }
